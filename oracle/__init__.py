@@ -1,0 +1,27 @@
+"""Slow, plain fp64 CPU oracle for the CERAR coding pipeline.
+
+THIS PACKAGE IS TEST INFRASTRUCTURE.  It exists so that the CUDA library can be
+checked against something written directly from the paper.  It shares no code,
+tables or helpers with the CUDA path, imports nothing from it, and nothing in
+the product may import it: only the test-suite, the smoke check and the
+benchmark's CPU-baseline leg call into it.
+
+Contents
+--------
+protocol : chunking, encoding, the ring rounds exactly as Algorithm 1 states
+           them, the observation matrix Y_i, decoding, the matrices M_i(U),
+           the least-squares objective Phi and the rate counters.
+designs  : the coefficient constructions (multiplicative perturbation
+           construction, Vandermonde, epsilon-construction, the
+           condition-number-constrained alternating least squares heuristic).
+
+Pins (what each function is checked against, see tests/test_oracle_*.py):
+  rounds / whole pipeline : brute-force composition Y_i = G^(i) M_i(U) for
+      arbitrary U; the worked example N=4, c=5 (Fig. 1 and Sec. II-A).
+  MPC / Vandermonde / epsilon designs : Prop. 1, Prop. 2, Theorem 1's closed
+      form, Eq. (error_scaling), Theorem 2 / Corollary 1 scaling laws, the
+      finite-difference identity (Lemma 2) and the printed F_3.
+  kappa-constrained design : invariants only (spectral interval, kappa bound,
+      monotone least-squares steps).  The fitted U, R values themselves have no
+      published counterpart: PARITY UNPINNED for `designs.kappa_constrained`.
+"""

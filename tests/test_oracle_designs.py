@@ -1,0 +1,302 @@
+"""Pins for oracle.designs: identities and scaling laws the paper states."""
+import os
+from math import ceil
+
+import mpmath as mp
+import numpy as np
+import pytest
+
+from oracle import designs as Dz
+from oracle import protocol as P
+
+
+def _maxabs(M):
+    return max(abs(M[i, j]) for i in range(M.rows) for j in range(M.cols))
+
+
+def _rng_B(N, c, seed=0):
+    return np.random.default_rng(seed).standard_normal((N, c))
+
+
+# ------------------------------------------------------------------ MPC core
+
+@pytest.mark.parametrize("N,c", [(2, 3), (3, 3), (4, 5), (4, 10), (5, 12)])
+def test_prop1_block_identity_diagonal_D(N, c):
+    """U_{i-1-s} W_s(R_i) = I (s >= i) or D^{-1} (s < i)."""
+    des = Dz.epsilon(N, c, 3e-2, _rng_B(N, c, N + c))
+    with mp.workdps(Dz.DEFAULT_DPS):
+        Dinv = mp.inverse(des.Dmat_mp)
+        for (i, s), blk in Dz.block_products_mp(des).items():
+            ref = mp.eye(c) if s >= i else Dinv
+            assert _maxabs(blk - ref) < mp.mpf(10) ** (-60)
+
+
+def test_prop1_and_prop2_full_matrix_D():
+    """Same identities with a non-diagonal perturbation H (general path with
+    negative powers of D)."""
+    N, c, eps = 3, 5, 2e-2
+    rng = np.random.default_rng(42)
+    B = rng.standard_normal((N, c))
+    H = rng.standard_normal((c, c))
+    H /= np.linalg.norm(H, 2)
+    Dm = np.eye(c) + eps * H
+    des = Dz.mpc(B.tolist(), mp.matrix(Dm.tolist()), N, c)
+    with mp.workdps(Dz.DEFAULT_DPS):
+        Dinv = mp.inverse(des.Dmat_mp)
+        for (i, s), blk in Dz.block_products_mp(des).items():
+            ref = mp.eye(c) if s >= i else Dinv
+            assert _maxabs(blk - ref) < mp.mpf(10) ** (-60)
+        E = Dinv - mp.eye(c)
+        closed = mp.mpf(N * (N - 1)) / 2 * sum(E[a, b] ** 2 for a in range(c) for b in range(c))
+        assert abs(Dz.phi_mp(des) - closed) < mp.mpf(10) ** (-60)
+
+
+def test_window_shift_identity():
+    """A_{l+N} = A_l D."""
+    N, c, eps = 4, 6, 1e-2
+    B = _rng_B(N, c, 1)
+    with mp.workdps(Dz.DEFAULT_DPS):
+        Dv = [1 + mp.mpf(eps) * mp.mpf(h) for h in Dz.default_h(c)]
+        Bm = mp.matrix(B.tolist())
+        for l in (-3, 0, 2, 5):
+            A0 = Dz.window_mp(Bm, Dv, N, c, l)
+            A1 = Dz.window_mp(Bm, Dv, N, c, l + N)
+            assert _maxabs(A1 - A0 * mp.diag(Dv)) < mp.mpf(10) ** (-80)
+
+
+def test_prop2_closed_form_value():
+    """Phi = N(N-1)/2 ||D^{-1} - I||_F^2, including the fp64 evaluation for a
+    mild design."""
+    N, c, eps = 4, 5, 1e-2
+    des = Dz.epsilon(N, c, eps, _rng_B(N, c))
+    closed = N * (N - 1) / 2 * sum((1 / (1 + eps * h) - 1) ** 2 for h in Dz.default_h(c))
+    assert float(Dz.phi_mp(des)) == pytest.approx(closed, rel=1e-12)
+    assert P.phi(des.U, des.R) == pytest.approx(closed, rel=1e-6)
+
+
+def test_decoder_rows_and_windows():
+    """R_i[l,:] = a_{l-i}; W_s(R_i) = A_{s-i}; U_k A_{N-1-k} = I."""
+    N, c = 4, 6
+    B = _rng_B(N, c, 2)
+    des = Dz.epsilon(N, c, 0.05, B)
+    with mp.workdps(Dz.DEFAULT_DPS):
+        Dv = [1 + mp.mpf(0.05) * mp.mpf(h) for h in Dz.default_h(c)]
+        Bm = mp.matrix(B.tolist())
+        for i in range(N):
+            for s in range(N):
+                A = Dz.window_mp(Bm, Dv, N, c, s - i)
+                assert _maxabs(des.R_mp[i][s:s + c, :] - A) < mp.mpf(10) ** (-80)
+        for k in range(N):
+            A = Dz.window_mp(Bm, Dv, N, c, N - 1 - k)
+            assert _maxabs(des.U_mp[k] * A - mp.eye(c)) < mp.mpf(10) ** (-60)
+    # first rows of the sequence are the rows of B itself
+    np.testing.assert_allclose(des.R[0][:N, :], B, rtol=1e-15)
+
+
+def test_phi_positive_when_c_exceeds_N():
+    """Lemma 1: no finite design reaches Phi = 0 for c > N."""
+    for (N, c) in [(3, 4), (4, 9)]:
+        for eps in (1e-1, 1e-3, 1e-6):
+            des = Dz.epsilon(N, c, eps, _rng_B(N, c))
+            assert Dz.phi_mp(des) > 0
+        assert Dz.phi_mp(Dz.vandermonde(N, c, 1e-3)) > 0
+
+
+# ------------------------------------------------------------------ Vandermonde
+
+@pytest.mark.parametrize("N,c,tau", [(4, 6, 0.1), (3, 5, 0.02), (4, 8, 0.1)])
+def test_vandermonde_phi_closed_form(N, c, tau):
+    des = Dz.vandermonde(N, c, tau)
+    xi = Dz.default_xi(c)
+    closed = N * (N - 1) / 2 * sum((np.exp(-N * tau * x) - 1) ** 2 for x in xi)
+    assert float(Dz.phi_mp(des)) == pytest.approx(closed, rel=1e-12)
+
+
+def test_vandermonde_leading_term_and_limit():
+    """Phi = N^3 (N-1)/2 tau^2 sum xi^2 + O(tau^3): the ratio to the leading
+    term tends to 1 and Phi -> 0 as tau -> 0."""
+    N, c = 4, 6
+    xi = Dz.default_xi(c)
+    lead = lambda t: N ** 3 * (N - 1) / 2 * t * t * sum(x * x for x in xi)
+    prev = None
+    for tau in (1e-1, 1e-2, 1e-3):
+        ph = float(Dz.phi_mp(Dz.vandermonde(N, c, tau)))
+        ratio = ph / lead(tau)
+        assert abs(ratio - 1) < 30 * tau
+        if prev is not None:
+            assert ph < prev / 50
+        prev = ph
+    # worked value: N=4, c=6, tau=0.1 gives 2.8952 against a leading term 2.688
+    assert float(Dz.phi_mp(Dz.vandermonde(4, 6, 0.1))) == pytest.approx(2.8952, abs=5e-4)
+    assert lead(0.1) == pytest.approx(2.688, abs=1e-3)
+
+
+def test_vandermonde_entries_and_conditioning():
+    N, c, tau = 3, 5, 0.2
+    des = Dz.vandermonde(N, c, tau)
+    z = np.exp(tau * np.array(Dz.default_xi(c)))
+    # R_0 rows are a_l = [z_j^l], l = 0..L
+    for l in range(des.L + 1):
+        np.testing.assert_allclose(des.R[0][l], z ** l, rtol=1e-14)
+    # R_i rows are a_{l-i}, negative powers included
+    np.testing.assert_allclose(des.R[2][0], z ** (-2.0), rtol=1e-14)
+    # kappa(U_k) grows without bound as tau decreases (Remark 2)
+    ks = [max(P.kappa2(u) for u in Dz.vandermonde(N, c, t).U) for t in (0.4, 0.2, 0.1, 0.05)]
+    assert all(b > 5 * a for a, b in zip(ks, ks[1:]))
+
+
+# ------------------------------------------------------------------ epsilon-construction
+
+def test_epsilon_phi_bound_and_quadratic_scaling():
+    N, c = 4, 10
+    B = _rng_B(N, c)
+    h = np.array(Dz.default_h(c))
+    vals = []
+    for eps in (1e-1, 1e-2, 1e-3):
+        ph = float(Dz.phi_mp(Dz.epsilon(N, c, eps, B)))
+        bound = N * (N - 1) / 2 * eps ** 2 * np.sum(h ** 2) / (1 - eps * np.max(np.abs(h))) ** 2
+        assert 0 < ph <= bound * (1 + 1e-12)
+        vals.append(ph)
+    assert vals[0] / vals[1] == pytest.approx(100, rel=0.3)
+    assert vals[1] / vals[2] == pytest.approx(100, rel=0.03)
+
+
+@pytest.mark.parametrize("N,c", [(4, 10), (4, 8), (3, 7)])
+def test_singular_value_hierarchy_and_kappa_slope(N, c):
+    """Theorem 2 / Corollary 1: the singular values of A_l(eps) fall in groups
+    Theta(eps^j) with N members for j < beta and s members at j = beta;
+    kappa_2(A_l) = Theta(eps^-r*), r* = ceil(c/N) - 1."""
+    beta, s = divmod(c, N)
+    rstar = ceil(c / N) - 1
+    B = _rng_B(N, c)
+    h = Dz.default_h(c)
+    kap = {}
+    svs = {}
+    with mp.workdps(Dz.DEFAULT_DPS):
+        Bm = mp.matrix(B.tolist())
+        for eps in (1e-3, 1e-4, 1e-5):
+            Dv = [1 + mp.mpf(eps) * mp.mpf(x) for x in h]
+            for l in range(N):
+                sv = [float(v) for v in Dz.singular_values_mp(Dz.window_mp(Bm, Dv, N, c, l))]
+                svs[(eps, l)] = sv
+                kap.setdefault(l, []).append(sv[0] / sv[-1])
+    expect = sorted([j for j in range(beta) for _ in range(N)] + [beta] * s)
+    for l in range(N):
+        # exponent of eps carried by the t-th singular value, from one decade of eps
+        expo = [np.log10(a / b) for a, b in zip(svs[(1e-4, l)], svs[(1e-5, l)])]
+        assert [int(round(e)) for e in expo] == expect, (l, expo)
+        assert max(abs(e - round(e)) for e in expo) < 0.1
+    for l, ks in kap.items():
+        slope1 = np.log10(ks[1] / ks[0])      # per decade of eps
+        slope2 = np.log10(ks[2] / ks[1])
+        assert slope1 == pytest.approx(rstar, abs=0.15)
+        assert slope2 == pytest.approx(rstar, abs=0.05)
+
+
+def test_worked_kappa_values_n4_c10():
+    """kappa_2 of the encoders for N=4, c=10, B from numpy seed 0, H =
+    diag(linspace(-1,1)): decades of eps change kappa by 10^r* = 100."""
+    N, c = 4, 10
+    B = _rng_B(N, c)
+    ks = []
+    for eps in (1e-1, 1e-2, 1e-3):
+        des = Dz.epsilon(N, c, eps, B)
+        with mp.workdps(Dz.DEFAULT_DPS):
+            k = max(float(sv[0] / sv[-1]) for sv in (Dz.singular_values_mp(u) for u in des.U_mp))
+        ks.append(k)
+    assert ks[1] / ks[0] == pytest.approx(100, rel=0.25)
+    assert ks[2] / ks[1] == pytest.approx(100, rel=0.05)
+
+
+def test_kappa_M_bound():
+    """kappa_2(M_j) <= sqrt(N) max sigma_max(U) / min sigma_min(U), and
+    sigma_max(M_j) >= max_k sigma_max(U_k) (appendix on U vs M conditioning)."""
+    N, c = 4, 7
+    des = Dz.epsilon(N, c, 1e-1, _rng_B(N, c))
+    smax = max(np.linalg.svd(u, compute_uv=False)[0] for u in des.U)
+    smin = min(np.linalg.svd(u, compute_uv=False)[-1] for u in des.U)
+    for j in range(N):
+        sv = np.linalg.svd(P.m_matrix(des.U, j), compute_uv=False)
+        assert sv[0] / sv[-1] <= np.sqrt(N) * smax / smin * (1 + 1e-9)
+        assert sv[0] >= smax * (1 - 1e-9)
+        assert sv[-1] >= smin * (1 - 1e-9)
+
+
+def test_finite_difference_matrix(golden_dir):
+    F3 = np.loadtxt(os.path.join(golden_dir, "f3.txt"), comments="#")
+    np.testing.assert_array_equal(Dz.finite_difference_matrix(3), F3)
+    for n in range(1, 9):
+        assert round(np.linalg.det(Dz.finite_difference_matrix(n).astype(float))) == 1
+
+
+def test_finite_difference_identity():
+    """Lemma 2: sum_k (-1)^(j-k) C(j,k) b D^(m+k) = eps^j b D^m H^j, and the
+    factorisation F Pi A_l = Lambda K_l on a full window."""
+    rng = np.random.default_rng(4)
+    c, eps = 6, 1e-2
+    H = rng.standard_normal((c, c))
+    Dm = np.eye(c) + eps * H
+    b = rng.standard_normal(c)
+    for m in (0, 1, 2):
+        for j in range(4):
+            F = Dz.finite_difference_matrix(j + 1)
+            lhs = sum(F[j, k] * b @ np.linalg.matrix_power(Dm, m + k) for k in range(j + 1))
+            rhs = eps ** j * b @ np.linalg.matrix_power(Dm, m) @ np.linalg.matrix_power(H, j)
+            np.testing.assert_allclose(lhs, rhs, atol=1e-12 * max(1, np.abs(lhs).max()))
+    # whole window, diagonal H, N=3, c=7 (beta=2, s=1), l=1
+    N, c, l, eps = 3, 7, 1, 1e-3
+    B = _rng_B(N, c, 8)
+    h = Dz.default_h(c)
+    with mp.workdps(60):
+        Bm = mp.matrix(B.tolist())
+        Dv = [1 + mp.mpf(eps) * mp.mpf(x) for x in h]
+        A = Dz.window_mp(Bm, Dv, N, c, l, 60)
+        idx = list(range(l, l + c))
+        for alpha in range(N):
+            rows = [t for t, jj in enumerate(idx) if jj % N == alpha]   # grouped by remainder
+            n = len(rows)
+            m0 = 0 if alpha >= l else 1
+            F = Dz.finite_difference_matrix(n)
+            for j in range(n):
+                lhs = [sum(int(F[j, k]) * A[rows[k], col] for k in range(j + 1)) for col in range(c)]
+                rhs = [mp.mpf(eps) ** j * Bm[alpha, col] * Dv[col] ** m0 * mp.mpf(h[col]) ** j for col in range(c)]
+                assert max(abs(a - b) for a, b in zip(lhs, rhs)) < mp.mpf(10) ** (-50)
+
+
+# ------------------------------------------------------------------ kappa-constrained
+
+def test_kappa_constrained_invariants():
+    N, c, C = 4, 12, 1e4
+    des = Dz.kappa_constrained(N, c, C, _rng_B(N, c), iters=40)
+    a0, b0 = des.info["a0"], des.info["b0"]
+    assert np.sqrt(N) * b0 / a0 <= C * (1 + 1e-12)
+    for u in des.U:
+        sv = np.linalg.svd(u, compute_uv=False)
+        assert sv[-1] >= a0 * (1 - 1e-9) and sv[0] <= b0 * (1 + 1e-9)
+    for i in range(N):
+        assert P.kappa2(P.m_matrix(des.U, i)) <= C
+    # least-squares steps never increase Phi (before the projection)
+    for before, after_U, _ in des.info["steps"]:
+        assert after_U <= before * (1 + 1e-9) + 1e-12
+    # R is the least-squares decoder for the final U
+    for i in range(N):
+        M = P.m_matrix(des.U, i)
+        grad = M.T @ (M @ des.R[i] - P.target(N, c))
+        assert np.abs(grad).max() < 1e-6 * max(1.0, np.abs(M).max() ** 2)
+    ph = P.phi(des.U, des.R)
+    assert 0 < ph < 1.0
+    # improves on simply clipping the initial design
+    assert ph <= des.info["phi_history"][0] * (1 + 1e-9)
+    # the error it gives on i.i.d. gradients is a few percent (same order as the
+    # paper's training-time figure for N=4, c=12; plausibility only)
+    rng = np.random.default_rng(1)
+    g = [rng.standard_normal(c * 64) for _ in range(N)]
+    res = P.allreduce(g, des.U, des.R)
+    err = max(P.rel_l2(res["out"][i], P.exact_sum(g)) for i in range(N))
+    assert 1e-3 < err < 0.1
+
+
+def test_surrogate_is_well_conditioned():
+    des = Dz.custom_orthogonal(4, 8, np.random.default_rng(0))
+    for u in des.U:
+        assert P.kappa2(u) == pytest.approx(1.0, abs=1e-9)
