@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the CERAR hot path (encode + L ring rounds + decode) on B200.
+
+One "step" is one aggregation: every logical worker's gradient is encoded, the
+L = c+N-2 ring rounds run, and every worker decodes its approximate mean.
+Default workload: the third configuration (N=8, c=32, epsilon-construction
+eps=1e-2, d=1,414,647,808 fp32 per worker, 24 layer-shaped Gaussian blocks),
+the "sim time at d=1.4B" point of the metric.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` is algorithmic GB/s over the whole job:
+N_workers*(8c+3N-8)*p*4 bytes per aggregation (every logical buffer touched once
+per use) divided by the device time per step, summed over ranks.  With more
+than one GPU every rank runs its own replica of the workload (the path has no
+exchange step: positions are independent), i.e. weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "cerar_encode_rounds_decode_hbm_gbps"
+UNIT = "GB/s"
+# DRAM bytes per ring-round launch measured by ncu, per (worker x position), on a
+# smaller case of the same kernel (see profiles/); None until a capture exists.
+NCU_ROUND_DRAM_BYTES_PER_WORKER_POSITION = None
+
+
+def algorithmic_bytes(N, c, p):
+    """Per aggregation, all workers: encode 2c, rounds 4c+2N-7, decode 2c+N-1 row
+    passes of p fp32 per worker."""
+    enc = 2 * c
+    rnd = 4 * c + 2 * N - 7
+    dec = 2 * c + N - 1
+    return {"encode": 4 * N * p * enc, "rounds": 4 * N * p * rnd, "decode": 4 * N * p * dec,
+            "total": 4 * N * p * (enc + rnd + dec)}
+
+
+def round_bytes(N, c, p, k):
+    terms = (1 if k >= 2 else 0) + (1 if k - 1 >= N else 0) + (1 if k <= c else 0) + 1
+    return 4 * N * p * terms
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            t = [x.strip() for x in line.split(",")]
+            if len(t) < 7:
+                continue
+            try:
+                sm.append(float(t[0])); mx.append(float(t[1])); power.append(float(t[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, t[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            # under load = samples in the upper half of the power range
+            thr = (max(power) + min(power)) / 2 if power else 0
+            loaded = [s for s, w in zip(sm, power) if w >= thr] or sm
+            out.update(sm_mhz=float(np.median(loaded)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=float(max(power)))
+        return out
+
+
+def build_design_oracle(cfg, B):
+    from oracle import designs as Dz
+    if cfg["kind"] == "vandermonde":
+        return Dz.vandermonde(cfg["N"], cfg["c"], cfg["param"])
+    if cfg["kind"] == "epsilon":
+        return Dz.epsilon(cfg["N"], cfg["c"], cfg["param"], B)
+    return Dz.kappa_constrained(cfg["N"], cfg["c"], cfg["param"], B)
+
+
+def oracle_step(des, g_sub, scale):
+    from oracle import protocol as P
+    return P.allreduce([x for x in g_sub], des.U, des.R, scale)
+
+
+def cpu_baseline(cfg, des, p_sample, seed=0):
+    """Times the oracle, as it stands, on the first p_sample positions of the
+    workload (all N workers, all c chunks)."""
+    from paper_2609_23898_b200 import inputs
+    N, c = cfg["N"], cfg["c"]
+    kw = {"std": cfg["std"]} if "std" in cfg else {}
+    g = inputs.gradients_numpy(N, c * p_sample, cfg["workload"], seed=seed, **kw).astype(np.float64)
+    t0 = time.perf_counter()
+    oracle_step(des, g, 1.0 / N)
+    dt = time.perf_counter() - t0
+    ab = algorithmic_bytes(N, c, p_sample)["total"]
+    try:
+        from threadpoolctl import threadpool_info
+        thr = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        thr = os.cpu_count() or 1
+    return {"value": ab / dt / 1e9, "unit": UNIT, "cores": int(thr), "kind": "oracle",
+            "sample": f"first {p_sample} of p={cfg['d'] // c} positions, all {N} workers and {c} chunks; "
+                      f"{dt:.2f} s of numpy fp64", "seconds": dt}
+
+
+def run_reference(args, cfg):
+    """--impl reference: the CPU oracle timed on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2609_23898_b200 import inputs
+    N, c, d = cfg["N"], cfg["c"], cfg["d"]
+    B = inputs.base_matrix(N, c, 0)
+    des = build_design_oracle(cfg, B)
+    p_sample = min(d // c, args.ref_positions)
+    for _ in range(args.warmup):
+        cpu_baseline(cfg, des, max(1, p_sample // 8))
+    times, base = [], None
+    for _ in range(args.steps):
+        base = cpu_baseline(cfg, des, p_sample)
+        times.append(base["seconds"])
+    dt = float(np.mean(times))
+    val = algorithmic_bytes(N, c, p_sample)["total"] / dt / 1e9
+    base["value"] = val
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(args.workload, cfg), "sample_positions": p_sample},
+            "cpu_baseline": base,
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def workload_name(key, cfg):
+    return (f"{key}: N={cfg['N']} c={cfg['c']} {cfg['kind']}({cfg['param']:g}) d={cfg['d']} fp32/worker "
+            f"{cfg['workload']} gradients")
+
+
+def sampled_parity(cfg, des, plan, grads, ws, out, scale, n_tiles=6, tile=512):
+    """Full-size check on sampled position tiles: positions are independent, so
+    the oracle runs the whole protocol on the sampled columns only."""
+    import torch
+    from oracle import protocol as P
+    N, c, d = cfg["N"], cfg["c"], cfg["d"]
+    p, L = d // c, c + N - 2
+    rng = np.random.default_rng(123)
+    starts = sorted(set([0, max(0, p - tile)] + [int(x) for x in rng.integers(0, max(1, p - tile), n_tiles)]))
+    idx = np.concatenate([np.arange(s, min(s + tile, p)) for s in starts])
+    idx_t = torch.from_numpy(idx).to(grads.device)
+    g_sub = grads.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy().astype(np.float64)
+    ora = P.allreduce([x for x in g_sub], des.U, des.R, scale)
+    wsv = ws.view(N, c + N, p)
+    rows = list(range(L)) + [L + 1]
+    Y_dev = wsv[:, rows, :][:, :, idx_t].cpu().numpy()                    # (N, L+1, S)
+    Y_ora = np.stack([ora["Y"][i].T for i in range(N)])
+    out_dev = out.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy()
+    kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+    return {"positions": int(idx.size), "rel_l2_Y": P.rel_l2(Y_dev, Y_ora),
+            "rel_l2_out_max": max(P.rel_l2(out_dev[i], ora["out"][i]) for i in range(N)),
+            "kappa_M": kap, "kappa_times_2^-24": kap * 2.0 ** -24,
+            "rel_l2_oracle_vs_exact_mean": max(P.rel_l2(ora["out"][i], P.exact_sum(list(g_sub)) * scale)
+                                               for i in range(N))}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3")
+    ap.add_argument("--d", type=int, default=0, help="override d per worker (multiple of c)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parity", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--ref-positions", type=int, default=1 << 20)
+    ap.add_argument("--kernel-mode", type=int, default=0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2609_23898_b200 import inputs
+    cfg = dict(inputs.CONFIGS[args.workload])
+    if args.d:
+        cfg["d"] = args.d
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_23898_b200 import cerar
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    N, c, d = cfg["N"], cfg["c"], cfg["d"]
+    p, L = d // c, c + N - 2
+    scale = 1.0 / N
+    B = inputs.base_matrix(N, c, 0)
+    kinds = {"vandermonde": cerar.VANDERMONDE, "epsilon": cerar.EPSILON, "kappa": cerar.KAPPA}
+    plan = cerar.Plan.create(N, c, kinds[cfg["kind"]], cfg["param"], B=B)
+    plan.set_kernel_mode(args.kernel_mode)
+
+    grads = torch.empty(N * d, dtype=torch.float32, device=dev)
+    kw = {"std": cfg["std"]} if "std" in cfg else {}
+    inputs.fill_gradients_torch([grads[i * d:(i + 1) * d] for i in range(N)], cfg["workload"], seed=rank, **kw)
+    ws = torch.empty(plan.workspace_bytes(d) // 4, dtype=torch.float32, device=dev)
+    out = torch.empty(N * d, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    ab = algorithmic_bytes(N, c, p)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
+    torch.cuda.synchronize()
+    plan.device_status(stream)
+
+    # ---- timed region: K steps, each the C-ABI sequence encode, rounds 1..L, decode
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 3)] for _ in range(K)]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    sync_all()
+    launches0 = plan.launch_count()
+    for s in range(K):
+        e = ev[s]
+        e[0].record()
+        plan.encode(grads, d, ws, d, stream)
+        e[1].record()
+        for k in range(1, L + 1):
+            plan.ring_round(ws, d, k, stream)
+            e[1 + k].record()
+        plan.decode(ws, out, d, d, scale, stream)
+        e[L + 2].record()
+    sync_all()
+    launches = plan.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    plan.device_status(stream)
+    total_ms = ev[0][0].elapsed_time(ev[K - 1][L + 2])
+    enc_ms = float(np.mean([ev[s][0].elapsed_time(ev[s][1]) for s in range(K)]))
+    dec_ms = float(np.mean([ev[s][L + 1].elapsed_time(ev[s][L + 2]) for s in range(K)]))
+    rnd_ms = [float(np.mean([ev[s][k].elapsed_time(ev[s][k + 1]) for s in range(K)])) for k in range(1, L + 1)]
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = float(t.item()) / K
+    value = world * ab["total"] / (ms_per_step * 1e-3) / 1e9
+
+    peak, peak_kind = load_peaks()
+    rounds_bytes = sum(round_bytes(N, c, p, k) for k in range(1, L + 1))
+    assert rounds_bytes == ab["rounds"]
+    rounds_ms = float(sum(rnd_ms))
+    shares = {"round_kernel": rounds_ms, "encode": enc_ms, "decode": dec_ms}
+    dominant = max(shares, key=shares.get)
+    dom_bytes = {"round_kernel": ab["rounds"] / L, "encode": ab["encode"], "decode": ab["decode"]}[dominant]
+    dom_ms = {"round_kernel": rounds_ms / L, "encode": enc_ms, "decode": dec_ms}[dominant]
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    traffic = None
+    if dominant == "round_kernel" and NCU_ROUND_DRAM_BYTES_PER_WORKER_POSITION is not None:
+        traffic = NCU_ROUND_DRAM_BYTES_PER_WORKER_POSITION * N * p
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": dom_ms,
+                "per_kernel": {
+                    "encode": {"ms": enc_ms, "GBps": ab["encode"] / enc_ms / 1e6, "launches_per_step": 1},
+                    "round_kernel": {"ms_total": rounds_ms, "GBps": ab["rounds"] / rounds_ms / 1e6,
+                                     "launches_per_step": L},
+                    "decode": {"ms": dec_ms, "GBps": ab["decode"] / dec_ms / 1e6, "launches_per_step": 1}},
+                "whole_path_frac": value / world / peak}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "seconds_per_aggregation": ms_per_step * 1e-3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": workload_name(args.workload, cfg), "N": N, "c": c, "L": L, "d": d,
+                       "scale": "1/N", "replicas": world, "l2": "inputs larger than L2" if ab["total"] / (L + 2) > 2.6e8
+                       else "working set may be L2 resident",
+                       "buffers": "out of place: grads, workspace and output are separate device buffers"},
+            "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks}
+
+    if rank == 0 and not args.no_parity:
+        des = build_design_oracle(cfg, B)
+        line["parity"] = sampled_parity(cfg, des, plan, grads, ws, out, scale)
+    else:
+        des = None
+
+    # ---- end to end through the host-buffer entry point (pinned host memory)
+    if not args.no_e2e:
+        need = 2 * N * d * 4
+        avail = 0
+        try:
+            for ln in open("/proc/meminfo"):
+                if ln.startswith("MemAvailable"):
+                    avail = int(ln.split()[1]) * 1024
+        except OSError:
+            pass
+        d_e2e = d
+        while need > 0.6 * avail / max(1, world) and d_e2e > c * 1024:
+            d_e2e = (d_e2e // 2 // c) * c
+            need = 2 * N * d_e2e * 4
+        del out
+        torch.cuda.empty_cache()
+        h_in = torch.empty(N * d_e2e, dtype=torch.float32).pin_memory()
+        h_out = torch.empty(N * d_e2e, dtype=torch.float32).pin_memory()
+        pe = d_e2e // c
+        # host inputs: the same device gradients (first d_e2e/c positions of every chunk)
+        h_in.view(N, c, pe).copy_(grads.view(N, c, p)[:, :, :pe])
+        torch.cuda.synchronize()
+        ksteps = max(1, args.e2e_steps)
+        plan.allreduce_sim_host(h_in, d_e2e, h_out, d_e2e, ws, d_e2e, scale, stream)      # warm-up
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(ksteps):
+            plan.allreduce_sim_host(h_in, d_e2e, h_out, d_e2e, ws, d_e2e, scale, stream)
+        e1.record()
+        sync_all()
+        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        ms_e2e = float(te.item()) / ksteps
+        abe = algorithmic_bytes(N, c, pe)["total"]
+        line["e2e"] = {"value": world * abe / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+                       "h2d_bytes_per_step": N * d_e2e * 4, "d2h_bytes_per_step": N * d_e2e * 4,
+                       "ms_per_step": ms_e2e, "steps": ksteps, "d": d_e2e,
+                       "note": "pinned host gradients -> device workspace rows, in-place pipeline, results back to "
+                               "pinned host; PCIe copies inside the timed region"}
+        plan.device_status(stream)
+        del h_in, h_out
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        if des is None:
+            des = build_design_oracle(cfg, B)
+        line["cpu_baseline"] = cpu_baseline(cfg, des, min(p, args.ref_positions))
+
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,206 @@
+/*
+ * cerar.h - C ABI of the CERAR coding pipeline for one B200.
+ *
+ * CERAR (communication-efficient ring all-reduce) lets N ring workers, each
+ * holding a length-d gradient split into c chunks of p = d/c values, obtain an
+ * approximation of the sum of all gradients in L = c + N - 2 rounds of
+ * length-p messages (problem statement, Sec. I; protocol, Sec. II).  In this
+ * library the N logical workers live in one GPU's memory and a ring hand-off
+ * is a store into the neighbour's buffer; there is no inter-GPU transport.
+ *
+ * Conventions for every call
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA
+ *     device memory on the device that was current when the plan was created.
+ *   - The caller owns every data buffer.  The library owns the plan (host fp64
+ *     matrices and fp32 device copies of them) and allocates nothing in the
+ *     data-path calls (encode, ring_round, decode, allreduce_sim).
+ *   - Data-path calls are asynchronous on the given stream and report
+ *     argument and launch errors only.  Nothing throws across this boundary.
+ *   - All matrices are row-major.  Gradients are fp32 on the device; the
+ *     coefficient matrices are built in fp64 on the host and rounded to fp32
+ *     for the device.
+ *
+ * Workspace layout (device, fp32): worker i owns a row-major (c+N) x p matrix
+ * at ws + i*(c+N)*p.  Row ("slot") s of worker i holds
+ *     s = 0 .. N-2      : B_{i,1} .. B_{i,N-1}  (first N-1 received messages)
+ *     s = N-1           : C_i                    (landing slot of message N)
+ *     s = N .. N+c-1    : D_{i,1} .. D_{i,c}     (encoded vectors delta_{i,j})
+ * which is exactly the (c+N) p values per worker of the paper's storage rate
+ * 1 + N/c (Sec. II-B).  Message k of worker i-1 lands in slot k-1 of worker i,
+ * so after L rounds slots 0..L-1 hold y_{i,1}..y_{i,L} in order and slot L+1
+ * holds y_{i,L+1} = delta_{i,c}; slot L keeps a stale delta_{i,c-1} that the
+ * decoder does not read.
+ */
+#ifndef CERAR_H_
+#define CERAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cerar_plan cerar_plan_t;          /* opaque, library-owned */
+typedef struct CUstream_st* cerar_stream_t;      /* a cudaStream_t */
+
+typedef enum {
+    CERAR_OK = 0,
+    CERAR_ERR_INVALID_ARG = 1,   /* null pointer, N < 2, c < N, bad parameter          */
+    CERAR_ERR_SHAPE = 2,         /* c does not divide d, stride too small, d <= 0       */
+    CERAR_ERR_SINGULAR = 3,      /* non-finite coefficients or a singular window        */
+    CERAR_ERR_NOT_CONVERGED = 4, /* kappa design: constraint not met after the last step */
+    CERAR_ERR_STATE = 5,         /* rounds out of order, decode before the last round    */
+    CERAR_ERR_CUDA = 6,          /* a CUDA runtime call failed, or no device             */
+    CERAR_ERR_NOMEM = 7,
+    CERAR_ERR_TIMEOUT = 8
+} cerar_status_t;
+
+typedef enum {
+    CERAR_VANDERMONDE = 0,   /* param = tau   (Sec. II-B.2)                     */
+    CERAR_EPSILON = 1,       /* param = eps   (Sec. II-C, D = I + eps H)        */
+    CERAR_KAPPA = 2          /* param = C, the bound on kappa_2(M_i) (Sec. II-D) */
+} cerar_construction_t;
+
+/* Optional settings for cerar_plan_create_ex.  Zero-initialise for defaults. */
+typedef struct {
+    uint64_t      seed;       /* seed of the built-in N(0,1) generator used for B when B == NULL */
+    const double* B;          /* host, N x c: base matrix of the epsilon / kappa designs, or NULL */
+    const double* h;          /* host, length c: diag(H) (epsilon, kappa) or the nodes xi_j
+                                 (Vandermonde); NULL = c equally spaced values in [-1, 1]        */
+    double        eps_init;   /* kappa design: eps of the initial epsilon-construction; 0 = 0.1  */
+    int           als_iters;  /* kappa design: maximum ALS iterations; 0 = 200                   */
+    double        als_tol;    /* kappa design: stop when Phi changes by less (relative); 0 = 1e-6 */
+    int           host_only;  /* 1 = never touch CUDA (plan usable for get_U / get_R / info only) */
+} cerar_options_t;
+
+typedef struct {
+    int      N, c, L;
+    int      construction;       /* cerar_construction_t, or 3 for a custom plan            */
+    double   param;
+    double   phi;                /* Phi(U,R) = sum_i ||M_i(U) R_i - T||_F^2 (Eq. F_unreg);
+                                    closed form of Prop. 2 for the explicit constructions   */
+    double   kappa_U_max;        /* max_k kappa_2(U_k)                                       */
+    double   kappa_M_max;        /* max_i kappa_2(M_i(U))                                    */
+    double   inv_residual_max;   /* max_k ||U_k A_{N-1-k} - I||_max (explicit constructions) */
+    double   abs_U_max, abs_R_max;
+    int      als_iters_done;
+    int      on_device;          /* 1 if fp32 copies were uploaded                            */
+} cerar_plan_info_t;
+
+typedef struct {
+    int      encoded;                      /* 1 after cerar_encode                          */
+    int      rounds_done;                  /* k of the last completed cerar_ring_round      */
+    uint64_t bytes_forwarded_per_worker;   /* sum over completed rounds of 4 p              */
+    uint64_t bytes_forwarded_last_round;   /* 4 p                                           */
+    uint64_t bytes_stored_per_worker;      /* 4 p (c + N)                                   */
+    uint64_t bytes_gradient;               /* 4 d, the denominator of both rates            */
+} cerar_counters_t;
+
+/* ---- plan: coefficient matrices U_0..U_{N-1} (c x c) and R_0..R_{N-1} ((L+1) x c) ----
+ *
+ * cerar_plan_create builds the multiplicative perturbation construction of
+ * Sec. II-B.1 (a_{r+mN} = b_r D^m, A_l = [a_l; ..; a_{l+c-1}], U_k = A_{N-1-k}^{-1},
+ * R_i[l,:] = a_{l-i}) for the Vandermonde (Sec. II-B.2) or epsilon (Sec. II-C)
+ * choice of (B, D), or runs the alternating least-squares heuristic of Sec. II-D
+ * started from an epsilon-construction.  Requires 2 <= N <= c.  On success *out
+ * is a new plan; on failure *out is NULL.  If a CUDA device is available (and
+ * host_only is 0) fp32 copies are uploaded to the current device. */
+cerar_status_t cerar_plan_create(int N, int c, cerar_construction_t kind, double param,
+                                 cerar_plan_t** out);
+cerar_status_t cerar_plan_create_ex(int N, int c, cerar_construction_t kind, double param,
+                                    const cerar_options_t* opt, cerar_plan_t** out);
+/* Plan from caller-supplied matrices (host, fp64): U is N*c*c, R is N*(L+1)*c.
+ * Any finite numbers are accepted: the data path is the protocol of Algorithm 1
+ * with these coefficients, whatever they decode to. */
+cerar_status_t cerar_plan_create_custom(int N, int c, const double* U, const double* R,
+                                        int host_only, cerar_plan_t** out);
+void           cerar_plan_destroy(cerar_plan_t* plan);
+
+/* Copies of the fp64 matrices (host buffers of c*c and (L+1)*c doubles). */
+cerar_status_t cerar_plan_get_U(const cerar_plan_t* plan, int worker, double* out_cxc);
+cerar_status_t cerar_plan_get_R(const cerar_plan_t* plan, int worker, double* out_Lp1xc);
+/* Diagnostics (computed on first request: a few SVDs on the host). */
+cerar_status_t cerar_plan_info(cerar_plan_t* plan, cerar_plan_info_t* out);
+
+/* Bytes of the device workspace for gradient length d: 4 * N * (c+N) * (d/c);
+ * 0 if c does not divide d. */
+size_t cerar_workspace_bytes(const cerar_plan_t* plan, int64_t d);
+
+/* ---- data path (device buffers, fp32) ----
+ *
+ * cerar_encode: Delta_i = G_i U_i for every worker (Sec. II, Initialization):
+ *   D_{i,j}[q] = sum_l U_i[l, j-1] * g_i[l*p + q].  grads: worker i's gradient
+ *   at grads + i*grads_stride (stride in floats, >= d).  In place: pass
+ *   grads = ws + N*p and grads_stride = (c+N)*p, i.e. the gradient already sits
+ *   in the D rows.  Resets the round counter.
+ *
+ * cerar_ring_round(k), k = 1..L in order: every worker forms the message of
+ *   round k, x_{i,k} = sigma_{i,k-1} (+ delta_{i,k} if k <= c) with
+ *   sigma_{i,k-1} = y_{i,k-1} (- delta_{i,k-N} if k-1 >= N), sigma_{i,0} = 0
+ *   (Eq. update_eqns; Algorithm 1 with the cancel step of round k-1 fused into
+ *   the send step of round k), and hands it to W_{i+1} by storing it in slot
+ *   k-1 of that worker's workspace.
+ *
+ * cerar_decode: g_hat_i = scale * Y_i R_i (Sec. II-A), Y_i = [y_{i,1} .. y_{i,L+1}].
+ *   out: worker i's result at out + i*out_stride (floats, >= d); every worker
+ *   gets its own (slightly different) approximation.  scale = 1 is the paper's
+ *   approximate sum, scale = 1/N the mean.  In place: out = ws + N*p with
+ *   out_stride = (c+N)*p overwrites the D rows.  Needs all L rounds done.
+ *
+ * cerar_allreduce_sim: encode, rounds 1..L, decode, on one stream.
+ *
+ * d must be a positive multiple of c (the caller zero-pads, Sec. II) else
+ * CERAR_ERR_SHAPE.  ws must hold cerar_workspace_bytes(plan, d) bytes.  Input,
+ * output and workspace may alias only in the two in-place forms above.
+ */
+cerar_status_t cerar_encode(cerar_plan_t* plan, const float* grads, int64_t grads_stride,
+                            float* ws, int64_t d, cerar_stream_t stream);
+cerar_status_t cerar_ring_round(cerar_plan_t* plan, float* ws, int64_t d, int k,
+                                cerar_stream_t stream);
+cerar_status_t cerar_decode(cerar_plan_t* plan, const float* ws, float* out, int64_t out_stride,
+                            int64_t d, float scale, cerar_stream_t stream);
+cerar_status_t cerar_allreduce_sim(cerar_plan_t* plan, const float* grads, int64_t grads_stride,
+                                   float* out, int64_t out_stride, float* ws, int64_t d,
+                                   float scale, cerar_stream_t stream);
+
+/* Same pipeline with HOST gradients and results: copies worker i's gradient
+ * (h_grads + i*h_grads_stride, d floats; pinned memory makes the copies
+ * asynchronous) into the D rows of the device workspace, runs encode, the L
+ * rounds and decode in place, and copies the results back to
+ * h_out + i*h_out_stride.  Work is issued on `stream`; the call returns after
+ * everything is enqueued.  ws: device, cerar_workspace_bytes(plan, d). */
+cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* plan, const float* h_grads,
+                                        int64_t h_grads_stride, float* h_out,
+                                        int64_t h_out_stride, float* ws, int64_t d,
+                                        float scale, cerar_stream_t stream);
+
+/* Rate counters (Sec. II-B: communication rate 1+(N-2)/c = bytes_forwarded /
+ * bytes_gradient after L rounds; storage rate 1+N/c = bytes_stored / bytes_gradient). */
+cerar_status_t cerar_get_counters(const cerar_plan_t* plan, cerar_counters_t* out);
+
+/* Number of kernels this library has launched through this plan so far. */
+uint64_t       cerar_launch_count(const cerar_plan_t* plan);
+
+/* Synchronises `stream` and reports CERAR_ERR_TIMEOUT if a kernel of this plan
+ * gave up on one of its bounded device-side waits since the last check (the
+ * results of that call are then invalid); CERAR_OK otherwise. */
+cerar_status_t cerar_device_status(cerar_plan_t* plan, cerar_stream_t stream);
+
+/* Kernel selection for encode/decode: 0 = automatic, 1 = plain per-position
+ * reference kernel, 2 = staged FMA kernel.  Returns the previous value. */
+int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
+
+/* Process-wide tuning knobs of the staged kernel, for experiments: name is one of
+ * "kc" (input rows per pipeline stage), "stages", "jt" (outputs per thread: 4, 8
+ * or 16), "slabs" (position slabs per CTA); value 0 restores the default.
+ * Returns 0, or -1 for an unknown name. */
+int            cerar_set_tuning(const char* name, int value);
+
+const char*    cerar_status_string(cerar_status_t s);
+const char*    cerar_last_error(void);   /* thread-local detail of the last failure */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CERAR_H_ */

@@ -1,0 +1,212 @@
+"""ctypes binding of libcerar.so: same names as the C ABI (include/cerar.h).
+
+Only marshals arguments: every step of the data path runs in the library's
+CUDA kernels.  torch is used by callers for device memory and streams; this
+module itself needs only pointers (ints) and never falls back to a CPU path:
+if the library cannot be loaded, importing fails.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+VANDERMONDE, EPSILON, KAPPA = 0, 1, 2
+KERNEL_AUTO, KERNEL_REF, KERNEL_STAGED = 0, 1, 2
+
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "SINGULAR", 4: "NOT_CONVERGED",
+                5: "STATE", 6: "CUDA", 7: "NOMEM", 8: "TIMEOUT"}
+
+
+class CerarError(RuntimeError):
+    def __init__(self, status: int, detail: str):
+        self.status = status
+        super().__init__(f"cerar status {status} ({STATUS_NAMES.get(status, '?')}): {detail}")
+
+
+class Options(C.Structure):
+    _fields_ = [("seed", C.c_uint64), ("B", C.POINTER(C.c_double)), ("h", C.POINTER(C.c_double)),
+                ("eps_init", C.c_double), ("als_iters", C.c_int), ("als_tol", C.c_double),
+                ("host_only", C.c_int)]
+
+
+class PlanInfo(C.Structure):
+    _fields_ = [("N", C.c_int), ("c", C.c_int), ("L", C.c_int), ("construction", C.c_int),
+                ("param", C.c_double), ("phi", C.c_double), ("kappa_U_max", C.c_double),
+                ("kappa_M_max", C.c_double), ("inv_residual_max", C.c_double),
+                ("abs_U_max", C.c_double), ("abs_R_max", C.c_double),
+                ("als_iters_done", C.c_int), ("on_device", C.c_int)]
+
+
+class Counters(C.Structure):
+    _fields_ = [("encoded", C.c_int), ("rounds_done", C.c_int),
+                ("bytes_forwarded_per_worker", C.c_uint64), ("bytes_forwarded_last_round", C.c_uint64),
+                ("bytes_stored_per_worker", C.c_uint64), ("bytes_gradient", C.c_uint64)]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB_PATH
+    if _build.is_stale():
+        path = _build.build()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing and could not be built")
+    return C.CDLL(path)
+
+
+lib = _load()
+_vp, _i64, _f32p = C.c_void_p, C.c_int64, C.c_void_p
+
+lib.cerar_plan_create.argtypes = [C.c_int, C.c_int, C.c_int, C.c_double, C.POINTER(_vp)]
+lib.cerar_plan_create_ex.argtypes = [C.c_int, C.c_int, C.c_int, C.c_double, C.POINTER(Options), C.POINTER(_vp)]
+lib.cerar_plan_create_custom.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                         C.c_int, C.POINTER(_vp)]
+lib.cerar_plan_destroy.argtypes = [_vp]
+lib.cerar_plan_destroy.restype = None
+lib.cerar_plan_get_U.argtypes = [_vp, C.c_int, C.POINTER(C.c_double)]
+lib.cerar_plan_get_R.argtypes = [_vp, C.c_int, C.POINTER(C.c_double)]
+lib.cerar_plan_info.argtypes = [_vp, C.POINTER(PlanInfo)]
+lib.cerar_workspace_bytes.argtypes = [_vp, _i64]
+lib.cerar_workspace_bytes.restype = C.c_size_t
+lib.cerar_encode.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _vp]
+lib.cerar_ring_round.argtypes = [_vp, _f32p, _i64, C.c_int, _vp]
+lib.cerar_decode.argtypes = [_vp, _f32p, _f32p, _i64, _i64, C.c_float, _vp]
+lib.cerar_allreduce_sim.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
+lib.cerar_allreduce_sim_host.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
+lib.cerar_get_counters.argtypes = [_vp, C.POINTER(Counters)]
+lib.cerar_launch_count.argtypes = [_vp]
+lib.cerar_launch_count.restype = C.c_uint64
+lib.cerar_set_kernel_mode.argtypes = [_vp, C.c_int]
+lib.cerar_device_status.argtypes = [_vp, _vp]
+lib.cerar_set_tuning.argtypes = [C.c_char_p, C.c_int]
+lib.cerar_status_string.argtypes = [C.c_int]
+lib.cerar_status_string.restype = C.c_char_p
+lib.cerar_last_error.restype = C.c_char_p
+
+
+def _check(status: int):
+    if status != 0:
+        raise CerarError(status, lib.cerar_last_error().decode())
+
+
+def _dptr(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float64).ctypes.data_as(C.POINTER(C.c_double))
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor / numpy array / int."""
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+def cerar_set_tuning(name: str, value: int) -> int:
+    return lib.cerar_set_tuning(name.encode(), int(value))
+
+
+class Plan:
+    """Owns a cerar_plan_t*.  Methods are the C calls with the plan bound."""
+
+    def __init__(self, handle: int, N: int, c: int):
+        self._h = C.c_void_p(handle)
+        self.N, self.c, self.L = N, c, c + N - 2
+
+    # ---- creation
+    @staticmethod
+    def create(N, c, kind, param, *, seed=0, B=None, h=None, eps_init=0.0, als_iters=0,
+               als_tol=0.0, host_only=False) -> "Plan":
+        keep = [None if B is None else np.ascontiguousarray(B, dtype=np.float64),
+                None if h is None else np.ascontiguousarray(h, dtype=np.float64)]
+        opt = Options()
+        opt.seed = seed
+        opt.B = keep[0].ctypes.data_as(C.POINTER(C.c_double)) if keep[0] is not None else None
+        opt.h = keep[1].ctypes.data_as(C.POINTER(C.c_double)) if keep[1] is not None else None
+        opt.eps_init, opt.als_iters, opt.als_tol, opt.host_only = eps_init, als_iters, als_tol, int(host_only)
+        out = C.c_void_p()
+        _check(lib.cerar_plan_create_ex(N, c, kind, float(param), C.byref(opt), C.byref(out)))
+        return Plan(out.value, N, c)
+
+    @staticmethod
+    def create_custom(N, c, U, R, host_only=False) -> "Plan":
+        L = c + N - 2
+        Ua = np.ascontiguousarray(np.stack([np.asarray(u, np.float64) for u in U]))
+        Ra = np.ascontiguousarray(np.stack([np.asarray(r, np.float64) for r in R]))
+        assert Ua.shape == (N, c, c) and Ra.shape == (N, L + 1, c)
+        out = C.c_void_p()
+        _check(lib.cerar_plan_create_custom(N, c, Ua.ctypes.data_as(C.POINTER(C.c_double)),
+                                            Ra.ctypes.data_as(C.POINTER(C.c_double)), int(host_only), C.byref(out)))
+        return Plan(out.value, N, c)
+
+    def destroy(self):
+        if self._h:
+            lib.cerar_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    # ---- host queries
+    def get_U(self, worker: int) -> np.ndarray:
+        out = np.empty((self.c, self.c), dtype=np.float64)
+        _check(lib.cerar_plan_get_U(self._h, worker, out.ctypes.data_as(C.POINTER(C.c_double))))
+        return out
+
+    def get_R(self, worker: int) -> np.ndarray:
+        out = np.empty((self.L + 1, self.c), dtype=np.float64)
+        _check(lib.cerar_plan_get_R(self._h, worker, out.ctypes.data_as(C.POINTER(C.c_double))))
+        return out
+
+    def info(self) -> dict:
+        s = PlanInfo()
+        _check(lib.cerar_plan_info(self._h, C.byref(s)))
+        return {f: getattr(s, f) for f, _ in PlanInfo._fields_}
+
+    def workspace_bytes(self, d: int) -> int:
+        return lib.cerar_workspace_bytes(self._h, d)
+
+    def counters(self) -> dict:
+        s = Counters()
+        _check(lib.cerar_get_counters(self._h, C.byref(s)))
+        return {f: getattr(s, f) for f, _ in Counters._fields_}
+
+    def launch_count(self) -> int:
+        return lib.cerar_launch_count(self._h)
+
+    def set_kernel_mode(self, mode: int) -> int:
+        return lib.cerar_set_kernel_mode(self._h, mode)
+
+    def device_status(self, stream=0):
+        _check(lib.cerar_device_status(self._h, stream))
+
+    # ---- data path (device pointers; stream = a cudaStream_t handle as int)
+    def encode(self, grads, grads_stride, ws, d, stream=0):
+        _check(lib.cerar_encode(self._h, _ptr(grads), grads_stride, _ptr(ws), d, stream))
+
+    def ring_round(self, ws, d, k, stream=0):
+        _check(lib.cerar_ring_round(self._h, _ptr(ws), d, k, stream))
+
+    def decode(self, ws, out, out_stride, d, scale=1.0, stream=0):
+        _check(lib.cerar_decode(self._h, _ptr(ws), _ptr(out), out_stride, d, scale, stream))
+
+    def allreduce_sim(self, grads, grads_stride, out, out_stride, ws, d, scale=1.0, stream=0):
+        _check(lib.cerar_allreduce_sim(self._h, _ptr(grads), grads_stride, _ptr(out), out_stride,
+                                       _ptr(ws), d, scale, stream))
+
+    def allreduce_sim_host(self, h_grads, h_grads_stride, h_out, h_out_stride, ws, d, scale=1.0, stream=0):
+        _check(lib.cerar_allreduce_sim_host(self._h, _ptr(h_grads), h_grads_stride, _ptr(h_out),
+                                            h_out_stride, _ptr(ws), d, scale, stream))
+
+
+def cerar_plan_create(N, c, kind, param, **kw) -> Plan:
+    return Plan.create(N, c, kind, param, **kw)
+
+
+def cerar_plan_create_custom(N, c, U, R, host_only=False) -> Plan:
+    return Plan.create_custom(N, c, U, R, host_only)

@@ -1,0 +1,366 @@
+// C ABI of the CERAR library: plan life-cycle, round state machine, counters,
+// argument checking, and the launches of the data-path kernels.
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/cerar.h"
+#include "kernels.cuh"
+#include "plan.hpp"
+
+namespace cerar {
+extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs;
+}
+
+struct cerar_plan {
+    cerar::HostPlan host;
+    // device copies (fp32): U_i as the c x c encode matrix, R_i as the (L+1) x c decode matrix
+    float* d_U = nullptr;
+    float* d_R = nullptr;
+    int* d_status = nullptr;
+    int device = -1;
+    int num_sms = 0;
+    bool on_device = false;
+    // diagnostics cache
+    bool info_done = false;
+    cerar_plan_info_t info{};
+    // state machine and counters
+    int encoded = 0;
+    int rounds_done = 0;
+    int64_t cur_d = 0;
+    uint64_t bytes_forwarded = 0;
+    uint64_t launches = 0;
+    int kernel_mode = 0;
+};
+
+namespace {
+
+thread_local std::string g_err;
+
+cerar_status_t fail(cerar_status_t s, const std::string& msg) {
+    g_err = msg;
+    return s;
+}
+
+cerar_status_t cuda_fail(cudaError_t e, const char* what) {
+    g_err = std::string(what) + ": " + cudaGetErrorString(e);
+    return CERAR_ERR_CUDA;
+}
+
+cerar_status_t upload(cerar_plan* P) {
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess || count == 0) {
+        cudaGetLastError();     // clear the sticky "no device" error
+        return CERAR_OK;        // host-only plan
+    }
+    const int N = P->host.N, c = P->host.c, L = P->host.L;
+    if ((e = cudaGetDevice(&P->device)) != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, P->device)) != cudaSuccess) return cuda_fail(e, "cudaGetDeviceProperties");
+    P->num_sms = prop.multiProcessorCount;
+    std::vector<float> hU((size_t)N * c * c), hR((size_t)N * (L + 1) * c);
+    for (int i = 0; i < N; ++i) {
+        for (size_t t = 0; t < (size_t)c * c; ++t) hU[(size_t)i * c * c + t] = (float)P->host.U[i][t];
+        for (size_t t = 0; t < (size_t)(L + 1) * c; ++t) hR[(size_t)i * (L + 1) * c + t] = (float)P->host.R[i][t];
+    }
+    for (float v : hU) if (!std::isfinite(v)) return fail(CERAR_ERR_SINGULAR, "an encoder entry overflows fp32");
+    for (float v : hR) if (!std::isfinite(v)) return fail(CERAR_ERR_SINGULAR, "a decoder entry overflows fp32");
+    if ((e = cudaMalloc(&P->d_U, hU.size() * sizeof(float))) != cudaSuccess) return cuda_fail(e, "cudaMalloc U");
+    if ((e = cudaMalloc(&P->d_R, hR.size() * sizeof(float))) != cudaSuccess) return cuda_fail(e, "cudaMalloc R");
+    if ((e = cudaMalloc(&P->d_status, sizeof(int))) != cudaSuccess) return cuda_fail(e, "cudaMalloc status");
+    if ((e = cudaMemcpy(P->d_U, hU.data(), hU.size() * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess)
+        return cuda_fail(e, "upload U");
+    if ((e = cudaMemcpy(P->d_R, hR.data(), hR.size() * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess)
+        return cuda_fail(e, "upload R");
+    if ((e = cudaMemset(P->d_status, 0, sizeof(int))) != cudaSuccess) return cuda_fail(e, "memset status");
+    P->on_device = true;
+    return CERAR_OK;
+}
+
+cerar_status_t finish_create(cerar_plan* P, bool host_only, cerar_plan_t** out) {
+    if (!host_only) {
+        cerar_status_t st = upload(P);
+        if (st != CERAR_OK) { cerar_plan_destroy(P); return st; }
+    }
+    *out = P;
+    return CERAR_OK;
+}
+
+cerar_status_t check_data_call(const cerar_plan* P, int64_t d, int64_t* p_out) {
+    if (!P) return fail(CERAR_ERR_INVALID_ARG, "plan is NULL");
+    if (!P->on_device) return fail(CERAR_ERR_CUDA, "plan has no device copies (no CUDA device, or host_only)");
+    if (d <= 0 || d % P->host.c != 0) return fail(CERAR_ERR_SHAPE, "d must be a positive multiple of c");
+    *p_out = d / P->host.c;
+    return CERAR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cerar_status_string(cerar_status_t s) {
+    switch (s) {
+        case CERAR_OK: return "ok";
+        case CERAR_ERR_INVALID_ARG: return "invalid argument";
+        case CERAR_ERR_SHAPE: return "bad shape";
+        case CERAR_ERR_SINGULAR: return "singular or non-finite design";
+        case CERAR_ERR_NOT_CONVERGED: return "design did not meet its constraint";
+        case CERAR_ERR_STATE: return "call out of order";
+        case CERAR_ERR_CUDA: return "CUDA error";
+        case CERAR_ERR_NOMEM: return "out of memory";
+        case CERAR_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+const char* cerar_last_error(void) { return g_err.c_str(); }
+
+cerar_status_t cerar_plan_create_ex(int N, int c, cerar_construction_t kind, double param,
+                                    const cerar_options_t* opt, cerar_plan_t** out) {
+    if (!out) return fail(CERAR_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (N < 2 || c < N || c > 512) return fail(CERAR_ERR_INVALID_ARG, "need 2 <= N <= c <= 512");
+    cerar_options_t o;
+    std::memset(&o, 0, sizeof(o));
+    if (opt) o = *opt;
+    cerar_plan* P = new (std::nothrow) cerar_plan();
+    if (!P) return fail(CERAR_ERR_NOMEM, "plan allocation failed");
+    std::string err;
+    int st = cerar::BUILD_INVALID;
+    std::vector<double> Bdef;
+    const double* B = o.B;
+    if (!B && kind != CERAR_VANDERMONDE) {
+        Bdef = cerar::default_base_matrix(N, c, o.seed);
+        B = Bdef.data();
+    }
+    switch (kind) {
+        case CERAR_VANDERMONDE: st = cerar::build_vandermonde(N, c, param, o.h, P->host, err); break;
+        case CERAR_EPSILON: st = cerar::build_epsilon(N, c, param, B, o.h, P->host, err); break;
+        case CERAR_KAPPA:
+            st = cerar::build_kappa(N, c, param, B, o.h, o.eps_init, o.als_iters, o.als_tol, P->host, err);
+            break;
+        default: err = "unknown construction"; break;
+    }
+    if (st != cerar::BUILD_OK) {
+        delete P;
+        return fail((cerar_status_t)st, err);
+    }
+    return finish_create(P, o.host_only != 0, out);
+}
+
+cerar_status_t cerar_plan_create(int N, int c, cerar_construction_t kind, double param, cerar_plan_t** out) {
+    return cerar_plan_create_ex(N, c, kind, param, nullptr, out);
+}
+
+cerar_status_t cerar_plan_create_custom(int N, int c, const double* U, const double* R, int host_only,
+                                        cerar_plan_t** out) {
+    if (!out) return fail(CERAR_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    if (N < 2 || c < N || c > 512) return fail(CERAR_ERR_INVALID_ARG, "need 2 <= N <= c <= 512");
+    if (!U || !R) return fail(CERAR_ERR_INVALID_ARG, "U or R is NULL");
+    cerar_plan* P = new (std::nothrow) cerar_plan();
+    if (!P) return fail(CERAR_ERR_NOMEM, "plan allocation failed");
+    const int L = c + N - 2;
+    P->host.N = N; P->host.c = c; P->host.L = L; P->host.kind = 3;
+    P->host.U.resize(N); P->host.R.resize(N);
+    for (int i = 0; i < N; ++i) {
+        P->host.U[i].assign(U + (size_t)i * c * c, U + (size_t)(i + 1) * c * c);
+        P->host.R[i].assign(R + (size_t)i * (L + 1) * c, R + (size_t)(i + 1) * (L + 1) * c);
+        for (double v : P->host.U[i]) if (!std::isfinite(v)) { delete P; return fail(CERAR_ERR_SINGULAR, "non-finite U"); }
+        for (double v : P->host.R[i]) if (!std::isfinite(v)) { delete P; return fail(CERAR_ERR_SINGULAR, "non-finite R"); }
+    }
+    return finish_create(P, host_only != 0, out);
+}
+
+void cerar_plan_destroy(cerar_plan_t* P) {
+    if (!P) return;
+    if (P->on_device || P->d_U || P->d_R || P->d_status) {
+        cudaFree(P->d_U); cudaFree(P->d_R); cudaFree(P->d_status);
+    }
+    delete P;
+}
+
+cerar_status_t cerar_plan_get_U(const cerar_plan_t* P, int worker, double* out) {
+    if (!P || !out || worker < 0 || worker >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "bad argument");
+    std::memcpy(out, P->host.U[worker].data(), P->host.U[worker].size() * sizeof(double));
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_plan_get_R(const cerar_plan_t* P, int worker, double* out) {
+    if (!P || !out || worker < 0 || worker >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "bad argument");
+    std::memcpy(out, P->host.R[worker].data(), P->host.R[worker].size() * sizeof(double));
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_plan_info(cerar_plan_t* P, cerar_plan_info_t* out) {
+    if (!P || !out) return fail(CERAR_ERR_INVALID_ARG, "bad argument");
+    if (!P->info_done) {
+        cerar_plan_info_t& I = P->info;
+        I.N = P->host.N; I.c = P->host.c; I.L = P->host.L;
+        I.construction = P->host.kind; I.param = P->host.param;
+        I.phi = (P->host.phi_closed >= 0) ? P->host.phi_closed : cerar::phi_direct(P->host);
+        I.kappa_U_max = cerar::kappa_U_max(P->host);
+        I.kappa_M_max = cerar::kappa_M_max(P->host);
+        I.inv_residual_max = P->host.inv_residual_max;
+        double mu = 0, mr = 0;
+        for (const auto& m : P->host.U) for (double v : m) mu = std::fmax(mu, std::fabs(v));
+        for (const auto& m : P->host.R) for (double v : m) mr = std::fmax(mr, std::fabs(v));
+        I.abs_U_max = mu; I.abs_R_max = mr;
+        I.als_iters_done = P->host.als_iters_done;
+        P->info_done = true;
+    }
+    P->info.on_device = P->on_device ? 1 : 0;
+    *out = P->info;
+    return CERAR_OK;
+}
+
+size_t cerar_workspace_bytes(const cerar_plan_t* P, int64_t d) {
+    if (!P || d <= 0 || d % P->host.c != 0) return 0;
+    return (size_t)4 * P->host.N * (size_t)(P->host.c + P->host.N) * (size_t)(d / P->host.c);
+}
+
+cerar_status_t cerar_encode(cerar_plan_t* P, const float* grads, int64_t grads_stride, float* ws, int64_t d,
+                            cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!grads || !ws) return fail(CERAR_ERR_INVALID_ARG, "grads or ws is NULL");
+    if (grads_stride < d) return fail(CERAR_ERR_SHAPE, "grads_stride < d");
+    const int N = P->host.N, c = P->host.c;
+    cerar::ContractArgs a{};
+    a.in = grads; a.in_wstride = grads_stride; a.in_rstride = p;
+    a.out = ws + (int64_t)N * p; a.out_wstride = (int64_t)(c + N) * p; a.out_rstride = p;
+    a.coef = P->d_U; a.K = c; a.J = c; a.skip_row = 1 << 30;
+    a.N = N; a.p = p; a.scale = 1.0f; a.status = P->d_status;
+    cudaError_t e = cerar::launch_contract(a, P->kernel_mode, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "encode launch");
+    P->encoded = 1; P->rounds_done = 0; P->cur_d = d; P->bytes_forwarded = 0;
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_ring_round(cerar_plan_t* P, float* ws, int64_t d, int k, cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws) return fail(CERAR_ERR_INVALID_ARG, "ws is NULL");
+    if (!P->encoded || d != P->cur_d) return fail(CERAR_ERR_STATE, "encode (with the same d) must come first");
+    if (k != P->rounds_done + 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "rounds must run in order 1..L");
+    cerar::RoundArgs a{ws, p, P->host.N, P->host.c, k};
+    cudaError_t e = cerar::launch_round(a, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "round launch");
+    P->rounds_done = k;
+    P->bytes_forwarded += (uint64_t)4 * (uint64_t)p;
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_decode(cerar_plan_t* P, const float* ws, float* out, int64_t out_stride, int64_t d,
+                            float scale, cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !out) return fail(CERAR_ERR_INVALID_ARG, "ws or out is NULL");
+    if (out_stride < d) return fail(CERAR_ERR_SHAPE, "out_stride < d");
+    if (!P->encoded || d != P->cur_d || P->rounds_done != P->host.L)
+        return fail(CERAR_ERR_STATE, "decode needs encode and all L rounds");
+    const int N = P->host.N, c = P->host.c, L = P->host.L;
+    cerar::ContractArgs a{};
+    a.in = ws; a.in_wstride = (int64_t)(c + N) * p; a.in_rstride = p;
+    a.out = out; a.out_wstride = out_stride; a.out_rstride = p;
+    a.coef = P->d_R; a.K = L + 1; a.J = c; a.skip_row = L;     // y_{L+1} sits in slot L+1
+    a.N = N; a.p = p; a.scale = scale; a.status = P->d_status;
+    cudaError_t e = cerar::launch_contract(a, P->kernel_mode, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "decode launch");
+    const float* ws_end = ws + (size_t)N * (size_t)(c + N) * (size_t)p;
+    if (out + (size_t)(N - 1) * out_stride + d > ws && out < ws_end)
+        P->encoded = 0;     // decoded in place: the observations are gone
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_allreduce_sim(cerar_plan_t* P, const float* grads, int64_t grads_stride, float* out,
+                                   int64_t out_stride, float* ws, int64_t d, float scale, cerar_stream_t stream) {
+    cerar_status_t st = cerar_encode(P, grads, grads_stride, ws, d, stream);
+    if (st != CERAR_OK) return st;
+    for (int k = 1; k <= P->host.L; ++k)
+        if ((st = cerar_ring_round(P, ws, d, k, stream)) != CERAR_OK) return st;
+    return cerar_decode(P, ws, out, out_stride, d, scale, stream);
+}
+
+cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* P, const float* h_grads, int64_t h_grads_stride,
+                                        float* h_out, int64_t h_out_stride, float* ws, int64_t d, float scale,
+                                        cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!h_grads || !h_out || !ws) return fail(CERAR_ERR_INVALID_ARG, "NULL buffer");
+    if (h_grads_stride < d || h_out_stride < d) return fail(CERAR_ERR_SHAPE, "stride < d");
+    const int N = P->host.N, c = P->host.c;
+    const int64_t wstride = (int64_t)(c + N) * p;
+    float* drows = ws + (int64_t)N * p;             // worker 0's D rows: d contiguous floats
+    cudaStream_t s = (cudaStream_t)stream;
+    for (int i = 0; i < N; ++i) {
+        cudaError_t e = cudaMemcpyAsync(drows + i * wstride, h_grads + i * h_grads_stride, (size_t)d * 4,
+                                        cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return cuda_fail(e, "H2D copy");
+    }
+    st = cerar_allreduce_sim(P, drows, wstride, drows, wstride, ws, d, scale, stream);
+    if (st != CERAR_OK) return st;
+    for (int i = 0; i < N; ++i) {
+        cudaError_t e = cudaMemcpyAsync(h_out + i * h_out_stride, drows + i * wstride, (size_t)d * 4,
+                                        cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return cuda_fail(e, "D2H copy");
+    }
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_get_counters(const cerar_plan_t* P, cerar_counters_t* out) {
+    if (!P || !out) return fail(CERAR_ERR_INVALID_ARG, "bad argument");
+    const int64_t p = P->cur_d / (P->host.c ? P->host.c : 1);
+    out->encoded = P->encoded;
+    out->rounds_done = P->rounds_done;
+    out->bytes_forwarded_per_worker = P->bytes_forwarded;
+    out->bytes_forwarded_last_round = P->rounds_done > 0 ? (uint64_t)4 * p : 0;
+    out->bytes_stored_per_worker = (uint64_t)4 * p * (uint64_t)(P->host.c + P->host.N);
+    out->bytes_gradient = (uint64_t)4 * (uint64_t)P->cur_d;
+    return CERAR_OK;
+}
+
+uint64_t cerar_launch_count(const cerar_plan_t* P) { return P ? P->launches : 0; }
+
+int cerar_set_kernel_mode(cerar_plan_t* P, int mode) {
+    if (!P) return -1;
+    int old = P->kernel_mode;
+    if (mode >= 0 && mode <= 2) P->kernel_mode = mode;
+    return old;
+}
+
+cerar_status_t cerar_device_status(cerar_plan_t* P, cerar_stream_t stream) {
+    if (!P) return fail(CERAR_ERR_INVALID_ARG, "plan is NULL");
+    if (!P->on_device) return fail(CERAR_ERR_CUDA, "plan has no device copies");
+    int flag = 0;
+    cudaError_t e = cudaMemcpyAsync(&flag, P->d_status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "status read");
+    if (flag != 0) {
+        cudaMemsetAsync(P->d_status, 0, sizeof(int), (cudaStream_t)stream);
+        return fail(CERAR_ERR_TIMEOUT, "a kernel gave up on a bounded wait");
+    }
+    return CERAR_OK;
+}
+
+int cerar_set_tuning(const char* name, int value) {
+    if (!name) return -1;
+    std::string n(name);
+    if (n == "kc") cerar::g_tune_kc = value;
+    else if (n == "stages") cerar::g_tune_stages = value;
+    else if (n == "jt") cerar::g_tune_jt = value;
+    else if (n == "slabs") cerar::g_tune_slabs = value;
+    else return -1;
+    return 0;
+}
+
+}  // extern "C"

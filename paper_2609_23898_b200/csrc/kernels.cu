@@ -1,0 +1,391 @@
+// CUDA kernels of the CERAR data path for sm_100a.
+//
+//  contract_ref_kernel     plain per-position contraction, any p and alignment
+//  contract_staged_kernel  warp-specialised contraction: one producer warp streams
+//                          row tiles into shared memory with bulk async copies
+//                          (cp.async.bulk + mbarrier), consumer warps run the FMA
+//                          register tile; used for encode and decode
+//  round_kernel            one ring round for all workers: fused cancel + add +
+//                          hand-off store into the neighbour's landing slot
+#include "kernels.cuh"
+
+#include <cstdio>
+
+namespace cerar {
+namespace {
+
+constexpr int REF_MAX_J = 512;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a bounded wait gives up after 2 s
+
+// ------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        " .reg .pred p;\n"
+        " mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        " selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for a phase of an mbarrier, but never forever: returns false after
+// WAIT_LIMIT_NS so that the caller can flag the error and leave.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+    }
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// ------------------------------------------------------------------ reference contraction
+__global__ void contract_ref_kernel(const ContractArgs a) {
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int w = blockIdx.y;
+    if (q >= a.p) return;
+    float acc[REF_MAX_J];
+    for (int j = 0; j < a.J; ++j) acc[j] = 0.f;
+    const float* in = a.in + (int64_t)w * a.in_wstride + q;
+    const float* cf = a.coef + (size_t)w * a.K * a.J;
+    for (int k = 0; k < a.K; ++k) {
+        const int row = (k < a.skip_row) ? k : k + 1;
+        const float x = in[(int64_t)row * a.in_rstride];
+        for (int j = 0; j < a.J; ++j) acc[j] = fmaf(cf[(size_t)k * a.J + j], x, acc[j]);
+    }
+    float* out = a.out + (int64_t)w * a.out_wstride + q;
+    for (int j = 0; j < a.J; ++j) out[(int64_t)j * a.out_rstride] = acc[j] * a.scale;
+}
+
+// ------------------------------------------------------------------ staged contraction
+//
+// grid = (CTAs per worker, N).  CTA (b, w) walks tiles b, b+gridDim.x, ... of
+// worker w.  A tile is tile_p = slabs*PV*128 consecutive positions; it is
+// streamed through shared memory in chunks of KC input rows.  Every consumer
+// thread owns 4*PV positions x JT outputs; all K inputs of a tile are consumed
+// before its outputs are stored, which makes in-place use (outputs overwriting
+// input rows) safe: tiles are disjoint in positions.
+//
+// shared memory: [full[stages], empty[stages] mbarriers | coef K x Jpad | stages x KC x tile_p]
+template <int PV, int JT, int MAXW>
+__global__ void __launch_bounds__(32 * (MAXW + 1), 1)
+contract_staged_kernel(const __grid_constant__ ContractArgs a) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int CW = a.slabs * a.jgroups;                 // consumer warps; warp CW is the producer
+    const int Jpad = a.jgroups * JT;
+    const int stages = a.stages, KC = a.KC, tile_p = a.tile_p;
+    const int nkc = (a.K + KC - 1) / KC;
+    const int w = blockIdx.y;
+
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_raw);
+    // (barriers take a whole number of 128-byte lines)
+    float* coef_s = reinterpret_cast<float*>(smem_raw + ((2 * stages * 8 + 127) / 128) * 128);
+    float* stage_s = coef_s + (((size_t)a.K * Jpad + 31) / 32) * 32;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8u * stages;
+    const uint32_t stage0 = smem_u32(stage_s);
+    const uint32_t stage_bytes = (uint32_t)KC * tile_p * 4u;
+
+    // set-up (the only CTA-wide barrier, before any bounded wait)
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(full0 + 8u * s, 1);
+            mbar_init(empty0 + 8u * s, CW);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    {
+        const float* cf = a.coef + (size_t)w * a.K * a.J;
+        for (int idx = threadIdx.x; idx < a.K * Jpad; idx += blockDim.x) {
+            const int k = idx / Jpad, j = idx - k * Jpad;
+            coef_s[idx] = (j < a.J) ? cf[(size_t)k * a.J + j] : 0.f;
+        }
+    }
+    __syncthreads();
+
+    uint32_t it = 0;            // chunk counter, same sequence in producer and consumers
+    bool failed = false;
+
+    if (warp == CW) {
+        // ---------------- producer warp
+        const float* in_w = a.in + (int64_t)w * a.in_wstride;
+        for (int64_t t = blockIdx.x; t < a.tiles_per_worker && !failed; t += gridDim.x) {
+            const int64_t q0 = t * tile_p;
+            const int64_t rem = a.p - q0;
+            const uint32_t valid = (uint32_t)(rem < tile_p ? rem : tile_p);
+            for (int kc = 0; kc < nkc; ++kc, ++it) {
+                const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                if (!mbar_wait_bounded(empty0 + 8u * s, ph ^ 1u)) { failed = true; break; }
+                const int k0 = kc * KC;
+                const int kcount = (a.K - k0 < KC) ? (a.K - k0) : KC;
+                if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * s, (uint32_t)kcount * valid * 4u);
+                __syncwarp();
+                for (int r = lane; r < kcount; r += 32) {
+                    const int k = k0 + r;
+                    const int row = (k < a.skip_row) ? k : k + 1;
+                    bulk_load(stage0 + s * stage_bytes + (uint32_t)r * tile_p * 4u,
+                              in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, full0 + 8u * s);
+                }
+            }
+        }
+        if (failed) {
+            if (lane == 0) atomicExch(a.status, 1);
+            // let copies that were already issued land before the CTA retires
+            const unsigned long long t0 = global_ns();
+            while (global_ns() - t0 < 1000000ull) { }
+        }
+    } else {
+        // ---------------- consumer warps
+        const int jg = warp % a.jgroups, slab = warp / a.jgroups;
+        const uint32_t coef_u32 = smem_u32(coef_s) + (uint32_t)(jg * JT) * 4u;
+        uint32_t pos[PV];
+#pragma unroll
+        for (int v = 0; v < PV; ++v) pos[v] = (uint32_t)(((slab * PV + v) * 32 + lane) * 4);
+        float* out_w = a.out + (int64_t)w * a.out_wstride;
+        for (int64_t t = blockIdx.x; t < a.tiles_per_worker && !failed; t += gridDim.x) {
+            const int64_t q0 = t * tile_p;
+            const int64_t rem = a.p - q0;
+            const uint32_t valid = (uint32_t)(rem < tile_p ? rem : tile_p);
+            float acc[JT][PV * 4];
+#pragma unroll
+            for (int j = 0; j < JT; ++j)
+#pragma unroll
+                for (int e = 0; e < PV * 4; ++e) acc[j][e] = 0.f;
+            for (int kc = 0; kc < nkc; ++kc, ++it) {
+                const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                if (!mbar_wait_bounded(full0 + 8u * s, ph)) { failed = true; break; }
+                const int k0 = kc * KC;
+                const int kcount = (a.K - k0 < KC) ? (a.K - k0) : KC;
+                const uint32_t st = stage0 + s * stage_bytes;
+                uint32_t cfa = coef_u32 + (uint32_t)(k0 * Jpad) * 4u;
+#pragma unroll 2
+                for (int kk = 0; kk < kcount; ++kk, cfa += (uint32_t)Jpad * 4u) {
+                    float4 x[PV];
+#pragma unroll
+                    for (int v = 0; v < PV; ++v) x[v] = lds128(st + ((uint32_t)kk * tile_p + pos[v]) * 4u);
+#pragma unroll
+                    for (int j4 = 0; j4 < JT / 4; ++j4) {
+                        const float4 cc = lds128(cfa + 16u * j4);
+                        const float cj[4] = {cc.x, cc.y, cc.z, cc.w};
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                            for (int v = 0; v < PV; ++v) {
+                                const int j = j4 * 4 + jj;
+                                acc[j][v * 4 + 0] = fmaf(cj[jj], x[v].x, acc[j][v * 4 + 0]);
+                                acc[j][v * 4 + 1] = fmaf(cj[jj], x[v].y, acc[j][v * 4 + 1]);
+                                acc[j][v * 4 + 2] = fmaf(cj[jj], x[v].z, acc[j][v * 4 + 2]);
+                                acc[j][v * 4 + 3] = fmaf(cj[jj], x[v].w, acc[j][v * 4 + 3]);
+                            }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8u * s);
+            }
+            if (failed) break;
+#pragma unroll
+            for (int j = 0; j < JT; ++j) {
+                const int jj = jg * JT + j;
+                if (jj < a.J) {
+                    float* orow = out_w + (int64_t)jj * a.out_rstride + q0;
+#pragma unroll
+                    for (int v = 0; v < PV; ++v)
+                        if (pos[v] < valid) {
+                            float4 o;
+                            o.x = acc[j][v * 4 + 0] * a.scale;
+                            o.y = acc[j][v * 4 + 1] * a.scale;
+                            o.z = acc[j][v * 4 + 2] * a.scale;
+                            o.w = acc[j][v * 4 + 3] * a.scale;
+                            *reinterpret_cast<float4*>(orow + pos[v]) = o;
+                        }
+                }
+            }
+        }
+        if (failed && lane == 0) atomicExch(a.status, 1);
+    }
+}
+
+// ------------------------------------------------------------------ ring round
+//
+// Round k for all workers and one (vector of) position(s) per thread:
+//   x_{i,k} = (y_{i,k-1} - delta_{i,k-N}) + delta_{i,k}    (terms that exist)
+// read from slots k-2, k-1 and N-1+k of worker i, stored into slot k-1 of
+// worker i+1.  Slot k-1 of worker i+1 is also that worker's cancel operand, so a
+// thread walks the ring downwards (i = N-1 .. 0) and keeps worker 0's operand in
+// a register: every slot is read before the same thread overwrites it, and no
+// other thread touches this position.
+template <typename VT> __device__ __forceinline__ VT vzero();
+template <> __device__ __forceinline__ float vzero<float>() { return 0.f; }
+template <> __device__ __forceinline__ float4 vzero<float4>() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ float combine(float y, float dc, float da) { return (y - dc) + da; }
+__device__ __forceinline__ float4 combine(float4 y, float4 dc, float4 da) {
+    return make_float4((y.x - dc.x) + da.x, (y.y - dc.y) + da.y, (y.z - dc.z) + da.z, (y.w - dc.w) + da.w);
+}
+
+template <typename VT, int WG>
+__global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
+    constexpr int VW = sizeof(VT) / 4;
+    const int64_t nv = a.p / VW;
+    const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= nv) return;
+    const int N = a.N, c = a.c, k = a.k;
+    const int64_t pv = a.p / VW;                               // row pitch in vectors
+    const int64_t wstride = (int64_t)(c + N) * pv;
+    const bool has_prev = k >= 2, has_cancel = (k - 1) >= N, has_add = k <= c;
+    VT* base = reinterpret_cast<VT*>(a.ws) + v;
+    const int64_t off_prev = (int64_t)(k - 2) * pv, off_land = (int64_t)(k - 1) * pv,
+                  off_add = (int64_t)(N - 1 + k) * pv;
+    VT carry = vzero<VT>();
+    if (has_cancel) carry = base[off_land];                   // worker 0's delta_{0,k-N}
+    for (int i0 = N - 1; i0 >= 0; i0 -= WG) {
+        VT y[WG], dc[WG], da[WG];
+#pragma unroll
+        for (int g = 0; g < WG; ++g) {
+            const int i = i0 - g;
+            y[g] = dc[g] = da[g] = vzero<VT>();
+            if (i >= 0) {
+                const VT* wb = base + (int64_t)i * wstride;
+                if (has_prev) y[g] = wb[off_prev];
+                if (has_cancel) dc[g] = (i == 0) ? carry : wb[off_land];
+                if (has_add) da[g] = wb[off_add];
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < WG; ++g) {
+            const int i = i0 - g;
+            if (i >= 0) {
+                const int dst = (i + 1 == N) ? 0 : i + 1;
+                base[(int64_t)dst * wstride + off_land] = combine(y[g], dc[g], da[g]);
+            }
+        }
+    }
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <int PV, int JT, int MAXW>
+cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
+    auto kern = contract_staged_kernel<PV, JT, MAXW>;
+    const int Jpad = a.jgroups * JT;
+    const size_t bar_bytes = ((2 * (size_t)a.stages * 8 + 127) / 128) * 128;
+    const size_t coef_bytes = (((size_t)a.K * Jpad + 31) / 32) * 32 * 4;
+    const size_t smem = bar_bytes + coef_bytes + (size_t)a.stages * a.KC * a.tile_p * 4;
+    static thread_local size_t configured = 0;
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = smem;
+    }
+    const int threads = 32 * (a.slabs * a.jgroups + 1);
+    int occ = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, threads, smem);
+    if (e != cudaSuccess) return e;
+    if (occ < 1) return cudaErrorInvalidConfiguration;
+    int64_t per_worker = ((int64_t)num_sms * occ) / a.N;
+    if (per_worker < 1) per_worker = 1;
+    if (per_worker > a.tiles_per_worker) per_worker = a.tiles_per_worker;
+    dim3 grid((unsigned)per_worker, (unsigned)a.N);
+    kern<<<grid, threads, smem, s>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// Tuning knobs (0 = default), settable through the C ABI for experiments.
+int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0;
+
+cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
+    if (a.p <= 0 || a.N <= 0) return cudaSuccess;
+    bool can_stage = (a.p % 4 == 0) && aligned16(a.in) && aligned16(a.out) && (a.in_wstride % 4 == 0) &&
+                     (a.out_wstride % 4 == 0) && (a.in_rstride % 4 == 0) && (a.out_rstride % 4 == 0);
+    if (mode == KERNEL_STAGED && !can_stage) return cudaErrorInvalidValue;
+    bool use_staged = can_stage && mode != KERNEL_REF;
+    if (use_staged) {
+        int JT = g_tune_jt ? g_tune_jt : ((a.J % 16 == 0) ? 16 : (a.J % 8 == 0) ? 8 : 4);
+        const int PV = 2;
+        a.jgroups = (a.J + JT - 1) / JT;
+        const int maxw = (JT == 16) ? 8 : 16;
+        if (a.jgroups > maxw) {
+            use_staged = false;
+        } else {
+            int slabs = g_tune_slabs ? g_tune_slabs : (8 + a.jgroups / 2) / a.jgroups;
+            if (slabs < 1) slabs = 1;
+            while (slabs > 1 && slabs * a.jgroups > maxw) --slabs;
+            a.slabs = slabs;
+            a.tile_p = slabs * PV * 128;
+            a.KC = g_tune_kc ? g_tune_kc : 8;
+            if (a.KC > a.K) a.KC = a.K;
+            a.stages = g_tune_stages ? g_tune_stages : 4;
+            a.tiles_per_worker = (int)((a.p + a.tile_p - 1) / a.tile_p);
+            a.total_tiles = (int64_t)a.tiles_per_worker * a.N;
+            // shared memory must fit: shrink the pipeline, then give up
+            auto smem_of = [&](int st) {
+                return ((2 * (size_t)st * 8 + 127) / 128) * 128 + (((size_t)a.K * a.jgroups * JT + 31) / 32) * 128 +
+                       (size_t)st * a.KC * a.tile_p * 4;
+            };
+            while (a.stages > 2 && smem_of(a.stages) > 200 * 1024) --a.stages;
+            if (smem_of(a.stages) > 220 * 1024) use_staged = false;
+            if (use_staged) {
+                cudaError_t e;
+                if (JT == 16) e = launch_staged<2, 16, 8>(a, num_sms, s);
+                else if (JT == 8) e = launch_staged<2, 8, 16>(a, num_sms, s);
+                else e = launch_staged<2, 4, 16>(a, num_sms, s);
+                if (e == cudaSuccess && launches) ++*launches;
+                return e;
+            }
+        }
+    }
+    if (mode == KERNEL_STAGED) return cudaErrorInvalidConfiguration;
+    if (a.J > REF_MAX_J) return cudaErrorInvalidValue;
+    const int threads = 128;
+    dim3 grid((unsigned)((a.p + threads - 1) / threads), (unsigned)a.N);
+    contract_ref_kernel<<<grid, threads, 0, s>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches) {
+    if (a.p <= 0) return cudaSuccess;
+    const int threads = 256;
+    if (a.p % 4 == 0 && aligned16(a.ws)) {
+        const int64_t nv = a.p / 4;
+        round_kernel<float4, 4><<<(unsigned)((nv + threads - 1) / threads), threads, 0, s>>>(a);
+    } else {
+        round_kernel<float, 4><<<(unsigned)((a.p + threads - 1) / threads), threads, 0, s>>>(a);
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace cerar

@@ -1,0 +1,44 @@
+// Device kernels of the CERAR data path and their launch descriptors (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+
+namespace cerar {
+
+// A skinny contraction out[j][q] = scale * sum_k coef[k][j] * in[row(k)][q] over
+// positions q in [0, p), for N workers.  Encoding (Delta_i = G_i U_i) and
+// decoding (G_hat_i = Y_i R_i) are both of this form.
+struct ContractArgs {
+    const float* in;        // worker 0, row 0
+    int64_t in_wstride;     // floats between workers
+    int64_t in_rstride;     // floats between rows
+    float* out;
+    int64_t out_wstride;
+    int64_t out_rstride;
+    const float* coef;      // device: worker i's K x J row-major matrix at coef + i*K*J
+    int K, J;
+    int skip_row;           // input row index r >= skip_row reads physical row r+1
+    int N;
+    int64_t p;
+    float scale;
+    int* status;            // device word; set non-zero when a bounded wait gives up
+    // staged kernel only
+    int KC, stages, slabs, jgroups, tile_p;
+    int tiles_per_worker;
+    int64_t total_tiles;
+};
+
+struct RoundArgs {
+    float* ws;              // workspace, worker i at ws + i*(c+N)*p
+    int64_t p;
+    int N, c, k;            // round k in 1..L
+};
+
+enum { KERNEL_AUTO = 0, KERNEL_REF = 1, KERNEL_STAGED = 2 };
+
+// Returns cudaSuccess or the launch error.  *launches is incremented by the
+// number of kernels launched.
+cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
+
+}  // namespace cerar

@@ -1,0 +1,158 @@
+"""Host-side logic of the library, no GPU needed: the fp64 plan builder against
+the oracle's designs, the exported symbols, argument checking."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import designs as Dz
+from oracle import protocol as P
+from paper_2609_23898_b200 import cerar, inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _plan_mats(pl):
+    return [pl.get_U(i) for i in range(pl.N)], [pl.get_R(i) for i in range(pl.N)]
+
+
+def _normwise(a, b):
+    return np.abs(np.asarray(a) - np.asarray(b)).max() / max(np.abs(np.asarray(b)).max(), 1e-300)
+
+
+def test_every_declared_symbol_is_exported():
+    header = open(os.path.join(ROOT, "include", "cerar.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    names = set(re.findall(r"\b(cerar_[a-z_A-Z0-9]+)\s*\(", header))
+    assert {"cerar_plan_create", "cerar_encode", "cerar_ring_round", "cerar_decode",
+            "cerar_allreduce_sim", "cerar_get_counters"} <= names
+    lib = ctypes.CDLL(os.path.join(ROOT, "paper_2609_23898_b200", "libcerar.so"))
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} is declared in cerar.h but not exported"
+
+
+@pytest.mark.parametrize("N,c,tau", [(4, 8, 0.1), (3, 5, 0.2), (4, 16, 0.05), (2, 2, 0.3), (8, 12, 0.1)])
+def test_vandermonde_plan_matches_oracle(N, c, tau):
+    pl = cerar.Plan.create(N, c, cerar.VANDERMONDE, tau, host_only=True)
+    des = Dz.vandermonde(N, c, tau)
+    U, R = _plan_mats(pl)
+    for i in range(N):
+        assert _normwise(U[i], des.U[i]) < 1e-13
+        assert _normwise(R[i], des.R[i]) < 1e-14
+    info = pl.info()
+    assert info["phi"] == pytest.approx(float(Dz.phi_mp(des)), rel=1e-10)
+    assert (info["N"], info["c"], info["L"]) == (N, c, c + N - 2)
+
+
+@pytest.mark.parametrize("N,c,eps", [(4, 5, 1e-2), (4, 16, 1e-3), (8, 32, 1e-2), (4, 4, 1e-3), (3, 7, 1e-1),
+                                     (4, 32, 1e-3), (4, 4, 0.0), (16, 16, 1e-3)])
+def test_epsilon_plan_matches_oracle(N, c, eps):
+    B = inputs.base_matrix(N, c, 0)
+    pl = cerar.Plan.create(N, c, cerar.EPSILON, eps, B=B, host_only=True)
+    des = Dz.epsilon(N, c, eps, B)
+    U, R = _plan_mats(pl)
+    for i in range(N):
+        assert _normwise(U[i], des.U[i]) < 1e-12, (i, _normwise(U[i], des.U[i]))
+        assert _normwise(R[i], des.R[i]) < 1e-14
+    assert pl.info()["phi"] == pytest.approx(float(Dz.phi_mp(des)), rel=1e-10, abs=1e-30)
+
+
+def test_epsilon_plan_with_custom_h_and_default_B():
+    N, c, eps = 3, 6, 5e-2
+    h = np.linspace(0.9, -0.7, c)
+    B = inputs.base_matrix(N, c, 3)
+    pl = cerar.Plan.create(N, c, cerar.EPSILON, eps, B=B, h=h, host_only=True)
+    des = Dz.epsilon(N, c, eps, B, list(h))
+    for i in range(N):
+        assert _normwise(pl.get_U(i), des.U[i]) < 1e-12
+    # built-in B: identities that hold for any B (Prop. 1 in block form)
+    pl2 = cerar.Plan.create(N, c, cerar.EPSILON, eps, seed=7, host_only=True)
+    U, R = _plan_mats(pl2)
+    Dinv = np.diag(1.0 / (1.0 + eps * np.array(Dz.default_h(c))))
+    for i in range(N):
+        for s in range(N):
+            blk = U[(i - 1 - s) % N] @ R[i][s:s + c, :]
+            np.testing.assert_allclose(blk, np.eye(c) if s >= i else Dinv, atol=1e-8)
+    # different seeds give different B, same seed the same
+    a = cerar.Plan.create(N, c, cerar.EPSILON, eps, seed=7, host_only=True).get_R(0)
+    b = cerar.Plan.create(N, c, cerar.EPSILON, eps, seed=8, host_only=True).get_R(0)
+    np.testing.assert_array_equal(a, R[0])
+    assert np.abs(a - b).max() > 1e-3
+    # the built-in draws look like N(0,1)
+    big = cerar.Plan.create(16, 128, cerar.EPSILON, 1e-3, seed=1, host_only=True).get_R(0)[:16, :]
+    assert abs(big.mean()) < 0.1 and abs(big.std() - 1.0) < 0.1
+
+
+def test_kappa_plan_matches_oracle_and_invariants():
+    N, c, C = 4, 12, 1e4
+    B = inputs.base_matrix(N, c, 0)
+    pl = cerar.Plan.create(N, c, cerar.KAPPA, C, B=B, als_iters=40, host_only=True)
+    des = Dz.kappa_constrained(N, c, C, B, iters=40)
+    U, R = _plan_mats(pl)
+    info = pl.info()
+    assert info["als_iters_done"] == des.info["iters_done"]
+    assert info["phi"] == pytest.approx(P.phi(des.U, des.R), rel=1e-6)
+    assert P.phi(U, R) == pytest.approx(info["phi"], rel=1e-8)
+    for i in range(N):
+        assert _normwise(U[i], des.U[i]) < 1e-6
+        assert _normwise(R[i], des.R[i]) < 1e-6
+        assert P.kappa2(P.m_matrix(U, i)) <= C
+        sv = np.linalg.svd(U[i], compute_uv=False)
+        assert sv[0] / sv[-1] <= C / np.sqrt(N) * (1 + 1e-9)
+    assert info["kappa_M_max"] == pytest.approx(max(P.kappa2(P.m_matrix(U, i)) for i in range(N)), rel=1e-6)
+    assert info["kappa_U_max"] == pytest.approx(max(P.kappa2(u) for u in U), rel=1e-6)
+
+
+def test_custom_plan_roundtrip_and_info():
+    rng = np.random.default_rng(0)
+    N, c = 3, 5
+    des = Dz.custom_orthogonal(N, c, rng)
+    pl = cerar.Plan.create_custom(N, c, des.U, des.R, host_only=True)
+    for i in range(N):
+        np.testing.assert_array_equal(pl.get_U(i), des.U[i])
+        np.testing.assert_array_equal(pl.get_R(i), des.R[i])
+    info = pl.info()
+    assert info["construction"] == 3
+    assert info["phi"] == pytest.approx(P.phi(des.U, des.R), rel=1e-10)
+    assert info["kappa_U_max"] == pytest.approx(1.0, abs=1e-8)
+    assert info["on_device"] == 0
+
+
+def test_argument_errors():
+    for N, c in [(1, 4), (4, 3), (0, 0), (4, 513)]:
+        with pytest.raises(cerar.CerarError) as e:
+            cerar.Plan.create(N, c, cerar.EPSILON, 1e-2, host_only=True)
+        assert e.value.status == 1
+    with pytest.raises(cerar.CerarError) as e:
+        cerar.Plan.create(4, 8, cerar.VANDERMONDE, -1.0, host_only=True)
+    assert e.value.status == 1
+    with pytest.raises(cerar.CerarError) as e:
+        cerar.Plan.create(4, 8, cerar.EPSILON, 2.0, host_only=True)      # eps ||H|| >= 1
+    assert e.value.status == 1
+    with pytest.raises(cerar.CerarError) as e:
+        cerar.Plan.create(4, 8, cerar.EPSILON, 0.0, host_only=True)      # D = I, c > N: singular windows
+    assert e.value.status == 3
+    with pytest.raises(cerar.CerarError) as e:
+        cerar.Plan.create(4, 8, 9, 0.1, host_only=True)                  # unknown construction
+    assert e.value.status == 1
+    with pytest.raises(cerar.CerarError) as e:
+        cerar.Plan.create(4, 8, cerar.KAPPA, 1.5, host_only=True)        # C <= sqrt(N)
+    assert e.value.status == 1
+    bad = np.full((2, 2, 2), np.nan)
+    with pytest.raises(cerar.CerarError) as e:
+        cerar.Plan.create_custom(2, 2, bad, np.zeros((2, 3, 2)), host_only=True)
+    assert e.value.status == 3
+    # fp32 overflow of the encoders is only checked when uploading; a host-only
+    # plan with huge entries is still returned
+    pl = cerar.Plan.create(4, 8, cerar.EPSILON, 1e-2, host_only=True)
+    assert pl.workspace_bytes(8 * 100) == 4 * 4 * 12 * 100
+    assert pl.workspace_bytes(801) == 0
+    # data-path calls on a host-only plan fail loudly instead of computing on the CPU
+    with pytest.raises(cerar.CerarError) as e:
+        pl.encode(0, 800, 0, 800)
+    assert e.value.status == 6
+    c = pl.counters()
+    assert c["rounds_done"] == 0 and c["bytes_forwarded_per_worker"] == 0
+    assert cerar.lib.cerar_status_string(5) == b"call out of order"
