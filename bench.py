@@ -76,6 +76,13 @@ class ClockSampler:
         except OSError:
             self.p = None
 
+    def wait_first_sample(self, timeout=3.0):
+        t0 = time.time()
+        while self.p is not None and time.time() - t0 < timeout:
+            if os.path.getsize(self.f.name) > 0:
+                return
+            time.sleep(0.05)
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.p is None:
@@ -193,8 +200,8 @@ def sampled_parity(cfg, des, plan, grads, ws, out, scale, n_tiles=6, tile=512):
     g_sub = grads.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy().astype(np.float64)
     ora = P.allreduce([x for x in g_sub], des.U, des.R, scale)
     wsv = ws.view(N, c + N, p)
-    rows = list(range(L)) + [L + 1]
-    Y_dev = wsv[:, rows, :][:, :, idx_t].cpu().numpy()                    # (N, L+1, S)
+    rows_t = torch.tensor(list(range(L)) + [L + 1], device=grads.device)
+    Y_dev = wsv[:, rows_t[:, None], idx_t[None, :]].cpu().numpy()         # (N, L+1, S)
     Y_ora = np.stack([ora["Y"][i].T for i in range(N)])
     out_dev = out.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy()
     kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
@@ -263,15 +270,17 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(args.warmup):
         plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
     torch.cuda.synchronize()
     plan.device_status(stream)
+    if sampler:
+        sampler.wait_first_sample()
 
     # ---- timed region: K steps, each the C-ABI sequence encode, rounds 1..L, decode
     K = args.steps
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 3)] for _ in range(K)]
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     sync_all()
     launches0 = plan.launch_count()
     for s in range(K):
