@@ -62,11 +62,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ float4 lds128(uint32_t addr) {
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
-}
 
 // ------------------------------------------------------------------ reference contraction
 __global__ void contract_ref_kernel(const ContractArgs a) {
@@ -166,7 +161,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
     } else {
         // ---------------- consumer warps
         const int jg = warp % a.jgroups, slab = warp / a.jgroups;
-        const uint32_t coef_u32 = smem_u32(coef_s) + (uint32_t)(jg * JT) * 4u;
+        const float* coef_w = coef_s + jg * JT;
         uint32_t pos[PV];
 #pragma unroll
         for (int v = 0; v < PV; ++v) pos[v] = (uint32_t)(((slab * PV + v) * 32 + lane) * 4);
@@ -185,16 +180,17 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                 if (!mbar_wait_bounded(full0 + 8u * s, ph)) { failed = true; break; }
                 const int k0 = kc * KC;
                 const int kcount = (a.K - k0 < KC) ? (a.K - k0) : KC;
-                const uint32_t st = stage0 + s * stage_bytes;
-                uint32_t cfa = coef_u32 + (uint32_t)(k0 * Jpad) * 4u;
+                const float* st = stage_s + (size_t)s * KC * tile_p;
+                const float* cfa = coef_w + (size_t)k0 * Jpad;
 #pragma unroll 2
-                for (int kk = 0; kk < kcount; ++kk, cfa += (uint32_t)Jpad * 4u) {
+                for (int kk = 0; kk < kcount; ++kk, cfa += Jpad) {
                     float4 x[PV];
 #pragma unroll
-                    for (int v = 0; v < PV; ++v) x[v] = lds128(st + ((uint32_t)kk * tile_p + pos[v]) * 4u);
+                    for (int v = 0; v < PV; ++v)
+                        x[v] = *reinterpret_cast<const float4*>(st + (size_t)kk * tile_p + pos[v]);
 #pragma unroll
                     for (int j4 = 0; j4 < JT / 4; ++j4) {
-                        const float4 cc = lds128(cfa + 16u * j4);
+                        const float4 cc = *reinterpret_cast<const float4*>(cfa + 4 * j4);
                         const float cj[4] = {cc.x, cc.y, cc.z, cc.w};
 #pragma unroll
                         for (int jj = 0; jj < 4; ++jj)
@@ -330,7 +326,8 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     if (mode == KERNEL_STAGED && !can_stage) return cudaErrorInvalidValue;
     bool use_staged = can_stage && mode != KERNEL_REF;
     if (use_staged) {
-        int JT = g_tune_jt ? g_tune_jt : ((a.J % 16 == 0) ? 16 : (a.J % 8 == 0) ? 8 : 4);
+        // 8 outputs x 8 positions per thread measured best on B200 (more resident warps than 16 x 8)
+        int JT = g_tune_jt ? g_tune_jt : ((a.J % 8 == 0) ? 8 : 4);
         const int PV = 2;
         a.jgroups = (a.J + JT - 1) / JT;
         const int maxw = (JT == 16) ? 8 : 16;
@@ -342,9 +339,13 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
             while (slabs > 1 && slabs * a.jgroups > maxw) --slabs;
             a.slabs = slabs;
             a.tile_p = slabs * PV * 128;
-            a.KC = g_tune_kc ? g_tune_kc : 8;
+            a.KC = g_tune_kc ? g_tune_kc : 16;
+            if (!g_tune_kc) {                      // keep a stage near 48 KB whatever the tile width
+                const int fit = (48 * 1024) / (a.tile_p * 4);
+                if (a.KC > fit) a.KC = fit < 2 ? 2 : fit;
+            }
             if (a.KC > a.K) a.KC = a.K;
-            a.stages = g_tune_stages ? g_tune_stages : 4;
+            a.stages = g_tune_stages ? g_tune_stages : 3;
             a.tiles_per_worker = (int)((a.p + a.tile_p - 1) / a.tile_p);
             a.total_tiles = (int64_t)a.tiles_per_worker * a.N;
             // shared memory must fit: shrink the pipeline, then give up
