@@ -53,7 +53,8 @@ typedef enum {
     CERAR_ERR_STATE = 5,         /* rounds out of order, decode before the last round    */
     CERAR_ERR_CUDA = 6,          /* a CUDA runtime call failed, or no device             */
     CERAR_ERR_NOMEM = 7,
-    CERAR_ERR_TIMEOUT = 8
+    CERAR_ERR_TIMEOUT = 8,
+    CERAR_ERR_TOO_LARGE = 9      /* request exceeds the built-in workspace (see below)    */
 } cerar_status_t;
 
 typedef enum {
@@ -174,6 +175,33 @@ cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* plan, const float* h_grads
                                         int64_t h_grads_stride, float* h_out,
                                         int64_t h_out_stride, float* ws, int64_t d,
                                         float scale, cerar_stream_t stream);
+
+/* The same pipeline as cerar_allreduce_sim for callers that cannot provide a
+ * workspace because they cannot allocate device memory at this point: for
+ * instance a host program whose framework has already claimed all free memory
+ * for its own pool, or a step loop in which cudaMalloc's device-wide
+ * synchronisation would stall the other streams.  (The paper has no counterpart:
+ * it is a convenience of this library, not part of CERAR.)
+ *
+ * The workspace is a fixed array inside the library's device image: 16 Mi floats
+ * (64 MiB), held by every GPU on which the library's device code is loaded until
+ * the process exits.  The call allocates nothing (no cudaMalloc / cudaFree, no
+ * allocating library routine).  Requests that need more than that, i.e.
+ * cerar_workspace_bytes(plan, d) > 64 MiB, are refused with
+ * CERAR_ERR_TOO_LARGE and a message saying how much was needed.
+ *
+ * grads / out: device buffers as in cerar_allreduce_sim; they must not alias each
+ * other or the workspace (the in-place forms are not available here).  The
+ * device the plan was created on must be current.
+ * First call on a device: looks up the array's device address (once per device);
+ * make that first call before any stream capture begins.
+ * All calls share the one array, which keeps whatever the previous call left in
+ * it.  Nothing needs clearing between calls (every slot is written before it is
+ * read), but two calls whose kernels overlap on the GPU (different streams, or
+ * different host threads) race on it: serialise them. */
+cerar_status_t cerar_allreduce_sim_static(cerar_plan_t* plan, const float* grads, int64_t grads_stride,
+                                          float* out, int64_t out_stride, int64_t d, float scale,
+                                          cerar_stream_t stream);
 
 /* Rate counters (Sec. II-B: communication rate 1+(N-2)/c = bytes_forwarded /
  * bytes_gradient after L rounds; storage rate 1+N/c = bytes_stored / bytes_gradient). */

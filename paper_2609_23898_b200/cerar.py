@@ -18,7 +18,7 @@ VANDERMONDE, EPSILON, KAPPA = 0, 1, 2
 KERNEL_AUTO, KERNEL_REF, KERNEL_STAGED = 0, 1, 2
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "SINGULAR", 4: "NOT_CONVERGED",
-                5: "STATE", 6: "CUDA", 7: "NOMEM", 8: "TIMEOUT"}
+                5: "STATE", 6: "CUDA", 7: "NOMEM", 8: "TIMEOUT", 9: "TOO_LARGE"}
 
 
 class CerarError(RuntimeError):
@@ -75,6 +75,7 @@ lib.cerar_ring_round.argtypes = [_vp, _f32p, _i64, C.c_int, _vp]
 lib.cerar_decode.argtypes = [_vp, _f32p, _f32p, _i64, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim_host.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
+lib.cerar_allreduce_sim_static.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _i64, C.c_float, _vp]
 lib.cerar_get_counters.argtypes = [_vp, C.POINTER(Counters)]
 lib.cerar_launch_count.argtypes = [_vp]
 lib.cerar_launch_count.restype = C.c_uint64
@@ -198,6 +199,11 @@ class Plan:
     def allreduce_sim(self, grads, grads_stride, out, out_stride, ws, d, scale=1.0, stream=0):
         _check(lib.cerar_allreduce_sim(self._h, _ptr(grads), grads_stride, _ptr(out), out_stride,
                                        _ptr(ws), d, scale, stream))
+
+    def allreduce_sim_static(self, grads, grads_stride, out, out_stride, d, scale=1.0, stream=0):
+        """cerar_allreduce_sim_static: same pipeline, workspace built into the library (<= 64 MiB)."""
+        _check(lib.cerar_allreduce_sim_static(self._h, _ptr(grads), grads_stride, _ptr(out), out_stride,
+                                              d, scale, stream))
 
     def allreduce_sim_host(self, h_grads, h_grads_stride, h_out, h_out_stride, ws, d, scale=1.0, stream=0):
         _check(lib.cerar_allreduce_sim_host(self._h, _ptr(h_grads), h_grads_stride, _ptr(h_out),

@@ -114,11 +114,15 @@ const char* cerar_status_string(cerar_status_t s) {
         case CERAR_ERR_CUDA: return "CUDA error";
         case CERAR_ERR_NOMEM: return "out of memory";
         case CERAR_ERR_TIMEOUT: return "device-side wait timed out";
+        case CERAR_ERR_TOO_LARGE: return "size beyond a fixed capacity";
     }
     return "unknown status";
 }
 
 const char* cerar_last_error(void) { return g_err.c_str(); }
+
+// for the library's other translation units
+void cerar_internal_set_error(const char* msg) { g_err = msg ? msg : ""; }
 
 cerar_status_t cerar_plan_create_ex(int N, int c, cerar_construction_t kind, double param,
                                     const cerar_options_t* opt, cerar_plan_t** out) {
