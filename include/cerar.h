@@ -216,12 +216,15 @@ uint64_t       cerar_launch_count(const cerar_plan_t* plan);
 cerar_status_t cerar_device_status(cerar_plan_t* plan, cerar_stream_t stream);
 
 /* Kernel selection for encode/decode: 0 = automatic, 1 = plain per-position
- * reference kernel, 2 = staged FMA kernel.  Returns the previous value. */
+ * kernel, 2 = staged FMA kernel, 3 = tensor-core (3 x TF32) kernel; a forced
+ * kernel that cannot take the shape makes the call fail instead of falling
+ * back.  Returns the previous value. */
 int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
 
 /* Process-wide tuning knobs of the staged kernel, for experiments: name is one of
  * "kc" (input rows per pipeline stage), "stages", "jt" (outputs per thread: 4, 8
- * or 16), "slabs" (position slabs per CTA); value 0 restores the default.
+ * or 16), "slabs" (position slabs per CTA), "tc_kc" / "tc_stages" (rows per stage and
+ * stages of the tensor-core kernel); value 0 restores the default.
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

@@ -15,7 +15,7 @@ import numpy as np
 from . import build as _build
 
 VANDERMONDE, EPSILON, KAPPA = 0, 1, 2
-KERNEL_AUTO, KERNEL_REF, KERNEL_STAGED = 0, 1, 2
+KERNEL_AUTO, KERNEL_REF, KERNEL_STAGED, KERNEL_TC = 0, 1, 2, 3
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "SINGULAR", 4: "NOT_CONVERGED",
                 5: "STATE", 6: "CUDA", 7: "NOMEM", 8: "TIMEOUT", 9: "TOO_LARGE"}

@@ -13,7 +13,7 @@
 #include "plan.hpp"
 
 namespace cerar {
-extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs;
+extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_dbg;
 }
 
 struct cerar_plan {
@@ -338,7 +338,7 @@ uint64_t cerar_launch_count(const cerar_plan_t* P) { return P ? P->launches : 0;
 int cerar_set_kernel_mode(cerar_plan_t* P, int mode) {
     if (!P) return -1;
     int old = P->kernel_mode;
-    if (mode >= 0 && mode <= 2) P->kernel_mode = mode;
+    if (mode >= 0 && mode <= 3) P->kernel_mode = mode;
     return old;
 }
 
@@ -363,6 +363,9 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "stages") cerar::g_tune_stages = value;
     else if (n == "jt") cerar::g_tune_jt = value;
     else if (n == "slabs") cerar::g_tune_slabs = value;
+    else if (n == "tc_kc") cerar::g_tune_tc_kc = value;
+    else if (n == "tc_stages") cerar::g_tune_tc_stages = value;
+    else if (n == "tc_dbg") cerar::g_tune_tc_dbg = value;
     else return -1;
     return 0;
 }

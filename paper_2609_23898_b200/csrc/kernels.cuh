@@ -34,11 +34,14 @@ struct RoundArgs {
     int N, c, k;            // round k in 1..L
 };
 
-enum { KERNEL_AUTO = 0, KERNEL_REF = 1, KERNEL_STAGED = 2 };
+enum { KERNEL_AUTO = 0, KERNEL_REF = 1, KERNEL_STAGED = 2, KERNEL_TC = 3 };
 
 // Returns cudaSuccess or the launch error.  *launches is incremented by the
 // number of kernels launched.
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches);
+// Tensor-core (tcgen05, 3 x TF32) contraction; tc_eligible says whether the shape fits it.
+bool tc_eligible(const ContractArgs& a);
+cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
 
 }  // namespace cerar
