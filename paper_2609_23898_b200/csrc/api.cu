@@ -13,7 +13,7 @@
 #include "plan.hpp"
 
 namespace cerar {
-extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_dbg;
+extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages;
 }
 
 struct cerar_plan {
@@ -365,7 +365,6 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "slabs") cerar::g_tune_slabs = value;
     else if (n == "tc_kc") cerar::g_tune_tc_kc = value;
     else if (n == "tc_stages") cerar::g_tune_tc_stages = value;
-    else if (n == "tc_dbg") cerar::g_tune_tc_dbg = value;
     else return -1;
     return 0;
 }

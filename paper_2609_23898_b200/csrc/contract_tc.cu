@@ -6,16 +6,21 @@
 // c >= 32 the FP32 FMA pipe cannot keep up with HBM (c/4 flop per byte), so the
 // products run on the 5th-generation tensor cores as 3 x TF32: every fp32 value
 // is split into hi = tf32(x) and lo = tf32(x - hi) and
-//   x*y ~ hi_x*hi_y + lo_x*hi_y + hi_x*lo_y           (relative error ~ 2^-22),
+//   x*y ~ lo_x*hi_y + hi_x*lo_y + hi_x*hi_y           (relative error ~ 2^-22),
 // accumulated in fp32 in tensor memory.
 //
-// Roles in a CTA of 10 warps (one CTA per SM, persistent over the tiles of one worker):
-//   warp 0      producer: TMA loads of [KC rows x 128 positions] chunks (swizzled 32 x KC boxes)
-//   warp 1      MMA issuer (one lane): tcgen05.mma kind::tf32, M=128, N=Npad, K=8; owns TMEM
-//   warps 2-5   epilogue: tcgen05.ld of the accumulator, scale, coalesced stores
-//   warps 6-9   splitter: rewrite a landed chunk as hi (in place) and lo (second buffer)
-// Both operands are "MN-major": positions (A) and outputs j (B) are the contiguous
-// dimension in shared memory, which is exactly how the data lies in HBM (no transpose).
+// One CTA of 10 warps per SM, persistent over the 128-position tiles of one worker:
+//   warp 0      producer: one TMA load per chunk ([KC rows] x [128 positions], row-major)
+//   warps 6-9   splitter: thread = position; reads its column of the chunk from shared
+//               memory, splits it, and writes hi | lo into tensor memory (tcgen05.st),
+//               where they are the A operand (rows = positions, columns = k)
+//   warp 1      MMA issuer (one lane): tcgen05.mma kind::tf32, A from TMEM, B = the
+//               coefficient matrix (hi and lo copies) resident in shared memory,
+//               M=128, N=Npad, K=8 per instruction; owns the TMEM allocation
+//   warps 2-5   epilogue: tcgen05.ld of the accumulator, scale, transpose through a
+//               shared-memory tile, one TMA store per 32 output rows
+// So the data tile is read from shared memory exactly once, and global memory is
+// touched only by TMA in rows of 512 contiguous bytes.  Every wait is bounded.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -29,8 +34,8 @@ namespace {
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr int TILE_M = 128;          // positions per tile = UMMA M
-constexpr int NSPLIT = 4;            // splitter warps
-constexpr int NUM_THREADS = 32 * (6 + NSPLIT);
+constexpr int NUM_THREADS = 320;
+constexpr int OUT_ROWS = 32;         // output rows per TMA store
 
 // ------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -64,16 +69,24 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
     }
 }
+// whole-warp wait with one outcome for all lanes (the .sync.aligned tcgen05 instructions
+// that follow need the warp converged)
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity) {
+    return __all_sync(0xffffffffu, mbar_wait_bounded(bar, parity) ? 1 : 0) != 0;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int u, uint32_t bar) {
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int y, int z, uint32_t src) {
     asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(u), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+        ::"l"(map), "r"(x), "r"(y), "r"(z), "r"(src) : "memory");
 }
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
@@ -82,11 +95,13 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[tmem] * B[smem descriptor]
+__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
     asm volatile(
         "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}\n"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
     uint32_t r[32];
@@ -102,18 +117,19 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ float tf32_rna(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
+// fp32 -> tf32 (10 explicit mantissa bits), round to nearest, ties away from zero
+__device__ __forceinline__ uint32_t tf32_bits(float x) { return (__float_as_uint(x) + 0x1000u) & 0xFFFFE000u; }
 
 // Shared-memory matrix descriptor for an MN-major 32-bit operand.  The only layout
 // the tensor core accepts for that case is the 128-byte swizzle with 32-byte atoms:
-// rows of 128 bytes (32 fp32 along M/N) at a 128-byte pitch along K, and inside every
-// group of 4 rows the 32-byte chunk index is XOR-ed with (row & 3) -- the pattern TMA
-// writes with CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B.  lbo = byte distance between
-// consecutive 32-element blocks along M/N, sbo = between consecutive 4-row groups.
+// rows of 128 bytes (32 fp32 along N) at a 128-byte pitch along K, and inside every
+// group of 4 rows the 32-byte chunk index is XOR-ed with (row & 3).  lbo = byte
+// distance between consecutive 32-element blocks along N, sbo = between 4-row groups.
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
     d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
@@ -124,54 +140,51 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes
     return d;
 }
 
-#ifdef CERAR_TC_DEBUG
-__device__ float g_dbg[1 << 16];
-#endif
-
 struct TcParams {
-    int K_rows;        // input rows that carry data (tensor-map rows); rows beyond read as zero
-    int K_pad;         // K_rows rounded up to KC
-    int KC;            // rows per pipeline stage (multiple of 8)
-    int stages;
+    int K_rows;        // physical input rows that carry data; rows beyond read as zero (TMA fill)
+    int K_pad;         // K_rows rounded up to a multiple of KC
+    int stages;        // shared-memory stages of raw chunks
+    int NA;            // A (hi|lo) chunk buffers in tensor memory
     int Npad;          // J rounded up to 32
-    int tmem_cols;     // power of two >= 2*Npad
-    int dbg;
+    int tmem_cols;     // power of two >= 2*Npad + NA*2*KC
 };
 
-// shared memory: [1024-aligned] B_hi | B_lo | stages x (raw/hi chunk, lo chunk) | barriers | tmem slot
-template <int DUMMY>
+// shared memory (1024-aligned): B_hi | B_lo | raw stages | 2 output tiles | barriers | tmem slot
+template <int KC>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_constant__ CUtensorMap tmap3,
+contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
                    const __grid_constant__ ContractArgs a, const __grid_constant__ TcParams tp) {
     extern __shared__ unsigned char smem_dyn[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int w = blockIdx.y;
-    const int KC = tp.KC, stages = tp.stages, Npad = tp.Npad, K_pad = tp.K_pad;
+    const int stages = tp.stages, NA = tp.NA, Npad = tp.Npad, K_pad = tp.K_pad;
     const int nkc = K_pad / KC;
     const int nblk = Npad / 32;
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* smem_al = smem_dyn + (smem_base - smem_u32(smem_dyn));
     const uint32_t b_bytes = (uint32_t)K_pad * Npad * 4u;            // one of B_hi / B_lo
-    const uint32_t chunk_bytes = (uint32_t)KC * TILE_M * 4u;         // one of hi / lo chunk
+    constexpr uint32_t chunk_bytes = (uint32_t)KC * TILE_M * 4u;
+    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * TILE_M * 4u;
     const uint32_t bhi_u32 = smem_base, blo_u32 = smem_base + b_bytes;
-    const uint32_t stage_u32 = smem_base + 2u * b_bytes;             // 1024-aligned: K_pad % 8 == 0
-    const uint32_t bar_u32 = stage_u32 + (uint32_t)stages * 2u * chunk_bytes;
-    // barriers: raw_full[s], lo_full[s], empty[s], acc_full[2], acc_empty[2]
-    const uint32_t raw_full = bar_u32, lo_full = bar_u32 + 8u * stages, empty = bar_u32 + 16u * stages;
-    const uint32_t acc_full = bar_u32 + 24u * stages, acc_empty = acc_full + 16u;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_al + (bar_u32 - smem_base) + 24u * stages + 32u);
+    const uint32_t raw_u32 = smem_base + 2u * b_bytes;
+    const uint32_t out_u32 = raw_u32 + (uint32_t)stages * chunk_bytes;
+    const uint32_t bar_u32 = out_u32 + 2u * out_bytes;
+    const uint32_t raw_full = bar_u32, raw_empty = raw_full + 8u * stages;
+    const uint32_t a_full = raw_empty + 8u * stages, a_empty = a_full + 8u * NA;
+    const uint32_t acc_full = a_empty + 8u * NA, acc_empty = acc_full + 16u;
+    const uint32_t out_full = acc_empty + 16u, out_free = out_full + 16u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_al + (out_free + 16u - smem_base));
+    const float* raw_s = reinterpret_cast<const float*>(smem_al + (raw_u32 - smem_base));
+    float* out_s = reinterpret_cast<float*>(smem_al + (out_u32 - smem_base));
 
     // ---------------- set-up
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) {
-            mbar_init(raw_full + 8u * s, 1);
-            mbar_init(lo_full + 8u * s, 1);
-            mbar_init(empty + 8u * s, 1);
-        }
+        for (int s = 0; s < stages; ++s) { mbar_init(raw_full + 8u * s, 1); mbar_init(raw_empty + 8u * s, 4); }
+        for (int b = 0; b < NA; ++b) { mbar_init(a_full + 8u * b, 4); mbar_init(a_empty + 8u * b, 1); }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(acc_full + 8u * b, 1);
-            mbar_init(acc_empty + 8u * b, 4);
+            mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, 4);
+            mbar_init(out_full + 8u * b, 4); mbar_init(out_free + 8u * b, 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -181,11 +194,11 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_const
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     {
-        // coefficients of this worker, split into tf32 hi / lo, written in the swizzled
-        // MN-major layout: block nb (32 outputs) | row k (128 B) | 32-byte chunk ^ (k & 3)
+        // coefficients of this worker, split into tf32 hi / lo, in the swizzled MN-major
+        // layout: block nb (32 outputs) | row k (128 B) | 32-byte chunk ^ (k & 3)
         const float* cf = a.coef + (size_t)w * a.K * a.J;
-        float* bhi = reinterpret_cast<float*>(smem_al);
-        float* blo = reinterpret_cast<float*>(smem_al + b_bytes);
+        uint32_t* bhi = reinterpret_cast<uint32_t*>(smem_al);
+        uint32_t* blo = reinterpret_cast<uint32_t*>(smem_al + b_bytes);
         for (int idx = threadIdx.x; idx < K_pad * Npad; idx += blockDim.x) {
             const int k = idx / Npad, j = idx - k * Npad;
             // physical input row k -> coefficient row (the row at skip_row is not part of Y: zero)
@@ -193,8 +206,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_const
             if (k < a.skip_row) src = k; else if (k > a.skip_row) src = k - 1;
             float v = 0.f;
             if (src >= 0 && src < a.K && j < a.J) v = cf[(size_t)src * a.J + j];
-            const float hi = tf32_rna(v);
-            const float lo = tf32_rna(v - hi);
+            const uint32_t hi = tf32_bits(v);
+            const uint32_t lo = tf32_bits(v - __uint_as_float(hi));
             const int nb = j >> 5, jj = j & 31;
             const int off = nb * (K_pad * 32) + k * 32 + ((((jj >> 3) ^ (k & 3)) << 3) | (jj & 7));
             bhi[off] = hi;
@@ -206,13 +219,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-#ifdef CERAR_TC_DEBUG
-    if (blockIdx.x == 0 && blockIdx.y == 0) {
-        const float* bh = reinterpret_cast<const float*>(smem_al);
-        for (int i = threadIdx.x; i < K_pad * Npad && i < 8192; i += blockDim.x) g_dbg[8192 + i] = bh[i];   // B_hi
-        if (threadIdx.x == 0) { g_dbg[20000] = __uint_as_float(tmem_base); g_dbg[20001] = (float)stages; g_dbg[20002] = (float)K_pad; }
-    }
-#endif
+    const uint32_t a_col0 = 2u * (uint32_t)Npad;            // A buffers start after the two accumulators
 
     const int64_t ntiles = a.tiles_per_worker;
     bool failed = false;
@@ -225,28 +232,20 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_const
                 const int q0 = (int)(t * TILE_M);
                 for (int kc = 0; kc < nkc; ++kc, ++it) {
                     const uint32_t s = it % stages, ph = (it / stages) & 1u;
-                    if (!mbar_wait_bounded(empty + 8u * s, ph ^ 1u)) { failed = true; break; }
+                    if (!mbar_wait_bounded(raw_empty + 8u * s, ph ^ 1u)) { failed = true; break; }
                     mbar_arrive_expect_tx(raw_full + 8u * s, chunk_bytes);
-                    const uint32_t dst = stage_u32 + s * 2u * chunk_bytes;
-                    if ((int64_t)q0 + TILE_M <= a.p) {
-                        // whole tile: one 4-D box = 4 blocks of 32 positions x KC rows (the smem layout of 4 boxes)
-                        tma_load_4d(dst, &tmap4, 0, kc * KC, q0 >> 5, w, raw_full + 8u * s);
-                    } else {
-                        // ragged last tile: position-bounded 3-D boxes, zero-filled beyond p
-#pragma unroll
-                        for (int b = 0; b < 4; ++b)
-                            tma_load_3d(dst + (uint32_t)b * KC * 128u, &tmap3, q0 + 32 * b, kc * KC, w, raw_full + 8u * s);
-                    }
+                    tma_load_3d(raw_u32 + s * chunk_bytes, &tmap_in, q0, kc * KC, w, raw_full + 8u * s);
                 }
             }
         }
     } else if (warp == 1) {
         // ================= MMA issuer
         if (lane == 0) {
-            // instruction descriptor: D=f32, A=B=tf32, both MN-major, N=Npad, M=128
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) |
+            // instruction descriptor: D=f32, A=B=tf32, A from TMEM (K-major), B MN-major, N=Npad, M=128
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) |
                                    ((uint32_t)(Npad >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
-            const uint32_t a_lbo = (uint32_t)KC * 128u, b_lbo = (uint32_t)K_pad * 128u;
+            const uint32_t b_lbo = (uint32_t)K_pad * 128u;
+            const uint64_t bhi0 = make_desc(bhi_u32, b_lbo, 512u), blo0 = make_desc(blo_u32, b_lbo, 512u);
             uint32_t it = 0, tc = 0;
             for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++tc) {
                 const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
@@ -254,24 +253,21 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_const
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * (uint32_t)Npad;
                 for (int kc = 0; kc < nkc; ++kc, ++it) {
-                    const uint32_t s = it % stages, ph = (it / stages) & 1u;
-                    if (!mbar_wait_bounded(lo_full + 8u * s, ph)) { failed = true; break; }
+                    const uint32_t ab = it % NA, ph = (it / NA) & 1u;
+                    if (!mbar_wait_bounded(a_full + 8u * ab, ph)) { failed = true; break; }
                     tc_fence_after();
-                    const uint32_t hi_u32 = stage_u32 + s * 2u * chunk_bytes, lo_u32 = hi_u32 + chunk_bytes;
+                    const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
                     int ksteps = KC / 8;
                     const int rows_left = tp.K_rows - kc * KC;               // rows with data in this chunk
                     if (rows_left < KC) ksteps = (rows_left + 7) / 8;
-                    for (int ks = 0; ks < ((tp.dbg & 4) ? 0 : ksteps); ++ks) {
-                        const uint64_t ahi = make_desc(hi_u32 + ks * 1024u, a_lbo, 512u);
-                        const uint64_t alo = make_desc(lo_u32 + ks * 1024u, a_lbo, 512u);
-                        const uint32_t boff = (uint32_t)(kc * KC + ks * 8) * 128u;
-                        const uint64_t bhi = make_desc(bhi_u32 + boff, b_lbo, 512u);
-                        const uint64_t blo = make_desc(blo_u32 + boff, b_lbo, 512u);
-                        tc_mma_tf32(d_tmem, alo, bhi, idesc, (kc | ks) != 0);
-                        tc_mma_tf32(d_tmem, ahi, blo, idesc, 1u);
-                        tc_mma_tf32(d_tmem, ahi, bhi, idesc, 1u);
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        // descriptor start address advances by 8 rows x 128 B (in 16-byte units)
+                        const uint64_t boff = (uint64_t)(((kc * KC + ks * 8) * 128) >> 4);
+                        tc_mma_tf32_ts(d_tmem, a_lo + ks * 8u, bhi0 + boff, idesc, (kc | ks) != 0);
+                        tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, blo0 + boff, idesc, 1u);
+                        tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, bhi0 + boff, idesc, 1u);
                     }
-                    tc_commit(empty + 8u * s);         // the stage is free once these MMAs have read it
+                    tc_commit(a_empty + 8u * ab);      // the A buffer is free once these MMAs have read it
                 }
                 if (failed) break;
                 tc_commit(acc_full + 8u * buf);        // the accumulator is complete
@@ -280,76 +276,80 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap4, const __grid_const
     } else if (warp < 6) {
         // ================= epilogue (warps 2..5; TMEM lanes 32*(warp%4) ..)
         const int qd = warp & 3;
-        float* out_w = a.out + (int64_t)w * a.out_wstride;
-        uint32_t tc = 0;
+        const int pos = qd * 32 + lane;
+        uint32_t tc = 0, oc = 0;
         for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++tc) {
             const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
-            if (!mbar_wait_bounded(acc_full + 8u * buf, aph)) { failed = true; break; }
+            if (!warp_wait(acc_full + 8u * buf, aph)) { failed = true; break; }
             tc_fence_after();
-            const int64_t pos = t * TILE_M + qd * 32 + lane;
-            const bool in_range = pos < a.p;
             const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + buf * (uint32_t)Npad;
-            for (int nb = 0; nb < nblk; ++nb) {
+            for (int nb = 0; nb < nblk; ++nb, ++oc) {
                 float v[32];
                 tc_ld32(taddr + (uint32_t)nb * 32u, v);
                 if (nb == nblk - 1) {
-                    // everything is in registers: hand the accumulator back before storing
+                    // everything is in registers: hand the accumulator back
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(acc_empty + 8u * buf);
                 }
-#ifdef CERAR_TC_DEBUG
-                if (blockIdx.x == 0 && blockIdx.y == 0 && tc == 0 && nb == 0)
-                    for (int j = 0; j < 32; ++j) g_dbg[(qd * 32 + lane) * 32 + j] = v[j];      // [0, 4096): D tile
-#endif
-                if (in_range && !(tp.dbg & 2)) {
-                    float* o = out_w + (int64_t)(nb * 32) * a.out_rstride + pos;
+                const uint32_t ob = oc & 1u, oph = (oc >> 1) & 1u;
+                if (!warp_wait(out_free + 8u * ob, oph ^ 1u)) { failed = true; break; }
+                float* o = out_s + (size_t)ob * (OUT_ROWS * TILE_M) + pos;
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (nb * 32 + j < a.J) o[(int64_t)j * a.out_rstride] = v[j] * a.scale;
-                }
-            }
-        }
-    } else {
-        // ================= splitter (warps 6..): every warp owns whole chunks (chunk it -> warp it % NSPLIT),
-        // so several chunks are being split at once; hi is written in place, lo to the second buffer
-        const int sw = warp - 6;
-        const int n4 = KC * TILE_M / 4;             // float4 per chunk
-        uint32_t it = 0;
-        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x) {
-            for (int kc = 0; kc < nkc; ++kc, ++it) {
-                if ((int)(it % NSPLIT) != sw) continue;
-                const uint32_t s = it % stages, ph = (it / stages) & 1u;
-                if (!mbar_wait_bounded(raw_full + 8u * s, ph)) { failed = true; break; }
-                float4* hi = reinterpret_cast<float4*>(smem_al + (stage_u32 - smem_base) + (size_t)s * 2u * chunk_bytes);
-                float4* lo = reinterpret_cast<float4*>(reinterpret_cast<unsigned char*>(hi) + chunk_bytes);
-                if (!(tp.dbg & 1)) {
-                    // 4 independent float4 per lane and step: loads first, then the stores
-                    for (int i0 = lane; i0 < n4; i0 += 128) {
-                        float4 x[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) x[u] = hi[i0 + 32 * u];          // n4 is a multiple of 128
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            float4 h, l;
-                            h.x = tf32_rna(x[u].x); l.x = tf32_rna(x[u].x - h.x);
-                            h.y = tf32_rna(x[u].y); l.y = tf32_rna(x[u].y - h.y);
-                            h.z = tf32_rna(x[u].z); l.z = tf32_rna(x[u].z - h.z);
-                            h.w = tf32_rna(x[u].w); l.w = tf32_rna(x[u].w - h.w);
-                            hi[i0 + 32 * u] = h;
-                            lo[i0 + 32 * u] = l;
+                for (int j = 0; j < 32; ++j) o[j * TILE_M] = v[j] * a.scale;
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(out_full + 8u * ob);
+                if (warp == 2 && lane == 0) {
+                    if (!mbar_wait_bounded(out_full + 8u * ob, oph)) {
+                        failed = true;
+                    } else {
+                        // rows beyond J and positions beyond p are clipped by the tensor map
+                        tma_store_3d(&tmap_out, (int)(t * TILE_M), nb * OUT_ROWS, w, out_u32 + ob * out_bytes);
+                        bulk_commit();
+                        if (oc >= 1) {                 // the store before this one has read its tile: free it
+                            bulk_wait_read_1();
+                            mbar_arrive(out_free + 8u * (ob ^ 1u));
                         }
                     }
                 }
-#ifdef CERAR_TC_DEBUG
-                if (blockIdx.x == 0 && blockIdx.y == 0 && it == 0) {
-                    const float* hf = reinterpret_cast<const float*>(hi);
-                    for (int i = lane; i < KC * TILE_M; i += 32) g_dbg[4096 + i] = hf[i];          // [4096, 4096+2048): hi chunk 0
+                if (warp == 2) failed = __any_sync(0xffffffffu, failed ? 1 : 0) != 0;
+                if (failed) break;
+            }
+        }
+        if (warp == 2 && lane == 0) bulk_wait_all();   // all output has left shared memory and is written
+    } else {
+        // ================= splitter (warps 6..9): thread = position
+        const int qd = warp & 3;
+        const int pos = qd * 32 + lane;
+        uint32_t it = 0;
+        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x) {
+            for (int kc = 0; kc < nkc; ++kc, ++it) {
+                const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                const uint32_t ab = it % NA, pa = (it / NA) & 1u;
+                if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
+                const float* col = raw_s + (size_t)s * (KC * TILE_M) + pos;
+                uint32_t hi[KC], lo[KC];
+#pragma unroll
+                for (int k = 0; k < KC; ++k) {
+                    const float x = col[k * TILE_M];
+                    hi[k] = tf32_bits(x);
+                    lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
                 }
-#endif
-                fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(lo_full + 8u * s);
+                if (lane == 0) mbar_arrive(raw_empty + 8u * s);        // the values are in registers
+                if (!warp_wait(a_empty + 8u * ab, pa ^ 1u)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC);
+#pragma unroll
+                for (int k8 = 0; k8 < KC / 8; ++k8) {
+                    tc_st8(ta + 8u * k8, hi + 8 * k8);
+                    tc_st8(ta + KC + 8u * k8, lo + 8 * k8);
+                }
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(a_full + 8u * ab);
             }
         }
     }
@@ -386,15 +386,40 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
+bool make_map(CUtensorMap* m, const float* base, int64_t p, int rows, int N, int64_t rstride, int64_t wstride,
+              int box_rows) {
+    cuuint64_t gdim[3] = {(cuuint64_t)p, (cuuint64_t)rows, (cuuint64_t)N};
+    cuuint64_t gstr[2] = {(cuuint64_t)rstride * 4, (cuuint64_t)wstride * 4};
+    cuuint32_t box[3] = {(cuuint32_t)TILE_M, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return get_encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), gdim, gstr, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int KC>
+cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a, const TcParams& tp,
+                      size_t smem, dim3 grid, cudaStream_t s) {
+    auto kern = contract_tc_kernel<KC>;
+    static thread_local size_t configured = 0;
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = smem;
+    }
+    kern<<<grid, NUM_THREADS, smem, s>>>(tin, tout, a, tp);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
-int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_dbg = 0;
+int g_tune_tc_kc = 0, g_tune_tc_stages = 0;
 
 bool tc_eligible(const ContractArgs& a) {
     if (a.J < 32 || a.J > 128) return false;      // N = J padded to 32; two coefficient copies must fit in smem
     if (a.p % 4 != 0 || a.p >= (int64_t)1 << 31) return false;
     if ((reinterpret_cast<uintptr_t>(a.in) & 15u) || (a.in_rstride % 4) || (a.in_wstride % 4)) return false;
-    if (a.in_rstride != a.p) return false;
+    if ((reinterpret_cast<uintptr_t>(a.out) & 15u) || (a.out_rstride % 4) || (a.out_wstride % 4)) return false;
     return get_encode_fn() != nullptr;
 }
 
@@ -403,88 +428,54 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     const bool has_skip = a.skip_row < a.K;                 // decode: one physical row is not part of Y
     tp.K_rows = a.K + (has_skip ? 1 : 0);
     tp.Npad = ((a.J + 31) / 32) * 32;
-    tp.dbg = g_tune_tc_dbg;
-    tp.tmem_cols = 32;
-    while (tp.tmem_cols < 2 * tp.Npad) tp.tmem_cols *= 2;
-    // rows per stage: as few padded rows as possible, then as large as possible, with at
-    // least NSPLIT stages in the shared memory that the two coefficient copies leave
-    const size_t budget = 225 * 1024;
+    // rows per chunk: as few padded rows as possible, then as large as possible, with at
+    // least 3 stages in the shared memory that the two coefficient copies leave
+    const size_t budget = 227 * 1024 - 1024;
     const int cands[4] = {40, 32, 24, 16};
     int best_kc = 0, best_pad = 1 << 30, best_stages = 0;
     for (int ci = 0; ci < 4; ++ci) {
         const int kc = cands[ci];
         if (g_tune_tc_kc && kc != g_tune_tc_kc) continue;
+        if (2 * tp.Npad + 2 * 2 * kc > 512) continue;       // two accumulators + at least two A buffers
         const int kpad = ((tp.K_rows + kc - 1) / kc) * kc;
-        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp.Npad * 4 + 256;
-        const size_t stage_c = 2 * (size_t)kc * TILE_M * 4;
-        if (fixed_c + NSPLIT * stage_c > budget) continue;
+        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp.Npad * 4 + 2 * OUT_ROWS * TILE_M * 4 + 512;
+        const size_t stage_c = (size_t)kc * TILE_M * 4;
+        if (fixed_c + 3 * stage_c > budget) continue;
         int st = (int)((budget - fixed_c) / stage_c);
-        if (st > 12) st = 12;
+        if (st > 8) st = 8;
         if (g_tune_tc_stages && g_tune_tc_stages < st) st = g_tune_tc_stages;
-        st -= st % NSPLIT;
-        if (st < NSPLIT) continue;
+        if (st < 2) continue;
         if (kpad < best_pad) { best_pad = kpad; best_kc = kc; best_stages = st; }
     }
     if (!best_kc) return cudaErrorInvalidConfiguration;
-    // Chunk i is split by warp i % NSPLIT and lives in stage i % stages.  With stages a
-    // multiple of NSPLIT the two uses of a stage that follow each other belong to the same
-    // warp, so a warp never waits on a barrier phase that is more than one step ahead.
-    tp.KC = best_kc;
+    const int KC = best_kc;
     tp.K_pad = best_pad;
     tp.stages = best_stages;
-    const size_t chunk_bytes = (size_t)tp.KC * TILE_M * 4;
-    const size_t fixed = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + 256;
-    const int stages = tp.stages;
-    const size_t smem = fixed + (size_t)stages * 2 * chunk_bytes + (size_t)stages * 24;
+    tp.NA = (512 - 2 * tp.Npad) / (2 * KC);
+    if (tp.NA > 4) tp.NA = 4;
+    tp.tmem_cols = 32;
+    while (tp.tmem_cols < 2 * tp.Npad + tp.NA * 2 * KC) tp.tmem_cols *= 2;
+    const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * TILE_M * 4 +
+                        2 * OUT_ROWS * TILE_M * 4 + 512;
 
-    // Tensor maps over the input.  tmap3: (positions, rows, workers), boxes of 32 positions x KC
-    // rows, bounded by p (ragged last tile).  tmap4: (32 positions, rows, blocks of 32 positions,
-    // workers) over the whole blocks only: one box brings a whole 128-position chunk.
-    CUtensorMap tmap3, tmap4;
-    {
-        cuuint64_t gdim[3] = {(cuuint64_t)a.p, (cuuint64_t)tp.K_rows, (cuuint64_t)a.N};
-        cuuint64_t gstr[2] = {(cuuint64_t)a.in_rstride * 4, (cuuint64_t)a.in_wstride * 4};
-        cuuint32_t box[3] = {32, (cuuint32_t)tp.KC, 1};
-        cuuint32_t estr[3] = {1, 1, 1};
-        CUresult r = get_encode_fn()(&tmap3, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(a.in), gdim, gstr,
-                                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
-                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    }
-    {
-        const cuuint64_t nblocks = (cuuint64_t)(a.p / 32) > 0 ? (cuuint64_t)(a.p / 32) : 1;
-        cuuint64_t gdim[4] = {32, (cuuint64_t)tp.K_rows, nblocks, (cuuint64_t)a.N};
-        cuuint64_t gstr[3] = {(cuuint64_t)a.in_rstride * 4, 128, (cuuint64_t)a.in_wstride * 4};
-        cuuint32_t box[4] = {32, (cuuint32_t)tp.KC, 4, 1};
-        cuuint32_t estr[4] = {1, 1, 1, 1};
-        CUresult r = get_encode_fn()(&tmap4, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(a.in), gdim, gstr,
-                                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
-                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
-    }
+    CUtensorMap tin, tout;
+    if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, KC)) return cudaErrorInvalidValue;
+    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, OUT_ROWS)) return cudaErrorInvalidValue;
 
-    auto kern = contract_tc_kernel<0>;
-    static thread_local size_t configured = 0;
-    if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        configured = smem;
-    }
     a.tiles_per_worker = (int)((a.p + TILE_M - 1) / TILE_M);
     int64_t per_worker = num_sms / a.N;
     if (per_worker < 1) per_worker = 1;
     if (per_worker > a.tiles_per_worker) per_worker = a.tiles_per_worker;
     dim3 grid((unsigned)per_worker, (unsigned)a.N);
-    kern<<<grid, NUM_THREADS, smem, s>>>(tmap4, tmap3, a, tp);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e;
+    switch (KC) {
+        case 40: e = launch_kc<40>(tin, tout, a, tp, smem, grid, s); break;
+        case 32: e = launch_kc<32>(tin, tout, a, tp, smem, grid, s); break;
+        case 24: e = launch_kc<24>(tin, tout, a, tp, smem, grid, s); break;
+        default: e = launch_kc<16>(tin, tout, a, tp, smem, grid, s); break;
+    }
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }
-
-#ifdef CERAR_TC_DEBUG
-extern "C" int cerar_debug_fetch(float* out, int n) {
-    return (int)cudaMemcpyFromSymbol(out, g_dbg, (size_t)n * 4);
-}
-#endif
 
 }  // namespace cerar
