@@ -9,14 +9,15 @@
 //   x*y ~ lo_x*hi_y + hi_x*lo_y + hi_x*hi_y           (relative error ~ 2^-22),
 // accumulated in fp32 in tensor memory.
 //
-// One CTA of 10 warps per SM, persistent over the 128-position tiles of one worker:
+// One CTA of 11 warps per SM, persistent over the 128-position tiles of one worker:
 //   warp 0      producer: one TMA load per chunk ([KC rows] x [128 positions], row-major)
 //   warps 6-9   splitter: thread = position; reads its column of the chunk from shared
 //               memory, splits it, and writes hi | lo into tensor memory (tcgen05.st),
 //               where they are the A operand (rows = positions, columns = k)
-//   warp 1      MMA issuer (one lane): tcgen05.mma kind::tf32, A from TMEM, B = the
+//   warps 1,10  MMA issuers (one lane each, even / odd tiles, so that one can issue while
+//               the other drains): tcgen05.mma kind::tf32, A from TMEM, B = the
 //               coefficient matrix (hi and lo copies) resident in shared memory,
-//               M=128, N=Npad, K=8 per instruction; owns the TMEM allocation
+//               M=128, N=Npad, K=8 per instruction; warp 1 owns the TMEM allocation
 //   warps 2-5   epilogue: tcgen05.ld of the accumulator, scale, transpose through a
 //               shared-memory tile, one TMA store per 32 output rows
 // So the data tile is read from shared memory exactly once, and global memory is
@@ -34,7 +35,7 @@ namespace {
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 constexpr int TILE_M = 128;          // positions per tile = UMMA M
-constexpr int NUM_THREADS = 320;
+constexpr int NUM_THREADS = 32 * 11;
 constexpr int OUT_ROWS = 32;         // output rows per TMA store
 
 // ------------------------------------------------------------------ PTX helpers
@@ -160,6 +161,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     const int stages = tp.stages, NA = tp.NA, Npad = tp.Npad, K_pad = tp.K_pad;
     const int nkc = K_pad / KC;
     const int nblk = Npad / 32;
+    const uint32_t NAh = (uint32_t)NA / 2u;      // A buffers per MMA issuer
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* smem_al = smem_dyn + (smem_base - smem_u32(smem_dyn));
@@ -238,22 +240,24 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 }
             }
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer
+    } else if (warp == 1 || warp == 10) {
+        // ================= MMA issuers: issuer m takes tiles m, m+2, ... into accumulator m
         if (lane == 0) {
+            const uint32_t m = (warp == 1) ? 0u : 1u;
             // instruction descriptor: D=f32, A=B=tf32, A from TMEM (K-major), B MN-major, N=Npad, M=128
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) |
                                    ((uint32_t)(Npad >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
             const uint32_t b_lbo = (uint32_t)K_pad * 128u;
             const uint64_t bhi0 = make_desc(bhi_u32, b_lbo, 512u), blo0 = make_desc(blo_u32, b_lbo, 512u);
-            uint32_t it = 0, tc = 0;
-            for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++tc) {
-                const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
-                if (!mbar_wait_bounded(acc_empty + 8u * buf, aph ^ 1u)) { failed = true; break; }
+            const uint32_t d_tmem = tmem_base + m * (uint32_t)Npad;
+            uint32_t tc = m;
+            for (int64_t t = blockIdx.x + (int64_t)m * gridDim.x; t < ntiles && !failed; t += 2 * (int64_t)gridDim.x, tc += 2) {
+                const uint32_t aph = (tc >> 1) & 1u;
+                if (!mbar_wait_bounded(acc_empty + 8u * m, aph ^ 1u)) { failed = true; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * (uint32_t)Npad;
-                for (int kc = 0; kc < nkc; ++kc, ++it) {
-                    const uint32_t ab = it % NA, ph = (it / NA) & 1u;
+                for (int kc = 0; kc < nkc; ++kc) {
+                    const uint32_t seq = (tc >> 1) * (uint32_t)nkc + (uint32_t)kc;
+                    const uint32_t ab = m * NAh + seq % NAh, ph = (seq / NAh) & 1u;
                     if (!mbar_wait_bounded(a_full + 8u * ab, ph)) { failed = true; break; }
                     tc_fence_after();
                     const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
@@ -270,7 +274,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     tc_commit(a_empty + 8u * ab);      // the A buffer is free once these MMAs have read it
                 }
                 if (failed) break;
-                tc_commit(acc_full + 8u * buf);        // the accumulator is complete
+                tc_commit(acc_full + 8u * m);          // the accumulator is complete
             }
         }
     } else if (warp < 6) {
@@ -322,11 +326,13 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         // ================= splitter (warps 6..9): thread = position
         const int qd = warp & 3;
         const int pos = qd * 32 + lane;
-        uint32_t it = 0;
-        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x) {
+        uint32_t it = 0, tc = 0;
+        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++tc) {
             for (int kc = 0; kc < nkc; ++kc, ++it) {
                 const uint32_t s = it % stages, ph = (it / stages) & 1u;
-                const uint32_t ab = it % NA, pa = (it / NA) & 1u;
+                // A buffers are split between the two MMA issuers: tile parity picks the half
+                const uint32_t seq = (tc >> 1) * (uint32_t)nkc + (uint32_t)kc;
+                const uint32_t ab = (tc & 1u) * NAh + seq % NAh, pa = (seq / NAh) & 1u;
                 if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
                 const float* col = raw_s + (size_t)s * (KC * TILE_M) + pos;
                 uint32_t hi[KC], lo[KC];
@@ -453,6 +459,7 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     tp.stages = best_stages;
     tp.NA = (512 - 2 * tp.Npad) / (2 * KC);
     if (tp.NA > 4) tp.NA = 4;
+    tp.NA -= tp.NA % 2;                                   // one half per MMA issuer
     tp.tmem_cols = 32;
     while (tp.tmem_cols < 2 * tp.Npad + tp.NA * 2 * KC) tp.tmem_cols *= 2;
     const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * TILE_M * 4 +
