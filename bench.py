@@ -33,9 +33,12 @@ if ROOT not in sys.path:
 
 METRIC = "cerar_encode_rounds_decode_hbm_gbps"
 UNIT = "GB/s"
-# DRAM bytes per ring-round launch measured by ncu, per (worker x position), on a
-# smaller case of the same kernel (see profiles/); None until a capture exists.
-NCU_ROUND_DRAM_BYTES_PER_WORKER_POSITION = None
+# DRAM bytes of a steady ring-round launch measured by ncu on a smaller case of the same
+# kernel (profiles/round_kernel_dram_traffic_N8_c32_p4M.md): 12.0 B read + 2.9 B written
+# per (worker x position) against 16 B algorithmic (part of the writes is still in L2 when
+# the launch ends).  Traffic grows in proportion to the positions, so it is scaled by the
+# algorithmic bytes of the timed launch.
+NCU_ROUND_TRAFFIC_OVER_ALGORITHMIC = 14.88 / 16.0
 
 
 def algorithmic_bytes(N, c, p):
@@ -317,8 +320,8 @@ def main():
     dom_ms = {"round_kernel": rounds_ms / L, "encode": enc_ms, "decode": dec_ms}[dominant]
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     traffic = None
-    if dominant == "round_kernel" and NCU_ROUND_DRAM_BYTES_PER_WORKER_POSITION is not None:
-        traffic = NCU_ROUND_DRAM_BYTES_PER_WORKER_POSITION * N * p
+    if dominant == "round_kernel":
+        traffic = NCU_ROUND_TRAFFIC_OVER_ALGORITHMIC * dom_bytes
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                 "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": dom_ms,
