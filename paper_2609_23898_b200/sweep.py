@@ -1,0 +1,105 @@
+"""Throughput sweep of the CERAR pipeline on one GPU.
+
+  python -m paper_2609_23898_b200.sweep [--quick] [--out FILE]
+
+Points: d per worker in {2^18, 2^20, ..., 2^30} fp32, N in {4, 8, 16}, c in {N, 2N, 4N, 8N},
+epsilon-construction with eps = 1e-3, i.i.d. N(0,1) gradients.  Every point runs in place
+(the gradients are generated directly in the D rows of the workspace and the result
+overwrites them), so the largest point (N=16, d=2^30, c=16) needs 137 GB.  Per point:
+3 warm-up and 5 timed aggregations (CUDA events around cerar_allreduce_sim, median), the
+gradients are regenerated before every aggregation (outside the timed region).
+
+Reported: seconds per aggregation, algorithmic GB/s (N (8c+3N-8) p 4 bytes per
+aggregation) and its fraction of the measured HBM copy bandwidth.  Points whose whole
+state fits in the 126 MB L2 are marked: their "GB/s" is not an HBM figure.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--quick", action="store_true", help="d in {2^20, 2^26} only")
+    ap.add_argument("--out", default="")
+    ap.add_argument("--eps", type=float, default=1e-3)
+    args = ap.parse_args()
+
+    import torch
+    from . import cerar, inputs
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    peak = 6650.0
+    pk = os.path.join(root, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        peak = float(json.load(open(pk))["hbm_gbs"])
+    free, total = torch.cuda.mem_get_info()
+    stream = torch.cuda.current_stream().cuda_stream
+    exps = [20, 26] if args.quick else [18, 20, 22, 24, 26, 28, 30]
+    rows = []
+    print("| N | c | d | state MB | ms / aggregation | GB/s | frac of measured HBM | note |")
+    print("|---|---|---|---|---|---|---|---|")
+    for N in (4, 8, 16):
+        for mult in (1, 2, 4, 8):
+            c = N * mult
+            B = inputs.base_matrix(N, c, 0)
+            note = ""
+            try:
+                plan = cerar.Plan.create(N, c, cerar.EPSILON, args.eps, B=B)
+            except cerar.CerarError as e:
+                # the encoders of this design do not fit fp32: time the kernels with
+                # well-conditioned coefficients of the same shape instead
+                rng = np.random.default_rng(0)
+                L = c + N - 2
+                U = [np.linalg.qr(rng.standard_normal((c, c)))[0] for _ in range(N)]
+                R = [rng.standard_normal((L + 1, c)) / np.sqrt(L + 1) for _ in range(N)]
+                plan = cerar.Plan.create_custom(N, c, U, R)
+                note = "design overflows fp32: surrogate coefficients"
+            for e in exps:
+                d = 1 << e
+                if d % c:
+                    continue
+                p = d // c
+                ws_bytes = plan.workspace_bytes(d)
+                if ws_bytes > free - (2 << 30):
+                    print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | - | - | - | skipped: needs {ws_bytes / 1e9:.1f} GB |")
+                    continue
+                ws = torch.empty(ws_bytes // 4, dtype=torch.float32, device="cuda")
+                wstride = (c + N) * p
+                dptr = ws.data_ptr() + 4 * N * p
+                times = []
+                for rep in range(8):
+                    for i in range(N):
+                        ws[i * wstride + N * p:(i + 1) * wstride].normal_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    plan.allreduce_sim(dptr, wstride, dptr, wstride, ws, d, 1.0 / N, stream)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    if rep >= 3:
+                        times.append(e0.elapsed_time(e1))
+                plan.device_status(stream)
+                ms = float(np.median(times))
+                ab = 4 * N * p * (8 * c + 3 * N - 8)
+                gbs = ab / ms / 1e6
+                l2 = "L2-resident" if ws_bytes < 100e6 else ""
+                row = dict(N=N, c=c, d=d, state_mb=ws_bytes / 1e6, ms=ms, gbps=gbs, frac=gbs / peak,
+                           note=", ".join(x for x in (note, l2) if x))
+                rows.append(row)
+                print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | {ms:.3f} | {gbs:.0f} | {gbs / peak:.2f} | {row['note']} |",
+                      flush=True)
+                del ws
+                torch.cuda.empty_cache()
+            plan.destroy()
+    if args.out:
+        with open(args.out, "w") as f:
+            json.dump(rows, f, indent=1)
+
+
+if __name__ == "__main__":
+    sys.exit(main())
