@@ -184,6 +184,22 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Slowest rank's time (the contract's max over ranks)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(bytes_per_replica: int, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank moves the same algorithmic bytes; GB/s of the whole job."""
+    return world * bytes_per_replica / (ms_per_step * 1e-3) / 1e9
+
+
 def workload_name(key, cfg):
     return (f"{key}: N={cfg['N']} c={cfg['c']} {cfg['kind']}({cfg['param']:g}) d={cfg['d']} fp32/worker "
             f"{cfg['workload']} gradients")
@@ -304,11 +320,8 @@ def main():
     enc_ms = float(np.mean([ev[s][0].elapsed_time(ev[s][1]) for s in range(K)]))
     dec_ms = float(np.mean([ev[s][L + 1].elapsed_time(ev[s][L + 2]) for s in range(K)]))
     rnd_ms = [float(np.mean([ev[s][k].elapsed_time(ev[s][k + 1]) for s in range(K)])) for k in range(1, L + 1)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = float(t.item()) / K
-    value = world * ab["total"] / (ms_per_step * 1e-3) / 1e9
+    ms_per_step = max_over_ranks(total_ms, world, dev) / K
+    value = whole_job_value(ab["total"], world, ms_per_step)
 
     peak, peak_kind = load_peaks()
     rounds_bytes = sum(round_bytes(N, c, p, k) for k in range(1, L + 1))
@@ -379,16 +392,13 @@ def main():
             plan.allreduce_sim_host(h_in, d_e2e, h_out, d_e2e, ws, d_e2e, scale, stream)
         e1.record()
         sync_all()
-        te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        ms_e2e = float(te.item()) / ksteps
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev) / ksteps
         abe = algorithmic_bytes(N, c, pe)["total"]
-        line["e2e"] = {"value": world * abe / (ms_e2e * 1e-3) / 1e9, "unit": UNIT,
+        line["e2e"] = {"value": whole_job_value(abe, world, ms_e2e), "unit": UNIT,
                        "h2d_bytes_per_step": N * d_e2e * 4, "d2h_bytes_per_step": N * d_e2e * 4,
                        "ms_per_step": ms_e2e, "steps": ksteps, "d": d_e2e,
-                       "note": "pinned host gradients -> device workspace rows, in-place pipeline, results back to "
-                               "pinned host; PCIe copies inside the timed region"}
+                       "note": "cerar_allreduce_sim_host: pinned host gradients in, pinned host results out; position "
+                               "slices overlap H2D, kernels (in place) and D2H; all PCIe copies inside the timed region"}
         plan.device_status(stream)
         del h_in, h_out
 

@@ -165,12 +165,15 @@ cerar_status_t cerar_allreduce_sim(cerar_plan_t* plan, const float* grads, int64
                                    float* out, int64_t out_stride, float* ws, int64_t d,
                                    float scale, cerar_stream_t stream);
 
-/* Same pipeline with HOST gradients and results: copies worker i's gradient
- * (h_grads + i*h_grads_stride, d floats; pinned memory makes the copies
- * asynchronous) into the D rows of the device workspace, runs encode, the L
- * rounds and decode in place, and copies the results back to
- * h_out + i*h_out_stride.  Work is issued on `stream`; the call returns after
- * everything is enqueued.  ws: device, cerar_workspace_bytes(plan, d). */
+/* Same pipeline with HOST gradients and results (pinned memory makes the copies
+ * asynchronous and lets them overlap the kernels).  Positions are independent, so
+ * the library cuts the job into position slices: while slice i is encoded, sent
+ * round the ring and decoded in place on `stream`, slice i+1 is copied in and
+ * slice i-1 copied out on two internal copy streams.  worker i's gradient is at
+ * h_grads + i*h_grads_stride, its result goes to h_out + i*h_out_stride (d floats
+ * each).  ws: device scratch of cerar_workspace_bytes(plan, d) bytes (only three
+ * slice-sized parts of it are used).  The call returns after everything is
+ * enqueued; `stream` is complete when all results are on the host. */
 cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* plan, const float* h_grads,
                                         int64_t h_grads_stride, float* h_out,
                                         int64_t h_out_stride, float* ws, int64_t d,

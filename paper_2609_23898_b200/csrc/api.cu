@@ -22,6 +22,10 @@ struct cerar_plan {
     float* d_U = nullptr;
     float* d_R = nullptr;
     int* d_status = nullptr;
+    // copy streams and events of the host-buffer entry point (created with the plan)
+    cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_h2d[3] = {nullptr, nullptr, nullptr}, ev_comp[3] = {nullptr, nullptr, nullptr},
+                ev_d2h[3] = {nullptr, nullptr, nullptr};
     int device = -1;
     int num_sms = 0;
     bool on_device = false;
@@ -78,6 +82,14 @@ cerar_status_t upload(cerar_plan* P) {
     if ((e = cudaMemcpy(P->d_R, hR.data(), hR.size() * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess)
         return cuda_fail(e, "upload R");
     if ((e = cudaMemset(P->d_status, 0, sizeof(int))) != cudaSuccess) return cuda_fail(e, "memset status");
+    if ((e = cudaStreamCreateWithFlags(&P->s_h2d, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e, "stream");
+    if ((e = cudaStreamCreateWithFlags(&P->s_d2h, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e, "stream");
+    if ((e = cudaEventCreateWithFlags(&P->ev_start, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e, "event");
+    for (int b = 0; b < 3; ++b) {
+        if ((e = cudaEventCreateWithFlags(&P->ev_h2d[b], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e, "event");
+        if ((e = cudaEventCreateWithFlags(&P->ev_comp[b], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e, "event");
+        if ((e = cudaEventCreateWithFlags(&P->ev_d2h[b], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e, "event");
+    }
     P->on_device = true;
     return CERAR_OK;
 }
@@ -185,6 +197,14 @@ void cerar_plan_destroy(cerar_plan_t* P) {
     if (!P) return;
     if (P->on_device || P->d_U || P->d_R || P->d_status) {
         cudaFree(P->d_U); cudaFree(P->d_R); cudaFree(P->d_status);
+        if (P->s_h2d) cudaStreamDestroy(P->s_h2d);
+        if (P->s_d2h) cudaStreamDestroy(P->s_d2h);
+        if (P->ev_start) cudaEventDestroy(P->ev_start);
+        for (int b = 0; b < 3; ++b) {
+            if (P->ev_h2d[b]) cudaEventDestroy(P->ev_h2d[b]);
+            if (P->ev_comp[b]) cudaEventDestroy(P->ev_comp[b]);
+            if (P->ev_d2h[b]) cudaEventDestroy(P->ev_d2h[b]);
+        }
     }
     delete P;
 }
@@ -303,21 +323,57 @@ cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* P, const float* h_grads, i
     if (!h_grads || !h_out || !ws) return fail(CERAR_ERR_INVALID_ARG, "NULL buffer");
     if (h_grads_stride < d || h_out_stride < d) return fail(CERAR_ERR_SHAPE, "stride < d");
     const int N = P->host.N, c = P->host.c;
-    const int64_t wstride = (int64_t)(c + N) * p;
-    float* drows = ws + (int64_t)N * p;             // worker 0's D rows: d contiguous floats
     cudaStream_t s = (cudaStream_t)stream;
-    for (int i = 0; i < N; ++i) {
-        cudaError_t e = cudaMemcpyAsync(drows + i * wstride, h_grads + i * h_grads_stride, (size_t)d * 4,
-                                        cudaMemcpyHostToDevice, s);
-        if (e != cudaSuccess) return cuda_fail(e, "H2D copy");
+    cudaError_t e;
+    // Positions are independent, so the job is cut into slices of ps positions that flow
+    // through three slice-sized workspaces carved out of ws: the H2D copy of slice i+1 and
+    // the D2H copy of slice i-1 (two copy streams, PCIe is full duplex) overlap the kernels
+    // of slice i, which run in place on `stream`.
+    int64_t ps = p;
+    if (p >= 3 * 262144) {
+        int64_t nsl = p / 1048576;
+        if (nsl < 3) nsl = 3;
+        if (nsl > 64) nsl = 64;
+        ps = ((p + nsl - 1) / nsl + 127) / 128 * 128;
     }
-    st = cerar_allreduce_sim(P, drows, wstride, drows, wstride, ws, d, scale, stream);
-    if (st != CERAR_OK) return st;
-    for (int i = 0; i < N; ++i) {
-        cudaError_t e = cudaMemcpyAsync(h_out + i * h_out_stride, drows + i * wstride, (size_t)d * 4,
-                                        cudaMemcpyDeviceToHost, s);
-        if (e != cudaSuccess) return cuda_fail(e, "D2H copy");
+    const int64_t nslices = (p + ps - 1) / ps;
+    const int nbuf = nslices >= 3 ? 3 : 1;
+    const int64_t slot_floats = (int64_t)N * (c + N) * ps;      // one slice workspace
+    if ((e = cudaEventRecord(P->ev_start, s)) != cudaSuccess) return cuda_fail(e, "event record");
+    if ((e = cudaStreamWaitEvent(P->s_h2d, P->ev_start, 0)) != cudaSuccess) return cuda_fail(e, "stream wait");
+    if ((e = cudaStreamWaitEvent(P->s_d2h, P->ev_start, 0)) != cudaSuccess) return cuda_fail(e, "stream wait");
+    for (int64_t i = 0; i < nslices; ++i) {
+        const int b = (int)(i % nbuf);
+        const int64_t q0 = i * ps;
+        const int64_t pl = (p - q0 < ps) ? (p - q0) : ps;      // positions in this slice
+        float* wsl = ws + b * slot_floats;
+        const int64_t wstride = (int64_t)(c + N) * pl;
+        float* drows = wsl + (int64_t)N * pl;
+        if (i >= nbuf && (e = cudaStreamWaitEvent(P->s_h2d, P->ev_d2h[b], 0)) != cudaSuccess) return cuda_fail(e, "stream wait");
+        for (int w = 0; w < N; ++w) {
+            e = cudaMemcpy2DAsync(drows + w * wstride, (size_t)pl * 4, h_grads + w * h_grads_stride + q0, (size_t)p * 4,
+                                  (size_t)pl * 4, (size_t)c, cudaMemcpyHostToDevice, P->s_h2d);
+            if (e != cudaSuccess) return cuda_fail(e, "H2D copy");
+        }
+        if ((e = cudaEventRecord(P->ev_h2d[b], P->s_h2d)) != cudaSuccess) return cuda_fail(e, "event record");
+        if ((e = cudaStreamWaitEvent(s, P->ev_h2d[b], 0)) != cudaSuccess) return cuda_fail(e, "stream wait");
+        st = cerar_allreduce_sim(P, drows, wstride, drows, wstride, wsl, (int64_t)c * pl, scale, stream);
+        if (st != CERAR_OK) return st;
+        if ((e = cudaEventRecord(P->ev_comp[b], s)) != cudaSuccess) return cuda_fail(e, "event record");
+        if ((e = cudaStreamWaitEvent(P->s_d2h, P->ev_comp[b], 0)) != cudaSuccess) return cuda_fail(e, "stream wait");
+        for (int w = 0; w < N; ++w) {
+            e = cudaMemcpy2DAsync(h_out + w * h_out_stride + q0, (size_t)p * 4, drows + w * wstride, (size_t)pl * 4,
+                                  (size_t)pl * 4, (size_t)c, cudaMemcpyDeviceToHost, P->s_d2h);
+            if (e != cudaSuccess) return cuda_fail(e, "D2H copy");
+        }
+        if ((e = cudaEventRecord(P->ev_d2h[b], P->s_d2h)) != cudaSuccess) return cuda_fail(e, "event record");
     }
+    // the caller's stream resumes when the last results are on the host
+    for (int b = 0; b < nbuf; ++b)
+        if ((e = cudaStreamWaitEvent(s, P->ev_d2h[b], 0)) != cudaSuccess) return cuda_fail(e, "stream wait");
+    // counters describe the whole job, not the last slice
+    P->cur_d = d;
+    P->bytes_forwarded = (uint64_t)4 * (uint64_t)p * (uint64_t)P->host.L;
     return CERAR_OK;
 }
 

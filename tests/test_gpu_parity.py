@@ -53,7 +53,9 @@ def _check_stages(lib_res, ora, tol_out, N):
 # positions), p not a multiple of 4 (plain kernels), tiny p, c = N, N = 2
 SHAPES = [(4, 8, 8192), (4, 8, 8192 + 260), (3, 5, 1031), (2, 2, 4), (5, 9, 7), (4, 12, 3000),
           (8, 20, 2052), (8, 32, 4100), (4, 16, 16384 + 12), (16, 16, 1028), (4, 4, 100000),
-          (8, 64, 1540), (6, 24, 2048)]
+          (8, 64, 1540), (6, 24, 2048),
+          # tensor-core kernel: one tile, ragged tiles, c not a multiple of 32, c = 128
+          (4, 32, 128), (8, 48, 260), (4, 96, 388), (16, 128, 520), (8, 40, 1028)]
 
 
 @pytest.mark.parametrize("N,c,p", SHAPES)
@@ -96,6 +98,29 @@ def test_staged_kernel_is_what_runs(cerar_mod):
     g2 = _inputs().gradients_numpy(N, c * 1031, "normal", seed=2)
     with pytest.raises(cerar_mod.CerarError):
         run_library(plan2, g2, 1.0)
+
+
+def test_tensor_core_kernel_is_what_runs(cerar_mod):
+    """Forcing the tensor-core kernel works on an eligible shape (so that 'auto' at
+    c >= 32 is not silently the FMA kernel), agrees with the FMA kernel to TF32x3
+    accuracy, and refuses shapes it cannot take."""
+    N, c, p = 8, 32, 2048 + 132
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(3))
+    g = _inputs().gradients_numpy(N, c * p, "normal", seed=5)
+    ora = run_oracle(des.U, des.R, g, 1.0)
+    outs = {}
+    for mode in (cerar_mod.KERNEL_TC, cerar_mod.KERNEL_STAGED):
+        plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+        plan.set_kernel_mode(mode)
+        res = run_library(plan, g, 1.0)
+        _check_stages(res, ora, OUT_TOL, N)
+        outs[mode] = res["out"]
+    assert rel_l2(outs[cerar_mod.KERNEL_TC], outs[cerar_mod.KERNEL_STAGED]) < 2e-6
+    des16 = Dz.custom_orthogonal(4, 16, np.random.default_rng(3))
+    plan = cerar_mod.Plan.create_custom(4, 16, des16.U, des16.R)
+    plan.set_kernel_mode(cerar_mod.KERNEL_TC)
+    with pytest.raises(cerar_mod.CerarError):
+        run_library(plan, _inputs().gradients_numpy(4, 16 * 1024, "normal", seed=5), 1.0)
 
 
 @pytest.mark.parametrize("N,c,eps,p", [(4, 4, 1e-3, 5000), (8, 8, 1e-3, 2052), (16, 16, 1e-3, 1028)])
@@ -225,22 +250,28 @@ def test_state_machine_and_counters(cerar_mod):
     plan.device_status()
 
 
-def test_host_buffer_entry_point(cerar_mod):
+@pytest.mark.parametrize("N,c,p", [(4, 8, 2048 + 4), (4, 8, 3 * 262144 + 132), (8, 32, 5 * 262144 + 260)])
+def test_host_buffer_entry_point(cerar_mod, N, c, p):
+    """Host gradients in, host results out.  The larger shapes are cut into several
+    position slices (ragged last slice) that overlap copies and kernels."""
     import torch
-    N, c, p = 4, 8, 2048 + 4
     d = c * p
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(6))
     plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
     g = _inputs().gradients_numpy(N, d, "normal", seed=7)
     h_in = torch.from_numpy(g).pin_memory()
-    h_out = torch.empty(N, d, dtype=torch.float32).pin_memory()
+    h_out = torch.full((N, d), float("nan"), dtype=torch.float32).pin_memory()
     ws = torch.empty(N * (c + N) * p, dtype=torch.float32, device="cuda")
     s = torch.cuda.current_stream().cuda_stream
-    plan.allreduce_sim_host(h_in, d, h_out, d, ws, d, 1.0 / N, s)
-    torch.cuda.synchronize()
+    for _ in range(2):                                    # twice: buffers and events are reused
+        plan.allreduce_sim_host(h_in, d, h_out, d, ws, d, 1.0 / N, s)
+        torch.cuda.synchronize()
+    plan.device_status(s)
     ora = run_oracle(des.U, des.R, g, 1.0 / N)
     assert max(rel_l2(h_out[i].numpy(), ora["out"][i]) for i in range(N)) < 5e-6
-    assert plan.counters()["rounds_done"] == plan.L
+    cnt = plan.counters()
+    assert cnt["rounds_done"] == plan.L
+    assert cnt["bytes_forwarded_per_worker"] * c == cnt["bytes_gradient"] * (c + N - 2)
 
 
 def test_full_size_config2(cerar_mod):
