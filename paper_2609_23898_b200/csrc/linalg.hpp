@@ -72,84 +72,94 @@ bool inverse(const Mat<T>& Ain, Mat<T>& out) {
 
 // Householder QR of an m x n matrix (m >= n), applied to a right-hand side:
 // solves min ||A X - Bm||_F.  Also returns the n x n triangular factor if asked.
+// Works on transposed copies so that every column is contiguous in memory.
 inline bool lstsq(const MatD& Ain, const MatD& Bin, MatD& X, MatD* Rout = nullptr) {
     const int m = Ain.rows, n = Ain.cols, k = Bin.cols;
     if (m < n || Bin.rows != m) return false;
-    MatD A = Ain, B = Bin;
+    MatD At = transpose(Ain), Bt = transpose(Bin);      // At(j, i) = A(i, j)
     std::vector<double> v(m);
     for (int j = 0; j < n; ++j) {
+        double* aj = &At(j, 0);
         double nrm = 0;
-        for (int i = j; i < m; ++i) nrm += A(i, j) * A(i, j);
+        for (int i = j; i < m; ++i) nrm += aj[i] * aj[i];
         nrm = std::sqrt(nrm);
         if (nrm == 0.0) continue;
-        double alpha = (A(j, j) > 0) ? -nrm : nrm;
-        for (int i = j; i < m; ++i) v[i] = A(i, j);
+        const double alpha = (aj[j] > 0) ? -nrm : nrm;
+        for (int i = j; i < m; ++i) v[i] = aj[i];
         v[j] -= alpha;
         double vnorm2 = 0;
         for (int i = j; i < m; ++i) vnorm2 += v[i] * v[i];
         if (vnorm2 == 0.0) continue;
+        const double inv = 2.0 / vnorm2;
         for (int c2 = j; c2 < n; ++c2) {
+            double* ac = &At(c2, 0);
             double dot = 0;
-            for (int i = j; i < m; ++i) dot += v[i] * A(i, c2);
-            double f = 2.0 * dot / vnorm2;
-            for (int i = j; i < m; ++i) A(i, c2) -= f * v[i];
+            for (int i = j; i < m; ++i) dot += v[i] * ac[i];
+            const double f = dot * inv;
+            for (int i = j; i < m; ++i) ac[i] -= f * v[i];
         }
         for (int c2 = 0; c2 < k; ++c2) {
+            double* bc = &Bt(c2, 0);
             double dot = 0;
-            for (int i = j; i < m; ++i) dot += v[i] * B(i, c2);
-            double f = 2.0 * dot / vnorm2;
-            for (int i = j; i < m; ++i) B(i, c2) -= f * v[i];
+            for (int i = j; i < m; ++i) dot += v[i] * bc[i];
+            const double f = dot * inv;
+            for (int i = j; i < m; ++i) bc[i] -= f * v[i];
         }
     }
     X = MatD(n, k);
     for (int c2 = 0; c2 < k; ++c2)
         for (int i = n - 1; i >= 0; --i) {
-            double s = B(i, c2);
-            for (int j = i + 1; j < n; ++j) s -= A(i, j) * X(j, c2);
-            if (A(i, i) == 0.0 || !std::isfinite(A(i, i))) return false;
-            X(i, c2) = s / A(i, i);
+            double s = Bt(c2, i);
+            for (int j = i + 1; j < n; ++j) s -= At(j, i) * X(j, c2);
+            const double d = At(i, i);
+            if (d == 0.0 || !std::isfinite(d)) return false;
+            X(i, c2) = s / d;
         }
     if (Rout) {
         *Rout = MatD(n, n);
         for (int i = 0; i < n; ++i)
-            for (int j = i; j < n; ++j) (*Rout)(i, j) = A(i, j);
+            for (int j = i; j < n; ++j) (*Rout)(i, j) = At(j, i);
     }
     return true;
 }
 
 // One-sided Jacobi SVD of an m x n matrix (m >= n): A = Uo diag(s) V^T with
 // Uo m x n (orthonormal columns where s > 0) and V n x n.  s is returned in
-// descending order.
+// descending order.  Columns are kept contiguous (transposed working copies).
 inline void svd_jacobi(const MatD& Ain, MatD& Uo, std::vector<double>& s, MatD& V) {
     const int m = Ain.rows, n = Ain.cols;
-    MatD A = Ain;
-    V = MatD(n, n);
-    for (int i = 0; i < n; ++i) V(i, i) = 1.0;
+    MatD At = transpose(Ain);                           // row j = column j of A
+    MatD Vt(n, n);                                      // row j = column j of V
+    for (int i = 0; i < n; ++i) Vt(i, i) = 1.0;
     const double eps = std::numeric_limits<double>::epsilon();
     for (int sweep = 0; sweep < 60; ++sweep) {
         bool rotated = false;
         for (int p = 0; p < n - 1; ++p)
             for (int q = p + 1; q < n; ++q) {
+                double* ap = &At(p, 0);
+                double* aq = &At(q, 0);
                 double alpha = 0, beta = 0, gamma = 0;
                 for (int i = 0; i < m; ++i) {
-                    alpha += A(i, p) * A(i, p);
-                    beta += A(i, q) * A(i, q);
-                    gamma += A(i, p) * A(i, q);
+                    alpha += ap[i] * ap[i];
+                    beta += aq[i] * aq[i];
+                    gamma += ap[i] * aq[i];
                 }
                 if (gamma == 0.0 || std::fabs(gamma) <= eps * std::sqrt(alpha * beta)) continue;
                 rotated = true;
-                double zeta = (beta - alpha) / (2.0 * gamma);
-                double t = ((zeta >= 0) ? 1.0 : -1.0) / (std::fabs(zeta) + std::sqrt(1.0 + zeta * zeta));
-                double cs = 1.0 / std::sqrt(1.0 + t * t), sn = cs * t;
+                const double zeta = (beta - alpha) / (2.0 * gamma);
+                const double t = ((zeta >= 0) ? 1.0 : -1.0) / (std::fabs(zeta) + std::sqrt(1.0 + zeta * zeta));
+                const double cs = 1.0 / std::sqrt(1.0 + t * t), sn = cs * t;
                 for (int i = 0; i < m; ++i) {
-                    double ap = A(i, p), aq = A(i, q);
-                    A(i, p) = cs * ap - sn * aq;
-                    A(i, q) = sn * ap + cs * aq;
+                    const double x = ap[i], y = aq[i];
+                    ap[i] = cs * x - sn * y;
+                    aq[i] = sn * x + cs * y;
                 }
+                double* vp = &Vt(p, 0);
+                double* vq = &Vt(q, 0);
                 for (int i = 0; i < n; ++i) {
-                    double vp = V(i, p), vq = V(i, q);
-                    V(i, p) = cs * vp - sn * vq;
-                    V(i, q) = sn * vp + cs * vq;
+                    const double x = vp[i], y = vq[i];
+                    vp[i] = cs * x - sn * y;
+                    vq[i] = sn * x + cs * y;
                 }
             }
         if (!rotated) break;
@@ -157,22 +167,21 @@ inline void svd_jacobi(const MatD& Ain, MatD& Uo, std::vector<double>& s, MatD& 
     std::vector<double> nrm(n);
     for (int j = 0; j < n; ++j) {
         double t = 0;
-        for (int i = 0; i < m; ++i) t += A(i, j) * A(i, j);
+        for (int i = 0; i < m; ++i) t += At(j, i) * At(j, i);
         nrm[j] = std::sqrt(t);
     }
     std::vector<int> order(n);
     for (int j = 0; j < n; ++j) order[j] = j;
     std::sort(order.begin(), order.end(), [&](int a, int b) { return nrm[a] > nrm[b]; });
     Uo = MatD(m, n);
-    MatD Vs(n, n);
+    V = MatD(n, n);
     s.assign(n, 0.0);
     for (int jj = 0; jj < n; ++jj) {
-        int j = order[jj];
+        const int j = order[jj];
         s[jj] = nrm[j];
-        for (int i = 0; i < m; ++i) Uo(i, jj) = (nrm[j] > 0) ? A(i, j) / nrm[j] : 0.0;
-        for (int i = 0; i < n; ++i) Vs(i, jj) = V(i, j);
+        for (int i = 0; i < m; ++i) Uo(i, jj) = (nrm[j] > 0) ? At(j, i) / nrm[j] : 0.0;
+        for (int i = 0; i < n; ++i) V(i, jj) = Vt(j, i);
     }
-    V = Vs;
 }
 
 inline double kappa2(const MatD& A) {

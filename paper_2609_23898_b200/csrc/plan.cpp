@@ -245,23 +245,30 @@ static MatD m_matrix(const HostPlan& P, int i) {
     return M;
 }
 
-double phi_direct(const HostPlan& P) {
+template <class Acc>
+static double phi_blocks(const HostPlan& P) {
     const int N = P.N, c = P.c;
-    ld tot = 0;
+    Acc tot = 0;
+    std::vector<Acc> rowacc(c);
     for (int i = 0; i < N; ++i)
         for (int s = 0; s < N; ++s) {
             const std::vector<double>& U = P.U[((i - 1 - s) % N + N) % N];
             const std::vector<double>& R = P.R[i];
-            for (int a = 0; a < c; ++a)
-                for (int b = 0; b < c; ++b) {
-                    ld acc = 0;
-                    for (int t = 0; t < c; ++t) acc += (ld)U[(size_t)a * c + t] * (ld)R[(size_t)(s + t) * c + b];
-                    acc -= (a == b) ? (ld)1 : (ld)0;
-                    tot += acc * acc;
+            for (int a = 0; a < c; ++a) {
+                // row a of U W_s(R_i) - I, accumulated over the window rows (contiguous in R)
+                for (int b = 0; b < c; ++b) rowacc[b] = (a == b) ? (Acc)-1 : (Acc)0;
+                for (int t = 0; t < c; ++t) {
+                    const Acc u = (Acc)U[(size_t)a * c + t];
+                    const double* r = &R[(size_t)(s + t) * c];
+                    for (int b = 0; b < c; ++b) rowacc[b] += u * (Acc)r[b];
                 }
+                for (int b = 0; b < c; ++b) tot += rowacc[b] * rowacc[b];
+            }
         }
     return (double)tot;
 }
+
+double phi_direct(const HostPlan& P) { return phi_blocks<ld>(P); }
 
 double kappa_U_max(const HostPlan& P) {
     double k = 0;
@@ -351,13 +358,13 @@ int build_kappa(int N, int c, double kappa_max, const double* B, const double* h
     const double b0 = a0 * kappa_max / std::sqrt((double)N);
     project(P, a0, b0);
     ls_R(P);
-    double prev = phi_direct(P);
+    double prev = phi_blocks<double>(P);     // the projected iterates are well conditioned: fp64 is enough here
     int done = 0;
     for (int it = 0; it < iters; ++it) {
         ls_U(P);
         project(P, a0, b0);
         ls_R(P);
-        double cur = phi_direct(P);
+        double cur = phi_blocks<double>(P);
         done = it + 1;
         bool stop = std::fabs(prev - cur) <= tol * std::max(cur, 1e-300);
         prev = cur;
