@@ -75,3 +75,28 @@ def run_oracle(U, R, grads_np, scale=1.0):
 
 def rel_l2(a, b):
     return P.rel_l2(a, b)
+
+
+def sampled_parity(cfg, des, plan, grads, ws, out, scale, n_tiles=6, tile=512):
+    """Full-size check on sampled position tiles: positions are independent, so
+    the oracle runs the whole protocol on the sampled columns only."""
+    import torch
+    N, c, d = cfg["N"], cfg["c"], cfg["d"]
+    p, L = d // c, c + N - 2
+    rng = np.random.default_rng(123)
+    starts = sorted(set([0, max(0, p - tile)] + [int(x) for x in rng.integers(0, max(1, p - tile), n_tiles)]))
+    idx = np.concatenate([np.arange(s, min(s + tile, p)) for s in starts])
+    idx_t = torch.from_numpy(idx).to(grads.device)
+    g_sub = grads.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy().astype(np.float64)
+    ora = P.allreduce([x for x in g_sub], des.U, des.R, scale)
+    wsv = ws.view(N, c + N, p)
+    rows_t = torch.tensor(list(range(L)) + [L + 1], device=grads.device)
+    Y_dev = wsv[:, rows_t[:, None], idx_t[None, :]].cpu().numpy()         # (N, L+1, S)
+    Y_ora = np.stack([ora["Y"][i].T for i in range(N)])
+    out_dev = out.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy()
+    kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+    return {"positions": int(idx.size), "rel_l2_Y": P.rel_l2(Y_dev, Y_ora),
+            "rel_l2_out_max": max(P.rel_l2(out_dev[i], ora["out"][i]) for i in range(N)),
+            "kappa_M": kap, "kappa_times_2^-24": kap * 2.0 ** -24,
+            "rel_l2_oracle_vs_exact_mean": max(P.rel_l2(ora["out"][i], P.exact_sum(list(g_sub)) * scale)
+                                               for i in range(N))}

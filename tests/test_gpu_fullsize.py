@@ -14,8 +14,8 @@ U32 = 2.0 ** -24
 
 def _run(cfg_name, des, plan_factory, need_gb):
     import torch
-    import bench
     from paper_2609_23898_b200 import inputs
+    from tests._harness import sampled_parity
     free, _ = torch.cuda.mem_get_info()
     if free < need_gb * 1e9:
         pytest.skip(f"needs {need_gb} GB of device memory")
@@ -31,7 +31,7 @@ def _run(cfg_name, des, plan_factory, need_gb):
     plan.allreduce_sim(grads, d, out, d, ws, d, 1.0 / N, s)
     torch.cuda.synchronize()
     plan.device_status(s)
-    res = bench.sampled_parity(cfg, des, plan, grads, ws, out, 1.0 / N, n_tiles=8, tile=384)
+    res = sampled_parity(cfg, des, plan, grads, ws, out, 1.0 / N, n_tiles=8, tile=384)
     cnt = plan.counters()
     assert cnt["bytes_forwarded_per_worker"] * c == cnt["bytes_gradient"] * (c + N - 2)
     assert cnt["bytes_stored_per_worker"] * c == cnt["bytes_gradient"] * (c + N)
