@@ -274,6 +274,36 @@ def test_host_buffer_entry_point(cerar_mod, N, c, p):
     assert cnt["bytes_forwarded_per_worker"] * c == cnt["bytes_gradient"] * (c + N - 2)
 
 
+def test_pipeline_can_be_replayed_from_a_cuda_graph(cerar_mod):
+    """The data-path calls only enqueue kernels on the given stream, so a caller can
+    capture one aggregation in a CUDA graph (after a warm-up call with the same
+    shapes) and replay it: the replay gives bit-identical results."""
+    import torch
+    for (N, c, p) in [(4, 8, 8192), (8, 32, 4096 + 128)]:
+        d = c * p
+        des = Dz.custom_orthogonal(N, c, np.random.default_rng(8))
+        plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+        g = torch.from_numpy(_inputs().gradients_numpy(N, d, "normal", seed=9)).cuda()
+        ws = torch.empty(N * (c + N) * p, dtype=torch.float32, device="cuda")
+        out = torch.empty(N, d, dtype=torch.float32, device="cuda")
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            plan.allreduce_sim(g, d, out, d, ws, d, 1.0 / N, st.cuda_stream)      # warm-up
+            torch.cuda.synchronize()
+            ref = out.clone()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=st):
+                plan.allreduce_sim(g, d, out, d, ws, d, 1.0 / N, st.cuda_stream)
+            for _ in range(2):
+                out.zero_()
+                graph.replay()
+                torch.cuda.synchronize()
+                assert torch.equal(out, ref)
+        plan.device_status()
+        ora = run_oracle(des.U, des.R, g.cpu().numpy().reshape(N, d), 1.0 / N)
+        assert max(rel_l2(ref[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
+
+
 def test_full_size_config2(cerar_mod):
     """Second configuration at full size (N=4, c=16, d=2^24, eps=1e-3, N(0,1e-4)
     gradients) in the one-call form the benchmark times; stages checked in full
