@@ -107,6 +107,9 @@ cerar_status_t check_data_call(const cerar_plan* P, int64_t d, int64_t* p_out) {
     if (!P) return fail(CERAR_ERR_INVALID_ARG, "plan is NULL");
     if (!P->on_device) return fail(CERAR_ERR_CUDA, "plan has no device copies (no CUDA device, or host_only)");
     if (d <= 0 || d % P->host.c != 0) return fail(CERAR_ERR_SHAPE, "d must be a positive multiple of c");
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != P->device)
+        return fail(CERAR_ERR_CUDA, "the device the plan was created on must be current");
     *p_out = d / P->host.c;
     return CERAR_OK;
 }

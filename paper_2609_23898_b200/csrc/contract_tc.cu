@@ -407,11 +407,9 @@ template <int KC>
 cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a, const TcParams& tp,
                       size_t smem, dim3 grid, cudaStream_t s) {
     auto kern = contract_tc_kernel<KC>;
-    static thread_local size_t configured = 0;
-    if (smem > configured) {
+    {   // per device and cheap: set on every launch rather than cached
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured = smem;
     }
     kern<<<grid, NUM_THREADS, smem, s>>>(tin, tout, a, tp);
     return cudaGetLastError();

@@ -295,11 +295,9 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
     const size_t bar_bytes = ((2 * (size_t)a.stages * 8 + 127) / 128) * 128;
     const size_t coef_bytes = (((size_t)a.K * Jpad + 31) / 32) * 32 * 4;
     const size_t smem = bar_bytes + coef_bytes + (size_t)a.stages * a.KC * a.tile_p * 4;
-    static thread_local size_t configured = 0;
-    if (smem > configured) {
+    {   // per device and cheap: set on every launch rather than cached
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured = smem;
     }
     const int threads = 32 * (a.slabs * a.jgroups + 1);
     int occ = 0;
@@ -330,22 +328,25 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     if (mode == KERNEL_STAGED && !can_stage) return cudaErrorInvalidValue;
     bool use_staged = can_stage && mode != KERNEL_REF;
     if (use_staged) {
-        // 8 outputs x 8 positions per thread measured best on B200 (more resident warps than 16 x 8)
-        int JT = g_tune_jt ? g_tune_jt : ((a.J % 8 == 0) ? 8 : 4);
+        // register tile: 8 outputs x 8 positions per thread where J allows it (more resident
+        // warps than 16 x 8), 4 x 8 otherwise; as many position slabs as the warp budget
+        // allows; stages of about 64 KB (values measured best on B200 for c = 8..24)
+        int JT = g_tune_jt ? g_tune_jt : ((a.J % 8 == 0 && a.J >= 16) ? 8 : 4);
         const int PV = 2;
         a.jgroups = (a.J + JT - 1) / JT;
         const int maxw = (JT == 16) ? 8 : 16;
         if (a.jgroups > maxw) {
             use_staged = false;
         } else {
-            int slabs = g_tune_slabs ? g_tune_slabs : (8 + a.jgroups / 2) / a.jgroups;
+            int slabs = g_tune_slabs ? g_tune_slabs : maxw / a.jgroups;
+            if (slabs > 8) slabs = 8;
             if (slabs < 1) slabs = 1;
             while (slabs > 1 && slabs * a.jgroups > maxw) --slabs;
             a.slabs = slabs;
             a.tile_p = slabs * PV * 128;
             a.KC = g_tune_kc ? g_tune_kc : 16;
-            if (!g_tune_kc) {                      // keep a stage near 48 KB whatever the tile width
-                const int fit = (48 * 1024) / (a.tile_p * 4);
+            if (!g_tune_kc) {
+                const int fit = (64 * 1024) / (a.tile_p * 4);
                 if (a.KC > fit) a.KC = fit < 2 ? 2 : fit;
             }
             if (a.KC > a.K) a.KC = a.K;
