@@ -325,3 +325,38 @@ def test_full_size_config2(cerar_mod):
     assert worst < 4 * kap * U32
     res1 = run_library(plan, g, 1.0 / N, stepwise=False)
     np.testing.assert_array_equal(res1["out"], res["out"])       # same kernels, same order: bit-identical
+
+
+@pytest.mark.parametrize("N,c,p", [(2, 2, 1), (2, 3, 5), (2, 16, 4), (3, 3, 4), (7, 7, 12), (4, 130, 8), (2, 512, 4),
+                                   (16, 16, 4), (8, 32, 4), (8, 32, 124), (4, 64, 132), (12, 36, 260)])
+def test_degenerate_and_extreme_shapes(cerar_mod, N, c, p):
+    """Smallest ring (N = 2, where L = c), c = N (the classic case), a single position,
+    fewer positions than one tile or one vector, the largest c the library accepts
+    (512, plain kernel), c just beyond the tensor-core range, odd N."""
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(N * 1000 + c))
+    g = _inputs().gradients_numpy(N, c * p, "normal", seed=11)
+    plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+    ora = run_oracle(des.U, des.R, g, 1.0 / N)
+    res = run_library(plan, g, 1.0 / N)
+    _check_stages(res, ora, OUT_TOL, N)
+    res = run_library(plan, g, 1.0 / N, inplace=True, stepwise=False)
+    assert max(rel_l2(res["out"][i], ora["out"][i]) for i in range(N)) < 1e-5
+    cnt = res["counters"]
+    assert cnt["rounds_done"] == c + N - 2
+    assert cnt["bytes_forwarded_per_worker"] == 4 * p * (c + N - 2)
+
+
+def test_classic_ring_allreduce_is_exact_on_the_device(cerar_mod):
+    """c = N with D = I (eps = 0): the protocol is the basic ring all-reduce with
+    2(N-1) rounds and recovers the exact sum (up to fp32 roundoff)."""
+    N = c = 4
+    p = 4096 + 4
+    B = _inputs().base_matrix(N, c, 5)
+    plan = cerar_mod.Plan.create(N, c, cerar_mod.EPSILON, 0.0, B=B)
+    assert plan.L == 2 * (N - 1)
+    g = _inputs().gradients_numpy(N, c * p, "normal", seed=12)
+    res = run_library(plan, g, 1.0)
+    exact = P.exact_sum(g)
+    kap = plan.info()["kappa_M_max"]
+    for i in range(N):
+        assert rel_l2(res["out"][i], exact) < 20 * kap * U32
