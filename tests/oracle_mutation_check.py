@@ -26,18 +26,23 @@ muts=[
  ('oracle/designs.py','(i - 1 - k) % N, c) for i in range(N)], axis=1)','(i - k) % N, c) for i in range(N)], axis=1)'),
  ('oracle/designs.py','b0 = a0 * kappa_max / np.sqrt(N)','b0 = a0 * kappa_max'),
 ]
-survived=[]
-for idx,(f,old,new) in enumerate(muts):
-    path=os.path.join(ROOT,f); src=open(path).read()
-    if old not in src:
-        print(idx,'PATTERN NOT FOUND',f,old[:40]); continue
-    open(path,'w').write(src.replace(old,new,1))
-    try:
-        r=subprocess.run([sys.executable,'-m','pytest','tests/test_oracle_protocol.py','tests/test_oracle_designs.py','-x','-q','-p','no:cacheprovider'],cwd=ROOT,capture_output=True,text=True,timeout=600)
-        failed = r.returncode!=0
-        last=[l for l in r.stdout.splitlines() if 'FAILED' in l or 'passed' in l or 'failed' in l or 'Error' in l][-2:]
-        print(idx,'KILLED' if failed else 'SURVIVED',f,'|',old[:50].replace('\n',' '),'|',last[:1])
-        if not failed: survived.append(idx)
-    finally:
-        open(path,'w').write(src)
-print('survived:',survived)
+def main():
+    survived=[]
+    for idx,(f,old,new) in enumerate(muts):
+        path=os.path.join(ROOT,f); src=open(path).read()
+        if old not in src:
+            print(idx,'PATTERN NOT FOUND',f,old[:40]); continue
+        open(path,'w').write(src.replace(old,new,1))
+        try:
+            r=subprocess.run([sys.executable,'-m','pytest','tests/test_oracle_protocol.py','tests/test_oracle_designs.py','-x','-q','-p','no:cacheprovider'],cwd=ROOT,capture_output=True,text=True,timeout=600)
+            failed = r.returncode!=0
+            last=[l for l in r.stdout.splitlines() if 'FAILED' in l or 'passed' in l or 'failed' in l or 'Error' in l][-2:]
+            print(idx,'KILLED' if failed else 'SURVIVED',f,'|',old[:50].replace('\n',' '),'|',last[:1])
+            if not failed: survived.append(idx)
+        finally:
+            open(path,'w').write(src)
+    print('survived:',survived)
+
+
+if __name__ == "__main__":
+    main()
