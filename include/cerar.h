@@ -184,6 +184,22 @@ cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* plan, const float* h_grads
                                         int64_t h_out_stride, float* ws, int64_t d,
                                         float scale, cerar_stream_t stream);
 
+/* Variant with the ring on chip (the paper's protocol, a different memory system:
+ * not the in-HBM pipeline above and reported separately from it).  One launch
+ * carries every position through encode (Sec. II), the L rounds of Algorithm 1
+ * and decode (Sec. II-A) with the (c+N) slots of all workers in shared memory,
+ * so HBM sees each gradient element once and each result element once and no
+ * workspace is needed; the hand-offs between workers happen in shared memory.
+ * Same arithmetic and order of operations as the FMA kernels (fp32).  Only for
+ * c <= 32 (a multiple of 4, or 5 or 6) and N (c+N) small enough for shared
+ * memory: cerar_fused_supported says so, otherwise CERAR_ERR_INVALID_ARG.
+ * grads / out as in cerar_allreduce_sim (device, no aliasing).  The counters
+ * afterwards describe the L logical rounds. */
+cerar_status_t cerar_allreduce_fused(cerar_plan_t* plan, const float* grads, int64_t grads_stride,
+                                     float* out, int64_t out_stride, int64_t d, float scale,
+                                     cerar_stream_t stream);
+int            cerar_fused_supported(const cerar_plan_t* plan);
+
 /* The same pipeline as cerar_allreduce_sim for callers that cannot provide a
  * workspace because they cannot allocate device memory at this point: for
  * instance a host program whose framework has already claimed all free memory

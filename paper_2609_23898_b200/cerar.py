@@ -76,6 +76,8 @@ lib.cerar_decode.argtypes = [_vp, _f32p, _f32p, _i64, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim_host.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim_static.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _i64, C.c_float, _vp]
+lib.cerar_allreduce_fused.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _i64, C.c_float, _vp]
+lib.cerar_fused_supported.argtypes = [_vp]
 lib.cerar_get_counters.argtypes = [_vp, C.POINTER(Counters)]
 lib.cerar_launch_count.argtypes = [_vp]
 lib.cerar_launch_count.restype = C.c_uint64
@@ -199,6 +201,14 @@ class Plan:
     def allreduce_sim(self, grads, grads_stride, out, out_stride, ws, d, scale=1.0, stream=0):
         _check(lib.cerar_allreduce_sim(self._h, _ptr(grads), grads_stride, _ptr(out), out_stride,
                                        _ptr(ws), d, scale, stream))
+
+    def allreduce_fused(self, grads, grads_stride, out, out_stride, d, scale=1.0, stream=0):
+        """cerar_allreduce_fused: whole protocol in one launch, slots in shared memory (small N (c+N))."""
+        _check(lib.cerar_allreduce_fused(self._h, _ptr(grads), grads_stride, _ptr(out), out_stride,
+                                         d, scale, stream))
+
+    def fused_supported(self) -> bool:
+        return bool(lib.cerar_fused_supported(self._h))
 
     def allreduce_sim_static(self, grads, grads_stride, out, out_stride, d, scale=1.0, stream=0):
         """cerar_allreduce_sim_static: same pipeline, workspace built into the library (<= 64 MiB)."""

@@ -380,6 +380,30 @@ cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* P, const float* h_grads, i
     return CERAR_OK;
 }
 
+cerar_status_t cerar_allreduce_fused(cerar_plan_t* P, const float* grads, int64_t grads_stride, float* out,
+                                     int64_t out_stride, int64_t d, float scale, cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!grads || !out) return fail(CERAR_ERR_INVALID_ARG, "grads or out is NULL");
+    if (grads_stride < d || out_stride < d) return fail(CERAR_ERR_SHAPE, "stride < d");
+    const int N = P->host.N, c = P->host.c;
+    if (!cerar::fused_supported(N, c))
+        return fail(CERAR_ERR_INVALID_ARG, "the on-chip path needs c <= 32 (a multiple of 4, or 5, 6) and N (c+N) small "
+                                           "enough for shared memory; use cerar_allreduce_sim");
+    cudaError_t e = cerar::launch_fused(grads, grads_stride, out, out_stride, P->d_U, P->d_R, N, c, p, scale,
+                                        P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "fused launch");
+    // the L rounds ran (on chip): the logical message bytes are the same
+    P->encoded = 0; P->rounds_done = P->host.L; P->cur_d = d;
+    P->bytes_forwarded = (uint64_t)4 * (uint64_t)p * (uint64_t)P->host.L;
+    return CERAR_OK;
+}
+
+int cerar_fused_supported(const cerar_plan_t* P) {
+    return (P && cerar::fused_supported(P->host.N, P->host.c)) ? 1 : 0;
+}
+
 cerar_status_t cerar_get_counters(const cerar_plan_t* P, cerar_counters_t* out) {
     if (!P || !out) return fail(CERAR_ERR_INVALID_ARG, "bad argument");
     const int64_t p = P->cur_d / (P->host.c ? P->host.c : 1);

@@ -28,6 +28,9 @@ def main():
     ap.add_argument("--quick", action="store_true", help="d in {2^20, 2^26} only")
     ap.add_argument("--out", default="")
     ap.add_argument("--eps", type=float, default=1e-3)
+    ap.add_argument("--fused", action="store_true",
+                    help="time cerar_allreduce_fused (ring on chip, out of place) next to the in-HBM pipeline "
+                         "for the (N, c) it supports")
     args = ap.parse_args()
 
     import torch
@@ -42,6 +45,8 @@ def main():
     stream = torch.cuda.current_stream().cuda_stream
     exps = [20, 26] if args.quick else [18, 20, 22, 24, 26, 28, 30]
     rows = []
+    if args.fused:
+        return fused_table(args, exps, peak, free, stream)
     print("| N | c | d | state MB | ms / aggregation | GB/s | frac of measured HBM | note |")
     print("|---|---|---|---|---|---|---|---|")
     for N in (4, 8, 16):
@@ -99,6 +104,57 @@ def main():
     if args.out:
         with open(args.out, "w") as f:
             json.dump(rows, f, indent=1)
+
+
+def fused_table(args, exps, peak, free, stream):
+    """Seconds per aggregation of the on-chip variant against the in-HBM pipeline (both out of place)."""
+    import torch
+    from . import cerar, inputs
+    print("| N | c | d | in-HBM pipeline ms | on-chip ms | speed-up | on-chip DRAM GB/s (8 N d bytes) |")
+    print("|---|---|---|---|---|---|---|")
+    rows = []
+    for N in (4, 8, 16):
+        for mult in (1, 2, 4, 8):
+            c = N * mult
+            B = inputs.base_matrix(N, c, 0)
+            try:
+                plan = cerar.Plan.create(N, c, cerar.EPSILON, args.eps, B=B)
+            except cerar.CerarError:
+                continue
+            if not plan.fused_supported():
+                plan.destroy()
+                continue
+            for e in exps:
+                d = 1 << e
+                p = d // c
+                need = plan.workspace_bytes(d) + 8 * N * d
+                if d % c or need > free - (2 << 30):
+                    continue
+                g = torch.empty(N * d, dtype=torch.float32, device="cuda").normal_()
+                out = torch.empty(N * d, dtype=torch.float32, device="cuda")
+                ws = torch.empty(plan.workspace_bytes(d) // 4, dtype=torch.float32, device="cuda")
+
+                def med(f):
+                    ts = []
+                    for rep in range(8):
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record(); f(); e1.record(); torch.cuda.synchronize()
+                        if rep >= 3:
+                            ts.append(e0.elapsed_time(e1))
+                    return float(np.median(ts))
+                t_hbm = med(lambda: plan.allreduce_sim(g, d, out, d, ws, d, 1.0 / N, stream))
+                t_chip = med(lambda: plan.allreduce_fused(g, d, out, d, d, 1.0 / N, stream))
+                plan.device_status(stream)
+                rows.append(dict(N=N, c=c, d=d, ms_hbm=t_hbm, ms_chip=t_chip))
+                print(f"| {N} | {c} | 2^{e} | {t_hbm:.3f} | {t_chip:.3f} | {t_hbm / t_chip:.2f} | {8 * N * d / t_chip / 1e6:.0f} |",
+                      flush=True)
+                del g, out, ws
+                torch.cuda.empty_cache()
+            plan.destroy()
+    if args.out:
+        with open(args.out, "w") as f:
+            json.dump(rows, f, indent=1)
+    return 0
 
 
 if __name__ == "__main__":
