@@ -360,3 +360,21 @@ def test_classic_ring_allreduce_is_exact_on_the_device(cerar_mod):
     kap = plan.info()["kappa_M_max"]
     for i in range(N):
         assert rel_l2(res["out"][i], exact) < 20 * kap * U32
+
+
+def test_randomised_shapes(cerar_mod):
+    """Seeded random (N, c, p) over all three contraction kernels and both round kernels."""
+    rng = np.random.default_rng(77)
+    for trial in range(24):
+        N = int(rng.integers(2, 13))
+        c = int(rng.choice([N, N + 1, N + 3, 2 * N, 16, 24, 32, 40, 64, 96]))
+        c = max(c, N)
+        p = int(rng.choice([1, 3, 4, 60, 128, 131, 516, 1000, 2052, 4104]))
+        des = Dz.custom_orthogonal(N, c, np.random.default_rng(trial))
+        g = _inputs().gradients_numpy(N, c * p, "normal", seed=100 + trial)
+        plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+        scale = float(rng.choice([1.0, 1.0 / N, 0.37]))
+        ora = run_oracle(des.U, des.R, g, scale)
+        res = run_library(plan, g, scale, inplace=bool(trial % 2), stepwise=bool(trial % 3))
+        worst = max(rel_l2(res["out"][i], ora["out"][i]) for i in range(N))
+        assert worst < 1e-5, (N, c, p, worst)

@@ -239,3 +239,28 @@ def test_error_identity_and_bound():
         lhs = np.linalg.norm(res["out"][i] - P.exact_sum(g))
         assert lhs == pytest.approx(np.linalg.norm(Gi @ E, "fro"), rel=1e-6, abs=1e-9)
         assert lhs <= np.linalg.norm(Gi, 2) * np.linalg.norm(E, "fro") * (1 + 1e-9) + 1e-9
+
+
+def test_randomised_shapes_composed_map_and_prop1():
+    """Seeded random (N, c, p): rounds == G^(i) M_i(U) for random encoders, the decoded
+    output is the one linear map G^(i) (M_i R_i), and for an epsilon design worker 0
+    recovers the exact sum (Prop. 1 with i = 0)."""
+    rng = np.random.default_rng(2024)
+    for _ in range(25):
+        N = int(rng.integers(2, 7))
+        c = int(rng.integers(N, N + 9))
+        p = int(rng.integers(1, 6))
+        L = c + N - 2
+        U = [rng.standard_normal((c, c)) for _ in range(N)]
+        R = [rng.standard_normal((L + 1, c)) for _ in range(N)]
+        g = [rng.standard_normal(c * p) for _ in range(N)]
+        G = [P.chunk_matrix(x, c) for x in g]
+        res = P.allreduce(g, U, R, 0.5)
+        for i in range(N):
+            Gi = P.stacked_gradients(G, i)
+            np.testing.assert_allclose(res["Y"][i], Gi @ P.m_matrix(U, i), atol=1e-9)
+            np.testing.assert_allclose(res["out"][i], P.unchunk(0.5 * Gi @ (P.m_matrix(U, i) @ R[i])), atol=1e-9)
+        assert res["values_sent_per_worker"] == [L * p] * N
+        des = Dz.epsilon(N, c, 0.03, rng.standard_normal((N, c)))
+        out = P.allreduce(g, des.U, des.R)["out"]
+        assert P.rel_l2(out[0], P.exact_sum(g)) < 1e-7
