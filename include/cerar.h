@@ -239,6 +239,13 @@ uint64_t       cerar_launch_count(const cerar_plan_t* plan);
  * results of that call are then invalid); CERAR_OK otherwise. */
 cerar_status_t cerar_device_status(cerar_plan_t* plan, cerar_stream_t stream);
 
+/* Failure-path self test: launches a one-warp kernel whose bounded wait cannot be
+ * satisfied (nothing ever arrives on its barrier), so that it gives up after
+ * limit_ms (1..1000) and flags the status word like the pipelined kernels do when a
+ * wait runs out; the next cerar_device_status then returns CERAR_ERR_TIMEOUT and
+ * clears the flag.  The device context stays usable. */
+cerar_status_t cerar_selftest_wait_timeout(cerar_plan_t* plan, int limit_ms, cerar_stream_t stream);
+
 /* Kernel selection for encode/decode: 0 = automatic, 1 = plain per-position
  * kernel, 2 = staged FMA kernel, 3 = tensor-core (3 x TF32) kernel; a forced
  * kernel that cannot take the shape makes the call fail instead of falling

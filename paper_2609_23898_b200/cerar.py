@@ -83,6 +83,7 @@ lib.cerar_launch_count.argtypes = [_vp]
 lib.cerar_launch_count.restype = C.c_uint64
 lib.cerar_set_kernel_mode.argtypes = [_vp, C.c_int]
 lib.cerar_device_status.argtypes = [_vp, _vp]
+lib.cerar_selftest_wait_timeout.argtypes = [_vp, C.c_int, _vp]
 lib.cerar_set_tuning.argtypes = [C.c_char_p, C.c_int]
 lib.cerar_status_string.argtypes = [C.c_int]
 lib.cerar_status_string.restype = C.c_char_p
@@ -187,6 +188,9 @@ class Plan:
 
     def device_status(self, stream=0):
         _check(lib.cerar_device_status(self._h, stream))
+
+    def selftest_wait_timeout(self, limit_ms=20, stream=0):
+        _check(lib.cerar_selftest_wait_timeout(self._h, limit_ms, stream))
 
     # ---- data path (device pointers; stream = a cudaStream_t handle as int)
     def encode(self, grads, grads_stride, ws, d, stream=0):

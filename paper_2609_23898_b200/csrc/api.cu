@@ -439,6 +439,17 @@ cerar_status_t cerar_device_status(cerar_plan_t* P, cerar_stream_t stream) {
     return CERAR_OK;
 }
 
+cerar_status_t cerar_selftest_wait_timeout(cerar_plan_t* P, int limit_ms, cerar_stream_t stream) {
+    if (!P) return fail(CERAR_ERR_INVALID_ARG, "plan is NULL");
+    if (!P->on_device) return fail(CERAR_ERR_CUDA, "plan has no device copies");
+    if (limit_ms < 1 || limit_ms > 1000) return fail(CERAR_ERR_INVALID_ARG, "limit_ms must be in 1..1000");
+    cudaError_t e = cerar::launch_wait_timeout_selftest(P->d_status, (unsigned long long)limit_ms * 1000000ull,
+                                                        (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e, "selftest launch");
+    ++P->launches;
+    return CERAR_OK;
+}
+
 int cerar_set_tuning(const char* name, int value) {
     if (!name) return -1;
     std::string n(name);

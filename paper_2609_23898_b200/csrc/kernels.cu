@@ -8,60 +8,14 @@
 //  round_kernel            one ring round for all workers: fused cancel + add +
 //                          hand-off store into the neighbour's landing slot
 #include "kernels.cuh"
-
-#include <cstdio>
+#include "ptx.cuh"
 
 namespace cerar {
 namespace {
 
 constexpr int REF_MAX_J = 512;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a bounded wait gives up after 2 s
 
-// ------------------------------------------------------------------ PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        " .reg .pred p;\n"
-        " mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        " selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Wait for a phase of an mbarrier, but never forever: returns false after
-// WAIT_LIMIT_NS so that the caller can flag the error and leave.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
-    }
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
+using namespace ptx;
 
 // ------------------------------------------------------------------ reference contraction
 __global__ void contract_ref_kernel(const ContractArgs a) {
@@ -116,7 +70,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
             mbar_init(full0 + 8u * s, 1);
             mbar_init(empty0 + 8u * s, CW);
         }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
     }
     {
         const float* cf = a.coef + (size_t)w * a.K * a.J;
@@ -286,6 +240,17 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
     }
 }
 
+// Nothing ever arrives on this barrier: the bounded wait runs out after limit_ns and the
+// kernel reports it through the status word, exactly as the pipelined kernels would.
+__global__ void wait_timeout_selftest_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        mbar_init_fence();
+        if (!mbar_wait_bounded(smem_u32(&bar), 0, limit_ns)) atomicExch(status, 3);
+    }
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 template <int PV, int JT, int MAXW>
@@ -378,6 +343,11 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
+}
+
+cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(status, limit_ns);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches) {

@@ -43,6 +43,8 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
 bool tc_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
+// A kernel whose bounded wait is made to run out (nothing arrives on its barrier).
+cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);
 // Whole protocol in one launch with the slots in shared memory (small N (c+N) only).
 bool fused_supported(int N, int c);
 cudaError_t launch_fused(const float* grads, int64_t grads_stride, float* out, int64_t out_stride, const float* U,

@@ -378,3 +378,28 @@ def test_randomised_shapes(cerar_mod):
         res = run_library(plan, g, scale, inplace=bool(trial % 2), stepwise=bool(trial % 3))
         worst = max(rel_l2(res["out"][i], ora["out"][i]) for i in range(N))
         assert worst < 1e-5, (N, c, p, worst)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives(cerar_mod):
+    """Failure path without a fault: a kernel whose bounded wait cannot be satisfied gives
+    up after its limit, the host reads CERAR_ERR_TIMEOUT once, and the library keeps
+    working afterwards."""
+    import time
+    import torch
+    N, c, p = 4, 8, 1024
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(4))
+    plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+    plan.device_status()                                     # clean to start with
+    t0 = time.time()
+    plan.selftest_wait_timeout(25)
+    with pytest.raises(cerar_mod.CerarError) as e:
+        plan.device_status()
+    assert e.value.status == 8                                # CERAR_ERR_TIMEOUT
+    assert 0.02 < time.time() - t0 < 5.0
+    plan.device_status()                                     # the flag was cleared
+    g = _inputs().gradients_numpy(N, c * p, "normal", seed=15)
+    ora = run_oracle(des.U, des.R, g, 1.0)
+    res = run_library(plan, g, 1.0)
+    _check_stages(res, ora, OUT_TOL, N)
+    with pytest.raises(cerar_mod.CerarError):
+        plan.selftest_wait_timeout(0)
