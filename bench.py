@@ -305,6 +305,7 @@ def main():
     rnd_ms = [float(np.mean([ev[s][k].elapsed_time(ev[s][k + 1]) for s in range(K)])) for k in range(1, L + 1)]
     ms_per_step = max_over_ranks(total_ms, world, dev) / K
     value = whole_job_value(ab["total"], world, ms_per_step)
+    step_ms = [ev[s][0].elapsed_time(ev[s][L + 2]) for s in range(K)]      # this rank's steps, one by one
 
     peak, peak_kind = load_peaks()
     rounds_bytes = sum(round_bytes(N, c, p, k) for k in range(1, L + 1))
@@ -330,6 +331,8 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "seconds_per_aggregation": ms_per_step * 1e-3,
+            "step_ms": {"median": float(np.median(step_ms)), "min": float(np.min(step_ms)),
+                        "p95": float(np.percentile(step_ms, 95)), "max": float(np.max(step_ms))},
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {"workload": workload_name(args.workload, cfg), "N": N, "c": c, "L": L, "d": d,
