@@ -13,7 +13,6 @@
 #include "plan.hpp"
 
 namespace cerar {
-extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages;
 }
 
 struct cerar_plan {
@@ -459,6 +458,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "slabs") cerar::g_tune_slabs = value;
     else if (n == "tc_kc") cerar::g_tune_tc_kc = value;
     else if (n == "tc_stages") cerar::g_tune_tc_stages = value;
+    else if (n == "tc_variant") cerar::g_tune_tc_variant = value;
     else return -1;
     return 0;
 }

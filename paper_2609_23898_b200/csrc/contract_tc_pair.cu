@@ -1,0 +1,379 @@
+// Tensor-core contraction for encode / decode, 32 <= c <= 64: 256 positions per tile.
+//
+//   out[j][q] = scale * sum_k coef[k][j] * in[k][q],   j < J (= c),  k < K rows,  q < p
+//
+// Same arithmetic as contract_tc_kernel (3 x TF32 on tcgen05, fp32 accumulation in
+// tensor memory), different geometry: global memory is read and written in rows of
+// 1 KB (256 positions) instead of 512 B, which HBM serves measurably better, and the
+// SIMT roles have two warps per TMEM lane quadrant.  A tile of 256 positions is two
+// UMMA tiles of M = 128 ("halves"); half h belongs to MMA issuer h for the whole run.
+//
+// One CTA of 19 warps per SM.  The tiles of all workers form one list that is cut
+// into one contiguous range per CTA, so every SM is busy; a range that crosses a
+// worker boundary is processed in two segments (the coefficients are per worker).
+//   warp 0        producer: one TMA load per chunk ([KC rows] x [256 positions])
+//   warps 11-18   splitter: thread = position (of both halves); the two warps of a
+//                 lane quadrant take one half of the chunk's rows each; values are split
+//                 into tf32 hi | lo and written to tensor memory (tcgen05.st), where
+//                 they are the A operand of their half
+//   warps 1, 2    MMA issuers (one lane each) for half 0 / 1: tcgen05.mma kind::tf32,
+//                 A from TMEM, B = the coefficients (hi and lo copies) in shared memory,
+//                 M=128, N=Npad, K=8; two accumulators each, so that the epilogue of one
+//                 tile overlaps the products of the next; warp 1 owns the TMEM allocation
+//   warps 3-10    epilogue: tcgen05.ld (16 of every 32 output rows per warp), scale,
+//                 transpose through a shared-memory tile, one TMA store per 32 output
+//                 rows x 256 positions
+// Every wait is bounded; a wait that runs out sets the status word and the CTA leaves
+// through the common exit, where tensor memory is freed.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "kernels.cuh"
+#include "tc_common.cuh"
+
+namespace cerar {
+namespace {
+
+using namespace tc;
+
+constexpr int HALF_M = 128;              // UMMA M
+constexpr int TILE_W = 2 * HALF_M;       // positions per tile
+constexpr int OUT_ROWS = 32;             // output rows per TMA store
+constexpr int NUM_WARPS = 19;
+constexpr int NUM_THREADS = 32 * NUM_WARPS;
+constexpr int WARP_EPI0 = 3, WARP_SPLIT0 = 11;
+
+struct PairParams {
+    int K_rows;        // physical input rows that carry data; rows beyond read as zero (TMA fill)
+    int K_pad;         // K_rows rounded up to a multiple of KC
+    int stages;        // shared-memory stages of raw chunks
+    int NAh;           // A (hi|lo) chunk buffers per half in tensor memory
+    int Npad;          // J rounded up to 32
+    int tmem_cols;     // power of two >= 4*Npad + 2*NAh*2*KC
+    int64_t tiles_per_worker;
+    int64_t total_tiles;
+};
+
+// shared memory (1024-aligned): B_hi | B_lo | raw stages | 2 output tiles | barriers | tmem slot
+template <int KC>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
+                        const __grid_constant__ ContractArgs a, const __grid_constant__ PairParams tp) {
+    extern __shared__ unsigned char smem_dyn[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int stages = tp.stages, Npad = tp.Npad, K_pad = tp.K_pad;
+    const uint32_t NAh = (uint32_t)tp.NAh;
+    const int nkc = K_pad / KC;
+    const int nblk = Npad / 32;
+    static_assert(KC % 8 == 0, "a chunk is a whole number of k-steps");
+    constexpr int KG = KC / 2;           // rows of a chunk per splitter warp of a quadrant (a multiple of 4)
+
+    const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    unsigned char* smem_al = smem_dyn + (smem_base - smem_u32(smem_dyn));
+    const uint32_t b_bytes = (uint32_t)K_pad * Npad * 4u;            // one of B_hi / B_lo
+    constexpr uint32_t chunk_bytes = (uint32_t)KC * TILE_W * 4u;
+    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * TILE_W * 4u;
+    const uint32_t bhi_u32 = smem_base, blo_u32 = smem_base + b_bytes;
+    const uint32_t raw_u32 = smem_base + 2u * b_bytes;
+    const uint32_t out_u32 = raw_u32 + (uint32_t)stages * chunk_bytes;
+    const uint32_t bar_u32 = out_u32 + 2u * out_bytes;
+    const uint32_t raw_full = bar_u32, raw_empty = raw_full + 8u * stages;
+    const uint32_t a_full = raw_empty + 8u * stages;                 // [half][NAh]
+    const uint32_t a_empty = a_full + 16u * NAh;
+    const uint32_t acc_full = a_empty + 16u * NAh;                   // [half][2]
+    const uint32_t acc_empty = acc_full + 32u;
+    const uint32_t out_full = acc_empty + 32u, out_free = out_full + 16u;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_al + (out_free + 16u - smem_base));
+    const float* raw_s = reinterpret_cast<const float*>(smem_al + (raw_u32 - smem_base));
+    float* out_s = reinterpret_cast<float*>(smem_al + (out_u32 - smem_base));
+
+    // ---------------- set-up
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) { mbar_init(raw_full + 8u * s, 1); mbar_init(raw_empty + 8u * s, 8); }
+        for (uint32_t b = 0; b < 2u * NAh; ++b) { mbar_init(a_full + 8u * b, 8); mbar_init(a_empty + 8u * b, 1); }
+        for (int b = 0; b < 4; ++b) { mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(out_full + 8u * b, 8); mbar_init(out_free + 8u * b, 1); }
+        mbar_init_fence();
+    }
+    if (warp == 1) tc_alloc(smem_u32(tmem_slot), (uint32_t)tp.tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t a_col0 = 4u * (uint32_t)Npad;            // A buffers start after the four accumulators
+
+    // this CTA's contiguous range of the tile list (worker-major), cut at worker boundaries
+    const int64_t T = tp.tiles_per_worker;
+    const int64_t g_begin = tp.total_tiles * blockIdx.x / gridDim.x;
+    const int64_t g_end = tp.total_tiles * (blockIdx.x + 1) / gridDim.x;
+    const int w_first = (int)(g_begin / T);
+    const int w_last = g_end > g_begin ? (int)((g_end - 1) / T) : w_first - 1;
+
+    bool failed = false;
+    uint32_t it = 0, tc = 0, oc = 0;      // chunks, tiles and output blocks this CTA has gone through (all roles count alike)
+
+    for (int w = w_first; w <= w_last; ++w) {
+        const int64_t t_begin = (w == w_first) ? g_begin - (int64_t)w * T : 0;
+        const int64_t t_end = (w == w_last) ? g_end - (int64_t)w * T : T;
+        {
+            // coefficients of this worker, split into tf32 hi / lo, in the only layout the tensor
+            // core takes for an MN-major 32-bit operand (128-byte swizzle, 32-byte atoms):
+            // block nb (32 outputs) | row k (128 B) | 32-byte chunk ^ (k & 3)
+            const float* cf = a.coef + (size_t)w * a.K * a.J;
+            uint32_t* bhi = reinterpret_cast<uint32_t*>(smem_al);
+            uint32_t* blo = reinterpret_cast<uint32_t*>(smem_al + b_bytes);
+            for (int idx = threadIdx.x; idx < K_pad * Npad; idx += blockDim.x) {
+                const int k = idx / Npad, j = idx - k * Npad;
+                // physical input row k -> coefficient row (the row at skip_row is not part of Y: zero)
+                int src = -1;
+                if (k < a.skip_row) src = k; else if (k > a.skip_row) src = k - 1;
+                float v = 0.f;
+                if (src >= 0 && src < a.K && j < a.J) v = cf[(size_t)src * a.J + j];
+                const uint32_t hi = tf32_bits(v);
+                const uint32_t lo = tf32_bits(v - __uint_as_float(hi));
+                const int nb = j >> 5, jj = j & 31;
+                const int off = nb * (K_pad * 32) + k * 32 + ((((jj >> 3) ^ (k & 3)) << 3) | (jj & 7));
+                bhi[off] = hi;
+                blo[off] = lo;
+            }
+            fence_proxy_async_smem();
+        }
+        __syncthreads();
+
+        if (failed) {
+            // a wait of this warp ran out in an earlier segment: only keep the CTA barriers company
+        } else if (warp == 0) {
+            // ================= producer
+            if (lane == 0) {
+                for (int64_t t = t_begin; t < t_end && !failed; ++t) {
+                    const int q0 = (int)(t * TILE_W);
+                    for (int kc = 0; kc < nkc; ++kc, ++it) {
+                        const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                        if (!mbar_wait_bounded(raw_empty + 8u * s, ph ^ 1u)) { failed = true; break; }
+                        mbar_arrive_expect_tx(raw_full + 8u * s, chunk_bytes);
+                        tma_load_3d(raw_u32 + s * chunk_bytes, &tmap_in, q0, kc * KC, w, raw_full + 8u * s);
+                    }
+                }
+            }
+        } else if (warp == 1 || warp == 2) {
+            // ================= MMA issuer of half m: accumulators 2m, 2m+1 alternate by tile
+            if (lane == 0) {
+                const uint32_t m = (uint32_t)(warp - 1);
+                const uint32_t idesc = idesc_tf32_ts((uint32_t)Npad);
+                const uint32_t b_lbo = (uint32_t)K_pad * 128u;
+                const uint64_t bhi0 = make_desc(bhi_u32, b_lbo, 512u), blo0 = make_desc(blo_u32, b_lbo, 512u);
+                for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                    const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
+                    const uint32_t d_tmem = tmem_base + (2u * m + buf) * (uint32_t)Npad;
+                    if (!mbar_wait_bounded(acc_empty + 8u * (2u * m + buf), aph ^ 1u)) { failed = true; break; }
+                    tc_fence_after();
+                    for (int kc = 0; kc < nkc; ++kc) {
+                        const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
+                        const uint32_t ab = m * NAh + seq % NAh, ph = (seq / NAh) & 1u;
+                        if (!mbar_wait_bounded(a_full + 8u * ab, ph)) { failed = true; break; }
+                        tc_fence_after();
+                        const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
+                        int ksteps = KC / 8;
+                        const int rows_left = tp.K_rows - kc * KC;               // rows with data in this chunk
+                        if (rows_left < KC) ksteps = (rows_left + 7) / 8;
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            // descriptor start address advances by 8 rows x 128 B (in 16-byte units)
+                            const uint64_t boff = (uint64_t)(((kc * KC + ks * 8) * 128) >> 4);
+                            tc_mma_tf32_ts(d_tmem, a_lo + ks * 8u, bhi0 + boff, idesc, (kc | ks) != 0);
+                            tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, blo0 + boff, idesc, 1u);
+                            tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, bhi0 + boff, idesc, 1u);
+                        }
+                        tc_commit(a_empty + 8u * ab);      // the A buffer is free once these MMAs have read it
+                    }
+                    if (failed) break;
+                    tc_commit(acc_full + 8u * (2u * m + buf));          // the accumulator is complete
+                }
+            }
+        } else if (warp < WARP_SPLIT0) {
+            // ================= epilogue (TMEM lanes 32*(warp%4) ..; group g takes rows 16g..16g+15 of every 32)
+            const int qd = warp & 3, g = (warp - WARP_EPI0) >> 2;
+            const int pos = qd * 32 + lane;
+            for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
+                for (int nb = 0; nb < nblk && !failed; ++nb, ++oc) {
+                    const uint32_t ob = oc & 1u, oph = (oc >> 1) & 1u;
+                    if (!warp_wait(out_free + 8u * ob, oph ^ 1u)) { failed = true; break; }
+                    float* o = out_s + (size_t)ob * (OUT_ROWS * TILE_W) + (size_t)(g * 16) * TILE_W + pos;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t acc = 2u * h + buf;
+                        if (nb == 0 && !warp_wait(acc_full + 8u * acc, aph)) { failed = true; break; }
+                        tc_fence_after();
+                        float v[16];
+                        tc_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + acc * (uint32_t)Npad + (uint32_t)(nb * 32 + g * 16), v);
+                        if (nb == nblk - 1) {
+                            // this warp's part of the accumulator is in registers: hand it back
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(acc_empty + 8u * acc);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) o[j * TILE_W + h * HALF_M] = v[j] * a.scale;
+                    }
+                    if (failed) break;
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(out_full + 8u * ob);
+                    if (warp == WARP_EPI0) {
+                        if (lane == 0) {
+                            if (!mbar_wait_bounded(out_full + 8u * ob, oph)) {
+                                failed = true;
+                            } else {
+                                // rows beyond J and positions beyond p are clipped by the tensor map
+                                tma_store_3d(&tmap_out, (int)(t * TILE_W), nb * OUT_ROWS, w, out_u32 + ob * out_bytes);
+                                bulk_commit();
+                                if (oc >= 1) {                 // the store before this one has read its tile: free it
+                                    bulk_wait_read_1();
+                                    mbar_arrive(out_free + 8u * (ob ^ 1u));
+                                }
+                            }
+                        }
+                        failed = __any_sync(0xffffffffu, failed ? 1 : 0) != 0;
+                    }
+                }
+            }
+        } else {
+            // ================= splitter (TMEM lanes 32*(warp%4) ..; group g takes rows [g*KG, (g+1)*KG) of the chunk)
+            const int qd = warp & 3, g = (warp - WARP_SPLIT0) >> 2;
+            const int pos = qd * 32 + lane;
+            const int r0 = g * KG;
+            for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                for (int kc = 0; kc < nkc && !failed; ++kc, ++it) {
+                    const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                    const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
+                    const uint32_t abi = seq % NAh, pa = (seq / NAh) & 1u;
+                    if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
+                    const float* col = raw_s + (size_t)s * (KC * TILE_W) + (size_t)r0 * TILE_W + pos;
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t hi[KG], lo[KG];
+#pragma unroll
+                        for (int k = 0; k < KG; ++k) {
+                            const float x = col[k * TILE_W + h * HALF_M];
+                            hi[k] = tf32_bits(x);
+                            lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
+                        }
+                        if (h == 1) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(raw_empty + 8u * s);        // both halves are in registers
+                        }
+                        const uint32_t ab = (uint32_t)h * NAh + abi;
+                        if (!warp_wait(a_empty + 8u * ab, pa ^ 1u)) { failed = true; break; }
+                        tc_fence_after();
+                        const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC) + (uint32_t)r0;
+#pragma unroll
+                        for (int k4 = 0; k4 < KG / 4; ++k4) {
+                            tc_st4(ta + 4u * k4, hi + 4 * k4);
+                            tc_st4(ta + KC + 4u * k4, lo + 4 * k4);
+                        }
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(a_full + 8u * ab);
+                    }
+                }
+            }
+        }
+        // ---------------- end of segment: all products that read these coefficients are done
+        // (the epilogue has waited for every accumulator) before the next worker's overwrite them
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+    }
+
+    if (warp == WARP_EPI0 && lane == 0) bulk_wait_all();   // all output has left shared memory and is written
+    if (failed) {
+        if (lane == 0) atomicExch(a.status, 2);
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 2000000ull) { }      // let async work that is in flight finish
+    }
+    // ---------------- tear-down: every warp arrives here (all waits above are bounded)
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tc_dealloc(tmem_base, (uint32_t)tp.tmem_cols);
+    }
+}
+
+template <int KC>
+cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a, const PairParams& tp,
+                      size_t smem, int grid, cudaStream_t s) {
+    auto kern = contract_tc_pair_kernel<KC>;
+    {   // per device and cheap: set on every launch rather than cached
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<grid, NUM_THREADS, smem, s>>>(tin, tout, a, tp);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_pair_eligible(const ContractArgs& a) {
+    return tc_eligible(a) && a.J <= 64;
+}
+
+cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches) {
+    PairParams tp;
+    const bool has_skip = a.skip_row < a.K;                 // decode: one physical row is not part of Y
+    tp.K_rows = a.K + (has_skip ? 1 : 0);
+    tp.Npad = ((a.J + 31) / 32) * 32;
+    // rows per chunk: as few padded rows as possible, then as large as possible, with at least
+    // 3 stages in the shared memory that the coefficient copies and the output tiles leave and
+    // at least two A buffers per half in the tensor memory that the four accumulators leave
+    const size_t budget = 227 * 1024 - 1024;
+    const int cands[4] = {40, 32, 24, 16};
+    int best_kc = 0, best_pad = 1 << 30, best_stages = 0;
+    for (int ci = 0; ci < 4; ++ci) {
+        const int kc = cands[ci];
+        if (g_tune_tc_kc && kc != g_tune_tc_kc) continue;
+        if (4 * tp.Npad + 2 * 2 * 2 * kc > 512) continue;
+        const int kpad = ((tp.K_rows + kc - 1) / kc) * kc;
+        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp.Npad * 4 + 2 * OUT_ROWS * TILE_W * 4 + 512;
+        const size_t stage_c = (size_t)kc * TILE_W * 4;
+        if (fixed_c + 3 * stage_c > budget) continue;
+        int st = (int)((budget - fixed_c) / stage_c);
+        if (st > 8) st = 8;
+        if (g_tune_tc_stages && g_tune_tc_stages < st) st = g_tune_tc_stages;
+        if (st < 2) continue;
+        if (kpad < best_pad) { best_pad = kpad; best_kc = kc; best_stages = st; }
+    }
+    if (!best_kc) return cudaErrorInvalidConfiguration;
+    const int KC = best_kc;
+    tp.K_pad = best_pad;
+    tp.stages = best_stages;
+    tp.NAh = (512 - 4 * tp.Npad) / (2 * 2 * KC);
+    if (tp.NAh > 4) tp.NAh = 4;
+    tp.tmem_cols = 32;
+    while (tp.tmem_cols < 4 * tp.Npad + 2 * tp.NAh * 2 * KC) tp.tmem_cols *= 2;
+    const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * TILE_W * 4 +
+                        2 * OUT_ROWS * TILE_W * 4 + 512;
+
+    CUtensorMap tin, tout;
+    if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, TILE_W, KC)) return cudaErrorInvalidValue;
+    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, TILE_W, OUT_ROWS)) return cudaErrorInvalidValue;
+
+    tp.tiles_per_worker = (a.p + TILE_W - 1) / TILE_W;
+    tp.total_tiles = tp.tiles_per_worker * a.N;
+    int grid = num_sms;
+    if ((int64_t)grid > tp.total_tiles) grid = (int)tp.total_tiles;
+    cudaError_t e;
+    switch (KC) {
+        case 40: e = launch_kc<40>(tin, tout, a, tp, smem, grid, s); break;
+        case 32: e = launch_kc<32>(tin, tout, a, tp, smem, grid, s); break;
+        case 24: e = launch_kc<24>(tin, tout, a, tp, smem, grid, s); break;
+        default: e = launch_kc<16>(tin, tout, a, tp, smem, grid, s); break;
+    }
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+}  // namespace cerar

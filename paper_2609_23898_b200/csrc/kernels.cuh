@@ -42,6 +42,11 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
 // Tensor-core (tcgen05, 3 x TF32) contraction; tc_eligible says whether the shape fits it.
 bool tc_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
+// The same contraction on tiles of 256 positions (1 KB rows in global memory), for c <= 64.
+bool tc_pair_eligible(const ContractArgs& a);
+cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
+// Tuning knobs (0 = default), settable through cerar_set_tuning.
+extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
 // A kernel whose bounded wait is made to run out (nothing arrives on its barrier).
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);

@@ -123,6 +123,31 @@ def test_tensor_core_kernel_is_what_runs(cerar_mod):
         run_library(plan, _inputs().gradients_numpy(4, 16 * 1024, "normal", seed=5), 1.0)
 
 
+@pytest.mark.parametrize("N,c,p", [(8, 32, 2048 + 132), (3, 32, 256 * 150 + 8), (2, 64, 51300), (8, 48, 260),
+                                   (16, 40, 1028), (4, 64, 256)])
+def test_tensor_core_tile_variants(cerar_mod, N, c, p):
+    """The tensor-core contraction has two tilings for c <= 64: tiles of 256 positions,
+    one contiguous range of the (worker, tile) list per CTA (ranges cross worker
+    boundaries in these shapes), and tiles of 128 positions per worker.  Both must
+    match the oracle, and each other bit for bit (same products in the same order)."""
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(100 * N + c))
+    g = _inputs().gradients_numpy(N, c * p, "normal", seed=8)
+    ora = run_oracle(des.U, des.R, g, 0.25)
+    outs = []
+    try:
+        for variant in (0, 1):
+            assert cerar_mod.cerar_set_tuning("tc_variant", variant) == 0
+            plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+            plan.set_kernel_mode(cerar_mod.KERNEL_TC)
+            res = run_library(plan, g, 0.25)
+            _check_stages(res, ora, OUT_TOL, N)
+            outs.append(res)
+    finally:
+        cerar_mod.cerar_set_tuning("tc_variant", 0)
+    assert np.array_equal(outs[0]["Delta"], outs[1]["Delta"])
+    assert np.array_equal(outs[0]["out"], outs[1]["out"])
+
+
 @pytest.mark.parametrize("N,c,eps,p", [(4, 4, 1e-3, 5000), (8, 8, 1e-3, 2052), (16, 16, 1e-3, 1028)])
 def test_well_conditioned_designs_meet_the_bar(cerar_mod, N, c, eps, p):
     """c = N designs (r* = 0) have kappa of order 10..100: decoded output within
