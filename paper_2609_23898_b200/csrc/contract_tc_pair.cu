@@ -8,7 +8,7 @@
 // SIMT roles have two warps per TMEM lane quadrant.  A tile of 256 positions is two
 // UMMA tiles of M = 128 ("halves"); half h belongs to MMA issuer h for the whole run.
 //
-// One CTA of 19 warps per SM.  The tiles of all workers form one list that is cut
+// One CTA of 21 warps per SM.  The tiles of all workers form one list that is cut
 // into one contiguous range per CTA, so every SM is busy; a range that crosses a
 // worker boundary is processed in two segments (the coefficients are per worker).
 //   warp 0        producer: one TMA load per chunk ([KC rows] x [256 positions])
@@ -16,7 +16,8 @@
 //                 lane quadrant take one half of the chunk's rows each; values are split
 //                 into tf32 hi | lo and written to tensor memory (tcgen05.st), where
 //                 they are the A operand of their half
-//   warps 1, 2    MMA issuers (one lane each) for half 0 / 1: tcgen05.mma kind::tf32,
+//   warps 1, 2    (and 19, 20 for the odd tiles where the A buffers allow it)
+//                 MMA issuers (one lane each) for half 0 / 1: tcgen05.mma kind::tf32,
 //                 A from TMEM, B = the coefficients (hi and lo copies) in shared memory,
 //                 M=128, N=Npad, K=8; two accumulators each, so that the epilogue of one
 //                 tile overlaps the products of the next; warp 1 owns the TMEM allocation
@@ -41,9 +42,9 @@ using namespace tc;
 constexpr int HALF_M = 128;              // UMMA M
 constexpr int TILE_W = 2 * HALF_M;       // positions per tile
 constexpr int OUT_ROWS = 32;             // output rows per TMA store
-constexpr int NUM_WARPS = 19;
+constexpr int NUM_WARPS = 21;
 constexpr int NUM_THREADS = 32 * NUM_WARPS;
-constexpr int WARP_EPI0 = 3, WARP_SPLIT0 = 11;
+constexpr int WARP_EPI0 = 3, WARP_SPLIT0 = 11, WARP_MMA2 = 19;
 
 struct PairParams {
     int K_rows;        // physical input rows that carry data; rows beyond read as zero (TMA fill)
@@ -52,6 +53,7 @@ struct PairParams {
     int NAh;           // A (hi|lo) chunk buffers per half in tensor memory
     int Npad;          // J rounded up to 32
     int tmem_cols;     // power of two >= 4*Npad + 2*NAh*2*KC
+    int four_issuers;  // 1: every half has one issuer per accumulator (even / odd tiles)
     int64_t tiles_per_worker;
     int64_t total_tiles;
 };
@@ -157,15 +159,19 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
                     }
                 }
             }
-        } else if (warp == 1 || warp == 2) {
-            // ================= MMA issuer of half m: accumulators 2m, 2m+1 alternate by tile
-            if (lane == 0) {
-                const uint32_t m = (uint32_t)(warp - 1);
+        } else if (warp == 1 || warp == 2 || warp >= WARP_MMA2) {
+            // ================= MMA issuer of half m: accumulators 2m, 2m+1 alternate by tile.
+            // With four issuers, warps 1, 2 take the even tiles and warps 19, 20 the odd ones
+            // (an issuing thread is limited by its own instruction stream, not by the tensor pipe).
+            const bool odd_only = warp >= WARP_MMA2;
+            if (lane == 0 && (tp.four_issuers || !odd_only)) {
+                const uint32_t m = (uint32_t)(odd_only ? warp - WARP_MMA2 : warp - 1);
                 const uint32_t idesc = idesc_tf32_ts((uint32_t)Npad);
                 const uint32_t b_lbo = (uint32_t)K_pad * 128u;
                 const uint64_t bhi0 = make_desc(bhi_u32, b_lbo, 512u), blo0 = make_desc(blo_u32, b_lbo, 512u);
                 for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
                     const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
+                    if (tp.four_issuers && (buf != 0u) != odd_only) continue;
                     const uint32_t d_tmem = tmem_base + (2u * m + buf) * (uint32_t)Npad;
                     if (!mbar_wait_bounded(acc_empty + 8u * (2u * m + buf), aph ^ 1u)) { failed = true; break; }
                     tc_fence_after();
@@ -352,6 +358,14 @@ cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s,
     tp.stages = best_stages;
     tp.NAh = (512 - 4 * tp.Npad) / (2 * 2 * KC);
     if (tp.NAh > 4) tp.NAh = 4;
+    // Two issuers per half wait on the same A-buffer barriers in turn; a parity wait is only
+    // sound if the waiter is at most one phase ahead, which holds when a tile's chunks plus
+    // one fit in the buffers of a half.
+    // Measured on B200 at c = 32: a second pair pays once a tile has more than 4 k-steps
+    // (decode +5 %), and costs 2 % below that (encode).
+    tp.four_issuers = (tp.NAh >= tp.K_pad / KC + 1 && (tp.K_rows + 7) / 8 > 4) ? 1 : 0;
+    if (g_tune_tc_variant == 2) tp.four_issuers = 0;
+    if (g_tune_tc_variant == 3 && tp.NAh >= tp.K_pad / KC + 1) tp.four_issuers = 1;
     tp.tmem_cols = 32;
     while (tp.tmem_cols < 4 * tp.Npad + 2 * tp.NAh * 2 * KC) tp.tmem_cols *= 2;
     const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * TILE_W * 4 +

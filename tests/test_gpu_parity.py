@@ -128,14 +128,15 @@ def test_tensor_core_kernel_is_what_runs(cerar_mod):
 def test_tensor_core_tile_variants(cerar_mod, N, c, p):
     """The tensor-core contraction has two tilings for c <= 64: tiles of 256 positions,
     one contiguous range of the (worker, tile) list per CTA (ranges cross worker
-    boundaries in these shapes), and tiles of 128 positions per worker.  Both must
-    match the oracle, and each other bit for bit (same products in the same order)."""
+    boundaries in these shapes) with one or two MMA issuers per half, and tiles of 128
+    positions per worker.  All must match the oracle, and each other bit for bit (same
+    products in the same order)."""
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(100 * N + c))
     g = _inputs().gradients_numpy(N, c * p, "normal", seed=8)
     ora = run_oracle(des.U, des.R, g, 0.25)
     outs = []
     try:
-        for variant in (0, 1):
+        for variant in (0, 1, 2, 3):
             assert cerar_mod.cerar_set_tuning("tc_variant", variant) == 0
             plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
             plan.set_kernel_mode(cerar_mod.KERNEL_TC)
@@ -144,8 +145,9 @@ def test_tensor_core_tile_variants(cerar_mod, N, c, p):
             outs.append(res)
     finally:
         cerar_mod.cerar_set_tuning("tc_variant", 0)
-    assert np.array_equal(outs[0]["Delta"], outs[1]["Delta"])
-    assert np.array_equal(outs[0]["out"], outs[1]["out"])
+    for other in outs[1:]:
+        assert np.array_equal(outs[0]["Delta"], other["Delta"])
+        assert np.array_equal(outs[0]["out"], other["out"])
 
 
 @pytest.mark.parametrize("N,c,eps,p", [(4, 4, 1e-3, 5000), (8, 8, 1e-3, 2052), (16, 16, 1e-3, 1028)])
