@@ -200,6 +200,39 @@ cerar_status_t cerar_allreduce_fused(cerar_plan_t* plan, const float* grads, int
                                      cerar_stream_t stream);
 int            cerar_fused_supported(const cerar_plan_t* plan);
 
+/* ---- One worker per GPU (the ring the paper runs between machines, Sec. II and
+ * Algorithm 1; its Sec. V names the fused compute/transfer form as future work).
+ * Each call serves ONE worker `rank` in 0..N-1, whose state is its own workspace of
+ * cerar_rank_workspace_bytes(plan, d) = (c+N+1) (d/c) 4 bytes on this GPU: row
+ * ("slot") k-1 receives message k, slot N+j holds delta_{rank,j}.  The one row more
+ * than the single-GPU layout is the landing buffer of the transport: the slot that
+ * the previous worker writes in round k is not one that its owner reads in round k.
+ *
+ * cerar_rank_encode: Delta = G U_rank from the worker's gradient `grad` (d floats,
+ *   device; may be the D rows of ws itself: ws + (N+1) (d/c)) into slots N+1..N+c.
+ * cerar_rank_round: forms message k, x = (y_{k-1} - delta_{k-N}) + delta_k with the
+ *   terms that exist (Eq. update_eqns), from this worker's slots and stores it into
+ *   slot k-1 of `peer_ws`, the workspace of worker rank+1 (mod N).  peer_ws may point
+ *   into another GPU's memory (peer access enabled by the caller): the kernel uses
+ *   plain 16-byte stores.  The CALLER orders the rounds: round k of a worker may
+ *   start once round k-1 has completed on this worker and on both neighbours (one
+ *   barrier per round between all workers is enough); the library keeps no round
+ *   state for these calls and waits on nothing.
+ * cerar_rank_decode: out (d floats, device) = scale * Y_rank R_rank after round L.
+ * cerar_rank_round_slots: the slots round k reads (-1 where the term is absent) and
+ *   the landing slot, for callers that schedule or check the transfers themselves.
+ * Errors as for the calls above; rank or k out of range is CERAR_ERR_INVALID_ARG /
+ * CERAR_ERR_STATE.  All device work is asynchronous on `stream`. */
+size_t         cerar_rank_workspace_bytes(const cerar_plan_t* plan, int64_t d);
+cerar_status_t cerar_rank_round_slots(const cerar_plan_t* plan, int k, int* slot_prev, int* slot_cancel,
+                                      int* slot_add, int* slot_land);
+cerar_status_t cerar_rank_encode(cerar_plan_t* plan, int rank, const float* grad, float* ws, int64_t d,
+                                 cerar_stream_t stream);
+cerar_status_t cerar_rank_round(cerar_plan_t* plan, int rank, const float* ws, float* peer_ws, int64_t d, int k,
+                                cerar_stream_t stream);
+cerar_status_t cerar_rank_decode(cerar_plan_t* plan, int rank, const float* ws, float* out, int64_t d,
+                                 float scale, cerar_stream_t stream);
+
 /* The same pipeline as cerar_allreduce_sim for callers that cannot provide a
  * workspace because they cannot allocate device memory at this point: for
  * instance a host program whose framework has already claimed all free memory

@@ -78,6 +78,12 @@ lib.cerar_allreduce_sim_host.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _
 lib.cerar_allreduce_sim_static.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _i64, C.c_float, _vp]
 lib.cerar_allreduce_fused.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _i64, C.c_float, _vp]
 lib.cerar_fused_supported.argtypes = [_vp]
+lib.cerar_rank_workspace_bytes.argtypes = [_vp, _i64]
+lib.cerar_rank_workspace_bytes.restype = C.c_size_t
+lib.cerar_rank_round_slots.argtypes = [_vp, C.c_int] + [C.POINTER(C.c_int)] * 4
+lib.cerar_rank_encode.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, _vp]
+lib.cerar_rank_round.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, C.c_int, _vp]
+lib.cerar_rank_decode.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, C.c_float, _vp]
 lib.cerar_get_counters.argtypes = [_vp, C.POINTER(Counters)]
 lib.cerar_launch_count.argtypes = [_vp]
 lib.cerar_launch_count.restype = C.c_uint64
@@ -213,6 +219,25 @@ class Plan:
 
     def fused_supported(self) -> bool:
         return bool(lib.cerar_fused_supported(self._h))
+
+    # ---- one worker per GPU
+    def rank_workspace_bytes(self, d: int) -> int:
+        return int(lib.cerar_rank_workspace_bytes(self._h, d))
+
+    def rank_round_slots(self, k: int):
+        """(slot_prev, slot_cancel, slot_add, slot_land) of round k; -1 where the term is absent."""
+        v = [C.c_int() for _ in range(4)]
+        _check(lib.cerar_rank_round_slots(self._h, k, *[C.byref(x) for x in v]))
+        return tuple(x.value for x in v)
+
+    def rank_encode(self, rank, grad, ws, d, stream=0):
+        _check(lib.cerar_rank_encode(self._h, rank, _ptr(grad), _ptr(ws), d, stream))
+
+    def rank_round(self, rank, ws, peer_ws, d, k, stream=0):
+        _check(lib.cerar_rank_round(self._h, rank, _ptr(ws), _ptr(peer_ws), d, k, stream))
+
+    def rank_decode(self, rank, ws, out, d, scale=1.0, stream=0):
+        _check(lib.cerar_rank_decode(self._h, rank, _ptr(ws), _ptr(out), d, scale, stream))
 
     def allreduce_sim_static(self, grads, grads_stride, out, out_stride, d, scale=1.0, stream=0):
         """cerar_allreduce_sim_static: same pipeline, workspace built into the library (<= 64 MiB)."""

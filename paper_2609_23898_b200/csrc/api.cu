@@ -261,7 +261,7 @@ cerar_status_t cerar_encode(cerar_plan_t* P, const float* grads, int64_t grads_s
     cerar::ContractArgs a{};
     a.in = grads; a.in_wstride = grads_stride; a.in_rstride = p;
     a.out = ws + (int64_t)N * p; a.out_wstride = (int64_t)(c + N) * p; a.out_rstride = p;
-    a.coef = P->d_U; a.K = c; a.J = c; a.skip_row = 1 << 30;
+    a.coef = P->d_U; a.K = c; a.J = c; a.skip_row = 1 << 30; a.skip_count = 0;
     a.N = N; a.p = p; a.scale = 1.0f; a.status = P->d_status;
     cudaError_t e = cerar::launch_contract(a, P->kernel_mode, P->num_sms, (cudaStream_t)stream, &P->launches);
     if (e != cudaSuccess) return cuda_fail(e, "encode launch");
@@ -297,7 +297,7 @@ cerar_status_t cerar_decode(cerar_plan_t* P, const float* ws, float* out, int64_
     cerar::ContractArgs a{};
     a.in = ws; a.in_wstride = (int64_t)(c + N) * p; a.in_rstride = p;
     a.out = out; a.out_wstride = out_stride; a.out_rstride = p;
-    a.coef = P->d_R; a.K = L + 1; a.J = c; a.skip_row = L;     // y_{L+1} sits in slot L+1
+    a.coef = P->d_R; a.K = L + 1; a.J = c; a.skip_row = L; a.skip_count = 1;     // y_{L+1} sits in slot L+1
     a.N = N; a.p = p; a.scale = scale; a.status = P->d_status;
     cudaError_t e = cerar::launch_contract(a, P->kernel_mode, P->num_sms, (cudaStream_t)stream, &P->launches);
     if (e != cudaSuccess) return cuda_fail(e, "decode launch");
@@ -376,6 +376,74 @@ cerar_status_t cerar_allreduce_sim_host(cerar_plan_t* P, const float* h_grads, i
     // counters describe the whole job, not the last slice
     P->cur_d = d;
     P->bytes_forwarded = (uint64_t)4 * (uint64_t)p * (uint64_t)P->host.L;
+    return CERAR_OK;
+}
+
+// ---------------------------------------------------------------- one worker per GPU
+size_t cerar_rank_workspace_bytes(const cerar_plan_t* P, int64_t d) {
+    if (!P || d <= 0 || d % P->host.c != 0) return 0;
+    return (size_t)4 * (size_t)(P->host.c + P->host.N + 1) * (size_t)(d / P->host.c);
+}
+
+cerar_status_t cerar_rank_round_slots(const cerar_plan_t* P, int k, int* slot_prev, int* slot_cancel, int* slot_add,
+                                      int* slot_land) {
+    if (!P || !slot_prev || !slot_cancel || !slot_add || !slot_land) return fail(CERAR_ERR_INVALID_ARG, "bad argument");
+    if (k < 1 || k > P->host.L) return fail(CERAR_ERR_INVALID_ARG, "round index outside 1..L");
+    cerar::rank_round_slots(P->host.N, P->host.c, k, slot_prev, slot_cancel, slot_add, slot_land);
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_rank_encode(cerar_plan_t* P, int rank, const float* grad, float* ws, int64_t d,
+                                 cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!grad || !ws) return fail(CERAR_ERR_INVALID_ARG, "grad or ws is NULL");
+    const int N = P->host.N, c = P->host.c;
+    if (rank < 0 || rank >= N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    cerar::ContractArgs a{};
+    // one worker per call: the worker strides are never stepped, but keep them what they would be
+    a.in = grad; a.in_wstride = (int64_t)c * p; a.in_rstride = p;
+    a.out = ws + (int64_t)(N + 1) * p; a.out_wstride = (int64_t)(c + N + 1) * p; a.out_rstride = p;
+    a.coef = P->d_U + (size_t)rank * c * c; a.K = c; a.J = c; a.skip_row = 1 << 30; a.skip_count = 0;
+    a.N = 1; a.p = p; a.scale = 1.0f; a.status = P->d_status;
+    cudaError_t e = cerar::launch_contract(a, P->kernel_mode, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rank encode launch");
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_rank_round(cerar_plan_t* P, int rank, const float* ws, float* peer_ws, int64_t d, int k,
+                                cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !peer_ws) return fail(CERAR_ERR_INVALID_ARG, "ws or peer_ws is NULL");
+    if (ws == peer_ws) return fail(CERAR_ERR_INVALID_ARG, "peer_ws must be the next worker's workspace, not this one's");
+    if (rank < 0 || rank >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    if (k < 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "round index outside 1..L");
+    cerar::RankRoundArgs a{};
+    a.ws = ws; a.peer_ws = peer_ws; a.p = p; a.N = P->host.N; a.c = P->host.c; a.k = k;
+    cudaError_t e = cerar::launch_rank_round(a, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rank round launch");
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_rank_decode(cerar_plan_t* P, int rank, const float* ws, float* out, int64_t d, float scale,
+                                 cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !out) return fail(CERAR_ERR_INVALID_ARG, "ws or out is NULL");
+    const int N = P->host.N, c = P->host.c, L = P->host.L;
+    if (rank < 0 || rank >= N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    cerar::ContractArgs a{};
+    a.in = ws; a.in_wstride = (int64_t)(c + N + 1) * p; a.in_rstride = p;
+    a.out = out; a.out_wstride = (int64_t)c * p; a.out_rstride = p;
+    // y_1..y_L sit in slots 0..L-1, y_{L+1} = delta_c in slot N+c = L+2; slots L and L+1 are spent deltas
+    a.coef = P->d_R + (size_t)rank * (L + 1) * c; a.K = L + 1; a.J = c; a.skip_row = L; a.skip_count = 2;
+    a.N = 1; a.p = p; a.scale = scale; a.status = P->d_status;
+    cudaError_t e = cerar::launch_contract(a, P->kernel_mode, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rank decode launch");
     return CERAR_OK;
 }
 

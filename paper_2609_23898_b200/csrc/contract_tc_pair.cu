@@ -128,9 +128,9 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
             uint32_t* blo = reinterpret_cast<uint32_t*>(smem_al + b_bytes);
             for (int idx = threadIdx.x; idx < K_pad * Npad; idx += blockDim.x) {
                 const int k = idx / Npad, j = idx - k * Npad;
-                // physical input row k -> coefficient row (the row at skip_row is not part of Y: zero)
+                // physical input row k -> coefficient row (skipped rows are not part of Y: zero)
                 int src = -1;
-                if (k < a.skip_row) src = k; else if (k > a.skip_row) src = k - 1;
+                if (k < a.skip_row) src = k; else if (k >= a.skip_row + a.skip_count) src = k - a.skip_count;
                 float v = 0.f;
                 if (src >= 0 && src < a.K && j < a.J) v = cf[(size_t)src * a.J + j];
                 const uint32_t hi = tf32_bits(v);
@@ -329,8 +329,7 @@ bool tc_pair_eligible(const ContractArgs& a) {
 
 cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches) {
     PairParams tp;
-    const bool has_skip = a.skip_row < a.K;                 // decode: one physical row is not part of Y
-    tp.K_rows = a.K + (has_skip ? 1 : 0);
+    tp.K_rows = a.K + a.skip_count;                         // decode: physical rows that are not part of Y
     tp.Npad = ((a.J + 31) / 32) * 32;
     // rows per chunk: as few padded rows as possible, then as large as possible, with at least
     // 3 stages in the shared memory that the coefficient copies and the output tiles leave and

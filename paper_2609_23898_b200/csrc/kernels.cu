@@ -27,7 +27,7 @@ __global__ void contract_ref_kernel(const ContractArgs a) {
     const float* in = a.in + (int64_t)w * a.in_wstride + q;
     const float* cf = a.coef + (size_t)w * a.K * a.J;
     for (int k = 0; k < a.K; ++k) {
-        const int row = (k < a.skip_row) ? k : k + 1;
+        const int row = (k < a.skip_row) ? k : k + a.skip_count;
         const float x = in[(int64_t)row * a.in_rstride];
         for (int j = 0; j < a.J; ++j) acc[j] = fmaf(cf[(size_t)k * a.J + j], x, acc[j]);
     }
@@ -100,7 +100,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                 __syncwarp();
                 for (int r = lane; r < kcount; r += 32) {
                     const int k = k0 + r;
-                    const int row = (k < a.skip_row) ? k : k + 1;
+                    const int row = (k < a.skip_row) ? k : k + a.skip_count;
                     bulk_load(stage0 + s * stage_bytes + (uint32_t)r * tile_p * 4u,
                               in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, full0 + 8u * s);
                 }

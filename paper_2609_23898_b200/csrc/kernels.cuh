@@ -17,7 +17,8 @@ struct ContractArgs {
     int64_t out_rstride;
     const float* coef;      // device: worker i's K x J row-major matrix at coef + i*K*J
     int K, J;
-    int skip_row;           // input row index r >= skip_row reads physical row r+1
+    int skip_row;           // input row index r >= skip_row reads physical row r + skip_count
+    int skip_count;         // physical rows skip_row .. skip_row+skip_count-1 are not inputs (0 = none)
     int N;
     int64_t p;
     float scale;
@@ -34,6 +35,15 @@ struct RoundArgs {
     int N, c, k;            // round k in 1..L
 };
 
+// One worker's ring round in the one-worker-per-GPU layout ((c+N+1) x p per worker).
+struct RankRoundArgs {
+    const float* ws;        // this worker's workspace
+    float* peer_ws;         // the next worker's workspace (may be peer-mapped memory of another GPU)
+    int64_t p;
+    int N, c, k;            // round k in 1..L
+    int slot_prev, slot_cancel, slot_add, slot_land;   // filled in by the launcher (-1 = term absent)
+};
+
 enum { KERNEL_AUTO = 0, KERNEL_REF = 1, KERNEL_STAGED = 2, KERNEL_TC = 3 };
 
 // Returns cudaSuccess or the launch error.  *launches is incremented by the
@@ -48,6 +58,10 @@ cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s,
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
 extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
+// Slots of the per-worker layout that round k reads (-1 = term absent) and the landing slot
+// in the neighbour's workspace; the one definition that launcher and callers share.
+void rank_round_slots(int N, int c, int k, int* slot_prev, int* slot_cancel, int* slot_add, int* slot_land);
+cudaError_t launch_rank_round(RankRoundArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // A kernel whose bounded wait is made to run out (nothing arrives on its barrier).
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);
 // Whole protocol in one launch with the slots in shared memory (small N (c+N) only).

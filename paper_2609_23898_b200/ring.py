@@ -1,0 +1,102 @@
+"""CERAR with one worker per rank: drivers around the cerar_rank_* calls.
+
+The protocol (Sec. II, Algorithm 1) per worker i: encode, then L rounds in which the
+worker forms message k from its own slots and stores it into the landing slot of
+worker i+1, then decode.  The kernels are the library's; this module only owns the
+buffers and the order of the calls.
+
+LocalRing         all N workers in this process on one GPU, each with its own
+                  workspace; "the neighbour's memory" is just another tensor and
+                  stream order stands in for the barrier between rounds.  This is
+                  what the GPU tests and the single-GPU measurements run.
+DistributedRing   one worker per process and GPU (torch.distributed, NCCL): the
+                  workspace lives in symmetric memory, the neighbour's copy is a
+                  peer-mapped tensor, and a device-side barrier on the stream
+                  separates the rounds.  Needs N GPUs with peer access.
+"""
+from __future__ import annotations
+
+from . import cerar
+
+
+def round_schedule(plan):
+    """[(k, slot_prev, slot_cancel, slot_add, slot_land)] for k = 1..L as the library
+    computes them (-1 = the term is absent in that round)."""
+    return [(k,) + plan.rank_round_slots(k) for k in range(1, plan.L + 1)]
+
+
+def y_slots(plan):
+    """Slots that hold y_1 .. y_{L+1} after round L (the rows decode reads, in order)."""
+    return list(range(plan.L)) + [plan.N + plan.c]
+
+
+class LocalRing:
+    def __init__(self, plan, d: int, device="cuda"):
+        import torch
+        if d % plan.c:
+            raise ValueError("d must be a multiple of c")
+        self.plan, self.d, self.p = plan, d, d // plan.c
+        self.N, self.c, self.L = plan.N, plan.c, plan.L
+        n = plan.rank_workspace_bytes(d) // 4
+        self.ws = [torch.empty(n, dtype=torch.float32, device=device) for _ in range(self.N)]
+
+    def grad_view(self, i):
+        """The D rows of worker i's workspace as a length-d tensor (in-place use)."""
+        o = (self.N + 1) * self.p
+        return self.ws[i][o:o + self.d]
+
+    def encode(self, grads, stream=0):
+        for i in range(self.N):
+            self.plan.rank_encode(i, grads[i], self.ws[i], self.d, stream)
+
+    def round(self, k, stream=0):
+        # every worker's launch of round k is queued after all launches of round k-1
+        for i in range(self.N):
+            self.plan.rank_round(i, self.ws[i], self.ws[(i + 1) % self.N], self.d, k, stream)
+
+    def decode(self, outs, scale=1.0, stream=0):
+        for i in range(self.N):
+            self.plan.rank_decode(i, self.ws[i], outs[i], self.d, scale, stream)
+
+    def allreduce(self, grads, outs, scale=1.0, stream=0):
+        self.encode(grads, stream)
+        for k in range(1, self.L + 1):
+            self.round(k, stream)
+        self.decode(outs, scale, stream)
+
+
+class DistributedRing:
+    """One worker per rank.  `group` is a torch.distributed process group of exactly
+    plan.N ranks whose devices have peer access to one another."""
+
+    def __init__(self, plan, d: int, group=None):
+        import torch
+        import torch.distributed as dist
+        import torch.distributed._symmetric_memory as symm_mem
+        group = group if group is not None else dist.group.WORLD
+        self.rank, world = dist.get_rank(group), dist.get_world_size(group)
+        if world != plan.N:
+            raise ValueError(f"the plan is for N={plan.N} workers, the group has {world} ranks")
+        if d % plan.c:
+            raise ValueError("d must be a multiple of c")
+        self.plan, self.d, self.p = plan, d, d // plan.c
+        self.N, self.c, self.L = plan.N, plan.c, plan.L
+        n = plan.rank_workspace_bytes(d) // 4
+        self.ws = symm_mem.empty(n, dtype=torch.float32, device=torch.device("cuda", torch.cuda.current_device()))
+        self._hdl = symm_mem.rendezvous(self.ws, group)
+        self.peer_ws = self._hdl.get_buffer((self.rank + 1) % self.N, (n,), torch.float32)
+        self.barrier_timeout_ms = 10000
+
+    def _barrier(self):
+        # on the current stream: all kernels of the round before, on every rank, are
+        # complete and visible before anything after it starts
+        self._hdl.barrier(channel=0, timeout_ms=self.barrier_timeout_ms)
+
+    def allreduce(self, grad, out, scale=1.0, stream=0):
+        """grad, out: this rank's length-d device tensors; `stream` must be torch's current stream."""
+        self._barrier()                      # the neighbours are done reading the previous call's slots
+        self.plan.rank_encode(self.rank, grad, self.ws, self.d, stream)
+        for k in range(1, self.L + 1):
+            self.plan.rank_round(self.rank, self.ws, self.peer_ws, self.d, k, stream)
+            self._barrier()
+        self.plan.rank_decode(self.rank, self.ws, out, self.d, scale, stream)

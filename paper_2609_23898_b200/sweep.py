@@ -31,6 +31,9 @@ def main():
     ap.add_argument("--fused", action="store_true",
                     help="time cerar_allreduce_fused (ring on chip, out of place) next to the in-HBM pipeline "
                          "for the (N, c) it supports")
+    ap.add_argument("--ring", action="store_true",
+                    help="time the one-worker-per-rank calls (LocalRing: N workers with separate workspaces on "
+                         "this one GPU, N launches per step) next to the all-workers-per-launch pipeline")
     args = ap.parse_args()
 
     import torch
@@ -47,6 +50,8 @@ def main():
     rows = []
     if args.fused:
         return fused_table(args, exps, peak, free, stream)
+    if args.ring:
+        return ring_table(args, exps, peak, free, stream)
     print("| N | c | d | state MB | ms / aggregation | GB/s | frac of measured HBM | note |")
     print("|---|---|---|---|---|---|---|---|")
     for N in (4, 8, 16):
@@ -154,6 +159,50 @@ def fused_table(args, exps, peak, free, stream):
     if args.out:
         with open(args.out, "w") as f:
             json.dump(rows, f, indent=1)
+    return 0
+
+
+def ring_table(args, exps, peak, free, stream):
+    """The rank-level calls on one GPU: same algorithmic bytes, N launches per step instead of one."""
+    import torch
+    from . import cerar, inputs, ring
+    print("| N | c | d | pipeline ms | rank-level ms | rank-level GB/s | frac of measured HBM | launches |")
+    print("|---|---|---|---|---|---|---|---|")
+    for (N, c) in ((4, 16), (8, 32), (8, 64)):
+        rng = np.random.default_rng(0)
+        L = c + N - 2
+        U = [np.linalg.qr(rng.standard_normal((c, c)))[0] for _ in range(N)]
+        R = [rng.standard_normal((L + 1, c)) / np.sqrt(L + 1) for _ in range(N)]
+        plan = cerar.Plan.create_custom(N, c, U, R)
+        for e in exps:
+            d = 1 << e
+            p = d // c
+            if d % c or 4 * N * (2 * c + 2 * N + 1) * p + 8 * N * d > free - (2 << 30):
+                continue
+            g = torch.empty(N * d, dtype=torch.float32, device="cuda").normal_()
+            out = torch.empty(N * d, dtype=torch.float32, device="cuda")
+            ws = torch.empty(plan.workspace_bytes(d) // 4, dtype=torch.float32, device="cuda")
+            r = ring.LocalRing(plan, d)
+            grads = [g[i * d:(i + 1) * d] for i in range(N)]
+            outs = [out[i * d:(i + 1) * d] for i in range(N)]
+
+            def med(f):
+                ts = []
+                for rep in range(8):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(); f(); e1.record(); torch.cuda.synchronize()
+                    if rep >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                return float(np.median(ts))
+            t_pipe = med(lambda: plan.allreduce_sim(g, d, out, d, ws, d, 1.0 / N, stream))
+            t_ring = med(lambda: r.allreduce(grads, outs, 1.0 / N, stream))
+            plan.device_status(stream)
+            ab = 4 * N * p * (8 * c + 3 * N - 8)
+            print(f"| {N} | {c} | 2^{e} | {t_pipe:.3f} | {t_ring:.3f} | {ab / t_ring / 1e6:.0f} | "
+                  f"{ab / t_ring / 1e6 / peak:.2f} | {N * (L + 2)} |", flush=True)
+            del g, out, ws, r, grads, outs
+            torch.cuda.empty_cache()
+        plan.destroy()
     return 0
 
 
