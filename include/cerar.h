@@ -289,8 +289,8 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  * "kc" (input rows per pipeline stage), "stages", "jt" (outputs per thread: 4, 8
  * or 16), "slabs" (position slabs per CTA), "tc_kc" / "tc_stages" (rows per stage and
  * stages of the tensor-core kernel), "tc_variant" (1 = always tiles of 128 positions;
- * by default c <= 64 runs on tiles of 256 positions; 2 / 3 = those with one / two MMA
- * issuers per half wherever possible); value 0 restores the default.
+ * by default c <= 64 runs on tiles of 256 positions;
+ * 2 / 3 = tiles of 256 wherever they fit, with one / two MMA issuers per half); value 0 restores the default.
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

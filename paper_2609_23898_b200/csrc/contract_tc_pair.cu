@@ -16,7 +16,7 @@
 //                 lane quadrant take one half of the chunk's rows each; values are split
 //                 into tf32 hi | lo and written to tensor memory (tcgen05.st), where
 //                 they are the A operand of their half
-//   warps 1, 2    (and 19, 20 for the odd tiles where the A buffers allow it)
+//   warps 1, 2    (and 19, 20 for the odd tiles when a tile has more than four k-steps)
 //                 MMA issuers (one lane each) for half 0 / 1: tcgen05.mma kind::tf32,
 //                 A from TMEM, B = the coefficients (hi and lo copies) in shared memory,
 //                 M=128, N=Npad, K=8; two accumulators each, so that the epilogue of one
@@ -82,8 +82,11 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
     const uint32_t out_u32 = raw_u32 + (uint32_t)stages * chunk_bytes;
     const uint32_t bar_u32 = out_u32 + 2u * out_bytes;
     const uint32_t raw_full = bar_u32, raw_empty = raw_full + 8u * stages;
-    const uint32_t a_full = raw_empty + 8u * stages;                 // [half][NAh]
-    const uint32_t a_empty = a_full + 16u * NAh;
+    // "A buffer filled": one barrier per (half, tile parity, buffer), so that each has ONE waiter
+    // (the issuer of that half and parity) who sees all of its phases in order; a barrier that two
+    // issuers took turns on could be two phases ahead of one of them, which a parity wait cannot tell
+    const uint32_t a_full = raw_empty + 8u * stages;                 // [half][parity][NAh]
+    const uint32_t a_empty = a_full + 32u * NAh;                     // [half][NAh]
     const uint32_t acc_full = a_empty + 16u * NAh;                   // [half][2]
     const uint32_t acc_empty = acc_full + 32u;
     const uint32_t out_full = acc_empty + 32u, out_free = out_full + 16u;
@@ -94,7 +97,8 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
     // ---------------- set-up
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(raw_full + 8u * s, 1); mbar_init(raw_empty + 8u * s, 8); }
-        for (uint32_t b = 0; b < 2u * NAh; ++b) { mbar_init(a_full + 8u * b, 8); mbar_init(a_empty + 8u * b, 1); }
+        for (uint32_t b = 0; b < 4u * NAh; ++b) mbar_init(a_full + 8u * b, 8);
+        for (uint32_t b = 0; b < 2u * NAh; ++b) mbar_init(a_empty + 8u * b, 1);
         for (int b = 0; b < 4; ++b) { mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, 8); }
         for (int b = 0; b < 2; ++b) { mbar_init(out_full + 8u * b, 8); mbar_init(out_free + 8u * b, 1); }
         mbar_init_fence();
@@ -115,6 +119,7 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
 
     bool failed = false;
     uint32_t it = 0, tc = 0, oc = 0;      // chunks, tiles and output blocks this CTA has gone through (all roles count alike)
+    uint32_t afull_ph = 0;                // issuers: next phase parity of their "filled" barriers, bit = 4 * parity + buffer
 
     for (int w = w_first; w <= w_last; ++w) {
         const int64_t t_begin = (w == w_first) ? g_begin - (int64_t)w * T : 0;
@@ -177,8 +182,10 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
                     tc_fence_after();
                     for (int kc = 0; kc < nkc; ++kc) {
                         const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
-                        const uint32_t ab = m * NAh + seq % NAh, ph = (seq / NAh) & 1u;
-                        if (!mbar_wait_bounded(a_full + 8u * ab, ph)) { failed = true; break; }
+                        const uint32_t b = seq % NAh, ab = m * NAh + b;
+                        const uint32_t bit = 4u * buf + b, ph = (afull_ph >> bit) & 1u;
+                        if (!mbar_wait_bounded(a_full + 8u * ((2u * m + buf) * NAh + b), ph)) { failed = true; break; }
+                        afull_ph ^= 1u << bit;
                         tc_fence_after();
                         const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
                         int ksteps = KC / 8;
@@ -257,14 +264,20 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
                     const uint32_t abi = seq % NAh, pa = (seq / NAh) & 1u;
                     if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
                     const float* col = raw_s + (size_t)s * (KC * TILE_W) + (size_t)r0 * TILE_W + pos;
+                    // rows of this chunk that some product reads (the last chunk may be short): rounded up
+                    // to the k-step, rows beyond the data are zero (TMA fill)
+                    const int rows_left = tp.K_rows - kc * KC;
+                    const int kuse = ((rows_left < KC ? rows_left : KC) + 7) / 8 * 8 - r0;   // relative to r0
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         uint32_t hi[KG], lo[KG];
 #pragma unroll
                         for (int k = 0; k < KG; ++k) {
-                            const float x = col[k * TILE_W + h * HALF_M];
-                            hi[k] = tf32_bits(x);
-                            lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
+                            if ((k & ~3) < kuse) {
+                                const float x = col[k * TILE_W + h * HALF_M];
+                                hi[k] = tf32_bits(x);
+                                lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
+                            }
                         }
                         if (h == 1) {
                             __syncwarp();
@@ -276,13 +289,15 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
                         const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC) + (uint32_t)r0;
 #pragma unroll
                         for (int k4 = 0; k4 < KG / 4; ++k4) {
-                            tc_st4(ta + 4u * k4, hi + 4 * k4);
-                            tc_st4(ta + KC + 4u * k4, lo + 4 * k4);
+                            if (4 * k4 < kuse) {               // uniform over the warp
+                                tc_st4(ta + 4u * k4, hi + 4 * k4);
+                                tc_st4(ta + KC + 4u * k4, lo + 4 * k4);
+                            }
                         }
                         tc_wait_st();
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(a_full + 8u * ab);
+                        if (lane == 0) mbar_arrive(a_full + 8u * ((2u * (uint32_t)h + (tc & 1u)) * NAh + abi));
                     }
                 }
             }
@@ -327,44 +342,49 @@ bool tc_pair_eligible(const ContractArgs& a) {
     return tc_eligible(a) && a.J <= 64;
 }
 
-cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches) {
-    PairParams tp;
-    tp.K_rows = a.K + a.skip_count;                         // decode: physical rows that are not part of Y
-    tp.Npad = ((a.J + 31) / 32) * 32;
-    // rows per chunk: as few padded rows as possible, then as large as possible, with at least
-    // 3 stages in the shared memory that the coefficient copies and the output tiles leave and
-    // at least two A buffers per half in the tensor memory that the four accumulators leave
+// Rows per chunk (0 if nothing fits): as few chunks as possible, then as few padded rows as
+// possible, with at least 3 stages in the shared memory that the coefficient copies and the
+// output tiles leave and at least two A buffers per half in the tensor memory that the four
+// accumulators leave.
+static int choose_chunk(const ContractArgs& a, PairParams* tp) {
+    tp->K_rows = a.K + a.skip_count;                        // decode: physical rows that are not part of Y
+    tp->Npad = ((a.J + 31) / 32) * 32;
     const size_t budget = 227 * 1024 - 1024;
     const int cands[4] = {40, 32, 24, 16};
-    int best_kc = 0, best_pad = 1 << 30, best_stages = 0;
+    int best_kc = 0, best_pad = 1 << 30, best_stages = 0, best_nk = 1 << 30;
     for (int ci = 0; ci < 4; ++ci) {
         const int kc = cands[ci];
         if (g_tune_tc_kc && kc != g_tune_tc_kc) continue;
-        if (4 * tp.Npad + 2 * 2 * 2 * kc > 512) continue;
-        const int kpad = ((tp.K_rows + kc - 1) / kc) * kc;
-        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp.Npad * 4 + 2 * OUT_ROWS * TILE_W * 4 + 512;
+        if (4 * tp->Npad + 2 * 2 * 2 * kc > 512) continue;
+        const int kpad = ((tp->K_rows + kc - 1) / kc) * kc;
+        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp->Npad * 4 + 2 * OUT_ROWS * TILE_W * 4 + 512;
         const size_t stage_c = (size_t)kc * TILE_W * 4;
         if (fixed_c + 3 * stage_c > budget) continue;
         int st = (int)((budget - fixed_c) / stage_c);
         if (st > 8) st = 8;
         if (g_tune_tc_stages && g_tune_tc_stages < st) st = g_tune_tc_stages;
         if (st < 2) continue;
-        if (kpad < best_pad) { best_pad = kpad; best_kc = kc; best_stages = st; }
+        // fewest chunks first (every chunk costs a round of barrier hand-offs), then fewest padded rows
+        const int nk = kpad / kc;
+        if (nk < best_nk || (nk == best_nk && kpad < best_pad)) { best_nk = nk; best_pad = kpad; best_kc = kc; best_stages = st; }
     }
+    tp->K_pad = best_pad;
+    tp->stages = best_stages;
+    return best_kc;
+}
+
+cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches) {
+    PairParams tp;
+    const int best_kc = choose_chunk(a, &tp);
     if (!best_kc) return cudaErrorInvalidConfiguration;
     const int KC = best_kc;
-    tp.K_pad = best_pad;
-    tp.stages = best_stages;
     tp.NAh = (512 - 4 * tp.Npad) / (2 * 2 * KC);
     if (tp.NAh > 4) tp.NAh = 4;
-    // Two issuers per half wait on the same A-buffer barriers in turn; a parity wait is only
-    // sound if the waiter is at most one phase ahead, which holds when a tile's chunks plus
-    // one fit in the buffers of a half.
-    // Measured on B200 at c = 32: a second pair pays once a tile has more than 4 k-steps
-    // (decode +5 %), and costs 2 % below that (encode).
-    tp.four_issuers = (tp.NAh >= tp.K_pad / KC + 1 && (tp.K_rows + 7) / 8 > 4) ? 1 : 0;
+    // Measured on B200 at c = 32: a second pair of issuers pays once a tile has more than 4 k-steps
+    // (decode +8 .. +25 %), and costs 2 % below that (encode).
+    tp.four_issuers = ((tp.K_rows + 7) / 8 > 4) ? 1 : 0;
     if (g_tune_tc_variant == 2) tp.four_issuers = 0;
-    if (g_tune_tc_variant == 3 && tp.NAh >= tp.K_pad / KC + 1) tp.four_issuers = 1;
+    if (g_tune_tc_variant == 3) tp.four_issuers = 1;
     tp.tmem_cols = 32;
     while (tp.tmem_cols < 4 * tp.Npad + 2 * tp.NAh * 2 * KC) tp.tmem_cols *= 2;
     const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * TILE_W * 4 +
