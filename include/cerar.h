@@ -124,6 +124,17 @@ cerar_status_t cerar_plan_get_R(const cerar_plan_t* plan, int worker, double* ou
 /* Diagnostics (computed on first request: a few SVDs on the host). */
 cerar_status_t cerar_plan_info(cerar_plan_t* plan, cerar_plan_info_t* out);
 
+/* gamma(B, H) = min_{l=0..N-1} sigma_min(K^(l)(B, H)) for H = diag(h): the constant that the
+ * analysis of the epsilon-construction assumes positive (Sec. II-C, the Assumption before the
+ * theorem on singular value scaling; K^(l) = [B; BH; ..; BH^(beta-1); (BH^beta)_{E_l}] with
+ * c = beta N + s, E_l = {l, .., l+s-1} mod N).  sigma_min(A_l(eps)) = Theta(eps^r*) carries it
+ * as its constant, so among several H the one with the largest gamma is the natural pick:
+ * the paper's "multiple trials for selecting H".  Host only, no CUDA.
+ * B: N x c row-major or NULL (built-in N(0,1) generator with `seed`); h: length c or NULL
+ * (equally spaced in [-1, 1]). */
+cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, const double* h,
+                                  double* gamma_out);
+
 /* Bytes of the device workspace for gradient length d: 4 * N * (c+N) * (d/c);
  * 0 if c does not divide d. */
 size_t cerar_workspace_bytes(const cerar_plan_t* plan, int64_t d);

@@ -200,6 +200,27 @@ def singular_values_mp(A, dps: int = DEFAULT_DPS):
         return sorted([S[i] for i in range(len(S))], reverse=True)
 
 
+def k_limit(B, h, N: int, c: int, l: int) -> np.ndarray:
+    """K^(l)(B, H), H = diag(h): the eps -> 0 limit of K_l(eps) in the factorisation
+    F~_l Pi_l A_l(eps) = Lambda_l(eps) K_l(eps) (Sec. II-C).  With c = beta N + s it
+    stacks B, BH, .., BH^(beta-1) and, if s > 0, the rows E_l = {l, .., l+s-1} mod N of
+    BH^beta."""
+    B = np.asarray(B, dtype=np.float64)
+    h = np.asarray(h, dtype=np.float64)
+    beta, s = divmod(c, N)
+    blocks = [B * h ** j for j in range(beta)]
+    if s > 0:
+        E = [(l + t) % N for t in range(s)]
+        blocks.append((B * h ** beta)[E, :])
+    return np.concatenate(blocks, axis=0)
+
+
+def gamma(B, h, N: int, c: int) -> float:
+    """min over l = 0..N-1 of sigma_min(K^(l)(B, H)): the constant the analysis of the
+    epsilon-construction assumes positive (the Assumption of Sec. II-C)."""
+    return min(float(np.linalg.svd(k_limit(B, h, N, c, l), compute_uv=False)[-1]) for l in range(N))
+
+
 # ---------------------------------------------------------- kappa-constrained design
 
 def _ls_R(U, N, c):

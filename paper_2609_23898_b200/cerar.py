@@ -68,6 +68,8 @@ lib.cerar_plan_destroy.restype = None
 lib.cerar_plan_get_U.argtypes = [_vp, C.c_int, C.POINTER(C.c_double)]
 lib.cerar_plan_get_R.argtypes = [_vp, C.c_int, C.POINTER(C.c_double)]
 lib.cerar_plan_info.argtypes = [_vp, C.POINTER(PlanInfo)]
+lib.cerar_design_gamma.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.c_uint64, C.POINTER(C.c_double),
+                                   C.POINTER(C.c_double)]
 lib.cerar_workspace_bytes.argtypes = [_vp, _i64]
 lib.cerar_workspace_bytes.restype = C.c_size_t
 lib.cerar_encode.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _vp]
@@ -112,6 +114,26 @@ def _ptr(t) -> int:
     if hasattr(t, "data_ptr"):
         return t.data_ptr()
     return t.ctypes.data
+
+
+def design_gamma(N: int, c: int, B=None, h=None, seed: int = 0) -> float:
+    """cerar_design_gamma: min_l sigma_min(K^(l)(B, diag(h))) (Sec. II-C)."""
+    import numpy as np
+    Ba = None if B is None else np.ascontiguousarray(B, dtype=np.float64)
+    ha = None if h is None else np.ascontiguousarray(h, dtype=np.float64)
+    dp = C.POINTER(C.c_double)
+    out = C.c_double()
+    _check(lib.cerar_design_gamma(N, c, Ba.ctypes.data_as(dp) if Ba is not None else None, seed,
+                                  ha.ctypes.data_as(dp) if ha is not None else None, C.byref(out)))
+    return out.value
+
+
+def select_h(N: int, c: int, B, candidates):
+    """The paper's "multiple trials for selecting H": of the candidate diagonals, the one with
+    the largest gamma(B, H).  Returns (index, gammas)."""
+    gammas = [design_gamma(N, c, B, h) for h in candidates]
+    best = max(range(len(gammas)), key=lambda i: gammas[i])
+    return best, gammas
 
 
 def cerar_set_tuning(name: str, value: int) -> int:

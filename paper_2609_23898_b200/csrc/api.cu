@@ -245,6 +245,17 @@ cerar_status_t cerar_plan_info(cerar_plan_t* P, cerar_plan_info_t* out) {
     return CERAR_OK;
 }
 
+cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, const double* h, double* gamma_out) {
+    if (!gamma_out || N < 2 || c < N) return fail(CERAR_ERR_INVALID_ARG, "need 2 <= N <= c and an output pointer");
+    std::vector<double> Bdef, hdef;
+    if (!B) { Bdef = cerar::default_base_matrix(N, c, seed); B = Bdef.data(); }
+    if (!h) { hdef = cerar::default_nodes(c); h = hdef.data(); }
+    for (int i = 0; i < N * c; ++i) if (!std::isfinite(B[i])) return fail(CERAR_ERR_INVALID_ARG, "B is not finite");
+    for (int i = 0; i < c; ++i) if (!std::isfinite(h[i])) return fail(CERAR_ERR_INVALID_ARG, "h is not finite");
+    *gamma_out = cerar::k_limit_gamma(N, c, B, h);
+    return CERAR_OK;
+}
+
 size_t cerar_workspace_bytes(const cerar_plan_t* P, int64_t d) {
     if (!P || d <= 0 || d % P->host.c != 0) return 0;
     return (size_t)4 * P->host.N * (size_t)(P->host.c + P->host.N) * (size_t)(d / P->host.c);

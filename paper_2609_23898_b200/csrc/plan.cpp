@@ -1,6 +1,7 @@
 // Host-side builder of the CERAR coefficient matrices (fp64 results; extended
 // precision inside where the windows A_l are ill-conditioned by construction).
 #include "plan.hpp"
+#include <algorithm>
 
 #include <cmath>
 #include <limits>
@@ -266,6 +267,38 @@ static double phi_blocks(const HostPlan& P) {
             }
         }
     return (double)tot;
+}
+
+double k_limit_gamma(int N, int c, const double* B, const double* h) {
+    const int beta = c / N, s = c % N;
+    // rows B H^j for j = 0..beta (the last block only partly used)
+    std::vector<double> pw((size_t)(beta + 1) * N * c);
+    for (int r = 0; r < N; ++r)
+        for (int q = 0; q < c; ++q) {
+            double v = B[(size_t)r * c + q];
+            for (int j = 0; j <= beta; ++j) {
+                pw[((size_t)j * N + r) * c + q] = v;
+                v *= h[q];
+            }
+        }
+    double gamma = std::numeric_limits<double>::infinity();
+    const int windows = (s == 0) ? 1 : N;          // without the partial block every l gives the same matrix
+    for (int l = 0; l < windows; ++l) {
+        la::MatD K(c, c);
+        int row = 0;
+        for (int j = 0; j < beta; ++j)
+            for (int r = 0; r < N; ++r, ++row)
+                for (int q = 0; q < c; ++q) K(row, q) = pw[((size_t)j * N + r) * c + q];
+        for (int t = 0; t < s; ++t, ++row) {
+            const int r = (l + t) % N;
+            for (int q = 0; q < c; ++q) K(row, q) = pw[((size_t)beta * N + r) * c + q];
+        }
+        la::MatD Uo, V;
+        std::vector<double> sv;
+        la::svd_jacobi(K, Uo, sv, V);
+        gamma = std::min(gamma, sv.back());
+    }
+    return gamma;
 }
 
 double phi_direct(const HostPlan& P) { return phi_blocks<ld>(P); }

@@ -33,6 +33,11 @@ int build_epsilon(int N, int c, double eps, const double* B, const double* h, Ho
 int build_kappa(int N, int c, double kappa_max, const double* B, const double* h, double eps_init,
                 int iters, double tol, HostPlan& out, std::string& err);
 
+// gamma(B, H) = min over l = 0..N-1 of sigma_min(K^(l)(B, H)), the quantity the analysis of the
+// epsilon-construction assumes positive (Sec. II-C): K^(l) stacks B, BH, .., BH^(beta-1) and, when
+// c = beta N + s with s > 0, the rows {l, .., l+s-1} mod N of BH^beta.  H = diag(h).
+double k_limit_gamma(int N, int c, const double* B, const double* h);
+
 // Phi(U,R) from the block form sum_{i,s} ||U_{i-1-s} W_s(R_i) - I||_F^2.
 double phi_direct(const HostPlan& P);
 double kappa_U_max(const HostPlan& P);

@@ -1,0 +1,72 @@
+"""Accuracy against conditioning of the CERAR designs, on the host (no GPU needed).
+
+  python -m paper_2609_23898_b200.tradeoff [--N 4] [--c 12] [--trials 16] [--seed 0]
+
+Three tables from the library's fp64 design builder (host_only plans):
+  1. epsilon-construction (Sec. II-C) over eps: Phi = O(eps^2) against kappa_2(M_i) = O(eps^-r*);
+  2. the same eps with H chosen among `trials` random diagonals by the largest
+     gamma(B, H) = min_l sigma_min(K^(l)(B, H)) (the paper's "multiple trials for selecting H");
+  3. the condition-number-constrained design (Sec. II-D) over the bound C: the Phi it reaches
+     and the kappa_2(M_i) it ends with.
+Phi is the squared least-squares error of Eq. (F); the relative error of the decoded sum is
+about sqrt(Phi / (N c)) for i.i.d. gradients.
+"""
+from __future__ import annotations
+
+import argparse
+
+import numpy as np
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--N", type=int, default=4)
+    ap.add_argument("--c", type=int, default=12)
+    ap.add_argument("--trials", type=int, default=16)
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--als-iters", type=int, default=200)
+    args = ap.parse_args()
+    from . import cerar, inputs
+    N, c = args.N, args.c
+    B = inputs.base_matrix(N, c, args.seed)
+    r_star = -(-c // N) - 1
+    print(f"N={N} c={c} r*={r_star} rates: communication {1 + (N - 2) / c:.3f}, storage {1 + N / c:.3f}")
+
+    def row(plan):
+        i = plan.info()
+        return i["phi"], i["kappa_M_max"], i["kappa_U_max"], i["abs_U_max"]
+
+    h0 = np.linspace(-1.0, 1.0, c) if c > 1 else np.zeros(1)
+    rng = np.random.default_rng(args.seed + 1)
+    cands = [h0] + [rng.uniform(-1.0, 1.0, c) for _ in range(args.trials)]
+    cands = [h / np.abs(h).max() for h in cands]                  # ||H||_2 = 1 for all of them
+    best, gammas = cerar.select_h(N, c, B, cands)
+    print(f"gamma(B, H): default H {gammas[0]:.3e}; best of {args.trials} random diagonals {gammas[best]:.3e} "
+          f"(median {np.median(gammas[1:]):.3e})")
+    print("\n| eps | Phi | kappa_M default H | kappa_M best-gamma H | max abs U default | max abs U best |")
+    print("|---|---|---|---|---|---|")
+    for eps in (1e-1, 3e-2, 1e-2, 3e-3, 1e-3):
+        out = []
+        for h in (cands[0], cands[best]):
+            try:
+                p = cerar.Plan.create(N, c, cerar.EPSILON, eps, B=B, h=h, host_only=True)
+                out.append(row(p))
+                p.destroy()
+            except cerar.CerarError as e:
+                out.append((float("nan"),) * 4)
+        print(f"| {eps:g} | {out[0][0]:.3e} / {out[1][0]:.3e} | {out[0][1]:.3e} | {out[1][1]:.3e} | "
+              f"{out[0][3]:.2e} | {out[1][3]:.2e} |", flush=True)
+    print("\n| C (bound on kappa_M) | Phi reached | kappa_M reached | ALS iterations |")
+    print("|---|---|---|---|")
+    for C in (1e2, 1e3, 1e4, 1e5, 1e6):
+        try:
+            p = cerar.Plan.create(N, c, cerar.KAPPA, C, B=B, als_iters=args.als_iters, host_only=True)
+            i = p.info()
+            print(f"| {C:g} | {i["phi"]:.3e} | {i["kappa_M_max"]:.3e} | {i["als_iters_done"]} |", flush=True)
+            p.destroy()
+        except cerar.CerarError as e:
+            print(f"| {C:g} | - | - | {e} |", flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -263,6 +263,62 @@ def test_finite_difference_identity():
                 assert max(abs(a - b) for a, b in zip(lhs, rhs)) < mp.mpf(10) ** (-50)
 
 
+def test_k_limit_rows_are_the_limit_of_the_factorised_window():
+    """K^(l)(B, H) against the factorisation it comes from: F~ Pi A_l(eps) = Lambda K_l(eps)
+    (checked above), K_l(eps) -> K^(l) as eps -> 0 up to the order of the rows."""
+    for (N, c) in [(3, 7), (4, 10), (4, 8), (5, 5)]:
+        B = _rng_B(N, c, 21)
+        h = np.array(Dz.default_h(c))
+        for l in range(N):
+            eps = 1e-9
+            with mp.workdps(80):
+                Bm = mp.matrix(B.tolist())
+                Dv = [1 + mp.mpf(eps) * mp.mpf(x) for x in h.tolist()]
+                A = Dz.window_mp(Bm, Dv, N, c, l, 80)
+                idx = list(range(l, l + c))
+                rows_eps = []
+                for alpha in range(N):
+                    rows = [t for t, jj in enumerate(idx) if jj % N == alpha]
+                    F = Dz.finite_difference_matrix(len(rows))
+                    for j in range(len(rows)):
+                        r = [sum(int(F[j, k]) * A[rows[k], col] for k in range(j + 1)) / mp.mpf(eps) ** j
+                             for col in range(c)]
+                        rows_eps.append(np.array([float(x) for x in r]))
+            K = Dz.k_limit(B, h, N, c, l)
+            assert K.shape == (c, c)
+            # same rows, some order: match each limit row to its nearest row of K
+            used = set()
+            for r in rows_eps:
+                dist = np.abs(K - r).max(axis=1)
+                t = int(np.argmin(dist))
+                assert dist[t] < 1e-6 and t not in used
+                used.add(t)
+
+
+def test_gamma_special_case_and_lower_bound_on_sigma_min():
+    """c = N: K^(l) = B, so gamma = sigma_min(B).  And from A_l = Pi^T F~^-1 Lambda K_l:
+    sigma_min(A_l(eps)) >= eps^r* sigma_min(K_l(eps)) / ||F~||_2, with sigma_min(K_l(eps))
+    within O(eps) of sigma_min(K^(l)) >= gamma."""
+    B = _rng_B(5, 5, 3)
+    assert Dz.gamma(B, Dz.default_h(5), 5, 5) == pytest.approx(np.linalg.svd(B, compute_uv=False)[-1], rel=1e-12)
+    N, c = 4, 10
+    beta, s = divmod(c, N)
+    r_star = -(-c // N) - 1
+    B = _rng_B(N, c, 5)
+    h = Dz.default_h(c)
+    g = Dz.gamma(B, h, N, c)
+    assert g > 0
+    normF = max(np.linalg.norm(Dz.finite_difference_matrix(n).astype(float), 2) for n in (beta, beta + 1))
+    for eps in (1e-2, 1e-3):
+        for l in range(N):
+            with mp.workdps(80):
+                Dv = [1 + mp.mpf(eps) * mp.mpf(x) for x in h]
+                A = Dz.window_mp(mp.matrix(B.tolist()), Dv, N, c, l, 80)
+                smin = float(Dz.singular_values_mp(A, 80)[-1])
+            assert smin >= eps ** r_star * (g - 20 * eps) / normF
+            assert smin <= 1e3 * eps ** r_star            # and not a different power of eps
+
+
 # ------------------------------------------------------------------ kappa-constrained
 
 def test_kappa_constrained_invariants():

@@ -156,3 +156,38 @@ def test_argument_errors():
     c = pl.counters()
     assert c["rounds_done"] == 0 and c["bytes_forwarded_per_worker"] == 0
     assert cerar.lib.cerar_status_string(5) == b"call out of order"
+
+
+def test_design_gamma_matches_oracle_and_selects_the_best_h():
+    """cerar_design_gamma against the oracle's K^(l) matrices, and the "multiple trials
+    for H" helper on fixed candidates."""
+    from oracle import designs as Dz
+    from paper_2609_23898_b200 import cerar, inputs
+    rng = np.random.default_rng(9)
+    for (N, c) in [(4, 4), (4, 10), (3, 7), (8, 32), (5, 9), (4, 16)]:
+        B = inputs.base_matrix(N, c, 0)
+        cands = [np.array(Dz.default_h(c))] + [rng.uniform(-1, 1, c) for _ in range(4)]
+        for h in cands:
+            g_lib = cerar.design_gamma(N, c, B, h)
+            g_ora = Dz.gamma(B, h, N, c)
+            assert g_lib == pytest.approx(g_ora, rel=1e-8, abs=1e-14)
+        best, gammas = cerar.select_h(N, c, B, cands)
+        assert gammas[best] == max(gammas)
+        assert best == int(np.argmax([Dz.gamma(B, h, N, c) for h in cands]))
+    # h = NULL means the equally spaced default; B = NULL the built-in generator (seeded)
+    B = inputs.base_matrix(4, 10, 0)
+    assert cerar.design_gamma(4, 10, B) == pytest.approx(Dz.gamma(B, Dz.default_h(10), 4, 10), rel=1e-8)
+    assert cerar.design_gamma(4, 10, seed=1) > 0 and cerar.design_gamma(4, 10, seed=1) != cerar.design_gamma(4, 10, seed=2)
+    with pytest.raises(cerar.CerarError):
+        cerar.design_gamma(4, 3)
+
+
+def test_tradeoff_report_runs_on_the_host(capsys, monkeypatch):
+    import sys as _sys
+    from paper_2609_23898_b200 import tradeoff
+    monkeypatch.setattr(_sys, "argv", ["tradeoff", "--N", "3", "--c", "7", "--trials", "3", "--als-iters", "5"])
+    tradeoff.main()
+    out = capsys.readouterr().out
+    assert "gamma(B, H)" in out and out.count("\n|---|") == 2
+    rows = [ln for ln in out.splitlines() if ln.startswith("| 0.001 |")]
+    assert len(rows) == 1 and "nan" not in rows[0]
