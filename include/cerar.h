@@ -244,6 +244,38 @@ cerar_status_t cerar_rank_round(cerar_plan_t* plan, int rank, const float* ws, f
 cerar_status_t cerar_rank_decode(cerar_plan_t* plan, int rank, const float* ws, float* out, int64_t d,
                                  float scale, cerar_stream_t stream);
 
+/* All L rounds in one launch per worker, ordered tile by tile instead of round by round.
+ * The positions are cut into tiles of CERAR_RING_TILE; per tile a worker keeps two 32-bit
+ * counters in its OWN memory that its neighbours write: `landed` (the previous worker has
+ * stored message k of that tile here: value epoch (L+1) + k) and `freed` (the next worker
+ * has finished round k on that tile, so the slot that message k+1 overwrites may be
+ * written).  The kernel polls its local counters, stores messages and counters into the
+ * neighbours' memory with system-scope release, and returns when message L has landed
+ * too; there is no barrier between rounds.  Every wait is bounded (2 s): on expiry the
+ * launch ends and cerar_device_status reports CERAR_ERR_TIMEOUT.
+ *   counters must be zero before the first use and `epoch` must grow by one with every
+ *   aggregation on the same buffers (nothing is reset in between).  Encode before and
+ *   decode after are cerar_rank_encode / cerar_rank_decode; across aggregations the
+ *   caller still orders "all decodes done" before "next encode" (stream order or one
+ *   barrier per aggregation).
+ * cerar_rank_rounds_fused: one worker (this GPU's); landed_local / freed_local: this
+ *   worker's counters (cerar_ring_tiles(plan, d) each); landed_next: the NEXT worker's
+ *   landed counters, freed_prev: the PREVIOUS worker's freed counters (peer-mapped).  All
+ *   N workers' kernels must be running at the same time on N GPUs; never launch several
+ *   of them on one GPU.
+ * cerar_ring_rounds_fused_local: all N workers of the plan on THIS GPU in one cooperative
+ *   launch (N <= 32): ws = host array of the N workspace pointers, counters = device array
+ *   of 2 N cerar_ring_tiles(plan, d) words.  This is the form that can be run and checked
+ *   on a single GPU. */
+#define CERAR_RING_TILE 8192
+int64_t        cerar_ring_tiles(const cerar_plan_t* plan, int64_t d);
+cerar_status_t cerar_rank_rounds_fused(cerar_plan_t* plan, int rank, const float* ws, float* peer_ws,
+                                       const unsigned* landed_local, const unsigned* freed_local,
+                                       unsigned* landed_next, unsigned* freed_prev, int64_t d, unsigned epoch,
+                                       cerar_stream_t stream);
+cerar_status_t cerar_ring_rounds_fused_local(cerar_plan_t* plan, float* const* ws, unsigned* counters, int64_t d,
+                                             unsigned epoch, cerar_stream_t stream);
+
 /* The same pipeline as cerar_allreduce_sim for callers that cannot provide a
  * workspace because they cannot allocate device memory at this point: for
  * instance a host program whose framework has already claimed all free memory
@@ -301,7 +333,8 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  * or 16), "slabs" (position slabs per CTA), "tc_kc" / "tc_stages" (rows per stage and
  * stages of the tensor-core kernel), "tc_variant" (1 = always tiles of 128 positions;
  * by default c <= 64 runs on tiles of 256 positions;
- * 2 / 3 = tiles of 256 wherever they fit, with one / two MMA issuers per half); value 0 restores the default.
+ * 2 / 3 = tiles of 256 wherever they fit, with one / two MMA issuers per half), "ring_wait_ms"
+ * (limit of the waits of the fused ring rounds, default 2000); value 0 restores the default.
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

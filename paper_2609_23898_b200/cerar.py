@@ -86,6 +86,10 @@ lib.cerar_rank_round_slots.argtypes = [_vp, C.c_int] + [C.POINTER(C.c_int)] * 4
 lib.cerar_rank_encode.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, _vp]
 lib.cerar_rank_round.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, C.c_int, _vp]
 lib.cerar_rank_decode.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, C.c_float, _vp]
+lib.cerar_ring_tiles.argtypes = [_vp, _i64]
+lib.cerar_ring_tiles.restype = _i64
+lib.cerar_rank_rounds_fused.argtypes = [_vp, C.c_int, _f32p, _f32p, _vp, _vp, _vp, _vp, _i64, C.c_uint, _vp]
+lib.cerar_ring_rounds_fused_local.argtypes = [_vp, C.POINTER(C.c_void_p), _vp, _i64, C.c_uint, _vp]
 lib.cerar_get_counters.argtypes = [_vp, C.POINTER(Counters)]
 lib.cerar_launch_count.argtypes = [_vp]
 lib.cerar_launch_count.restype = C.c_uint64
@@ -257,6 +261,18 @@ class Plan:
 
     def rank_round(self, rank, ws, peer_ws, d, k, stream=0):
         _check(lib.cerar_rank_round(self._h, rank, _ptr(ws), _ptr(peer_ws), d, k, stream))
+
+    def ring_tiles(self, d: int) -> int:
+        return int(lib.cerar_ring_tiles(self._h, d))
+
+    def rank_rounds_fused(self, rank, ws, peer_ws, landed_local, freed_local, landed_next, freed_prev, d, epoch,
+                          stream=0):
+        _check(lib.cerar_rank_rounds_fused(self._h, rank, _ptr(ws), _ptr(peer_ws), _ptr(landed_local),
+                                           _ptr(freed_local), _ptr(landed_next), _ptr(freed_prev), d, epoch, stream))
+
+    def ring_rounds_fused_local(self, ws_list, counters, d, epoch, stream=0):
+        arr = (C.c_void_p * len(ws_list))(*[_ptr(w) for w in ws_list])
+        _check(lib.cerar_ring_rounds_fused_local(self._h, arr, _ptr(counters), d, epoch, stream))
 
     def rank_decode(self, rank, ws, out, d, scale=1.0, stream=0):
         _check(lib.cerar_rank_decode(self._h, rank, _ptr(ws), _ptr(out), d, scale, stream))

@@ -458,6 +458,91 @@ cerar_status_t cerar_rank_decode(cerar_plan_t* P, int rank, const float* ws, flo
     return CERAR_OK;
 }
 
+namespace {
+// Positions per tile of the fused rounds: small enough that a short job still has a few tiles
+// per resident block, large enough that polling and publishing two counters per tile and round
+// stays a few per cent of the tile's memory time.
+int64_t ring_tile_positions(int64_t p) {
+    if (cerar::g_tune_ring_tile > 0) return (int64_t)cerar::g_tune_ring_tile;
+    return p >= ((int64_t)1 << 23) ? 4 * CERAR_RING_TILE : CERAR_RING_TILE;
+}
+}  // namespace
+
+int64_t cerar_ring_tiles(const cerar_plan_t* P, int64_t d) {
+    if (!P || d <= 0 || d % P->host.c != 0) return 0;
+    const int64_t p = d / P->host.c;
+    const int64_t tile = ring_tile_positions(p);
+    return (p + tile - 1) / tile;
+}
+
+namespace {
+cerar_status_t ring_fused_common(cerar_plan_t* P, int64_t d, int64_t* p_out) {
+    cerar_status_t st = check_data_call(P, d, p_out);
+    if (st != CERAR_OK) return st;
+    if (P->host.N > cerar::RING_MAX_WORKERS) return fail(CERAR_ERR_INVALID_ARG, "more workers than one launch can serve");
+    return CERAR_OK;
+}
+void ring_fused_fill(cerar::RingFusedArgs& a, const cerar_plan_t* P, int64_t p, unsigned epoch) {
+    a.N = P->host.N; a.c = P->host.c; a.p = p;
+    a.tile = ring_tile_positions(p); a.ntiles = (p + a.tile - 1) / a.tile;
+    a.base = epoch * (unsigned)(P->host.L + 1);
+    a.status = P->d_status;
+    a.limit_ns = (unsigned long long)(cerar::g_tune_ring_wait_ms > 0 ? cerar::g_tune_ring_wait_ms : 2000) * 1000000ull;
+}
+}  // namespace
+
+cerar_status_t cerar_ring_rounds_fused_local(cerar_plan_t* P, float* const* ws, unsigned* counters, int64_t d,
+                                             unsigned epoch, cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = ring_fused_common(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !counters) return fail(CERAR_ERR_INVALID_ARG, "ws or counters is NULL");
+    const int N = P->host.N;
+    cerar::RingFusedArgs a{};
+    ring_fused_fill(a, P, p, epoch);
+    bool vec = (p % 4 == 0);
+    for (int i = 0; i < N; ++i) {
+        if (!ws[i]) return fail(CERAR_ERR_INVALID_ARG, "a workspace pointer is NULL");
+        for (int j = 0; j < i; ++j) if (ws[i] == ws[j]) return fail(CERAR_ERR_INVALID_ARG, "two workers share a workspace");
+        vec = vec && ((reinterpret_cast<uintptr_t>(ws[i]) & 15u) == 0);
+    }
+    a.vec = vec ? 1 : 0;
+    for (int i = 0; i < N; ++i) {
+        const int nx = (i + 1) % N, pv = (i + N - 1) % N;
+        a.ws[i] = ws[i]; a.peer_ws[i] = ws[nx];
+        a.landed_local[i] = counters + (size_t)(2 * i) * a.ntiles;
+        a.freed_local[i] = counters + (size_t)(2 * i + 1) * a.ntiles;
+        a.landed_next[i] = counters + (size_t)(2 * nx) * a.ntiles;
+        a.freed_prev[i] = counters + (size_t)(2 * pv + 1) * a.ntiles;
+    }
+    cudaError_t e = cerar::launch_ring_rounds(a, N, true, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "fused ring rounds launch");
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_rank_rounds_fused(cerar_plan_t* P, int rank, const float* ws, float* peer_ws,
+                                       const unsigned* landed_local, const unsigned* freed_local,
+                                       unsigned* landed_next, unsigned* freed_prev, int64_t d, unsigned epoch,
+                                       cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = ring_fused_common(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !peer_ws || !landed_local || !freed_local || !landed_next || !freed_prev)
+        return fail(CERAR_ERR_INVALID_ARG, "NULL buffer");
+    if (ws == peer_ws) return fail(CERAR_ERR_INVALID_ARG, "peer_ws must be the next worker's workspace, not this one's");
+    if (rank < 0 || rank >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    cerar::RingFusedArgs a{};
+    ring_fused_fill(a, P, p, epoch);
+    a.vec = ((p % 4 == 0) && ((reinterpret_cast<uintptr_t>(ws) & 15u) == 0) &&
+             ((reinterpret_cast<uintptr_t>(peer_ws) & 15u) == 0)) ? 1 : 0;
+    a.ws[0] = ws; a.peer_ws[0] = peer_ws;
+    a.landed_local[0] = landed_local; a.freed_local[0] = freed_local;
+    a.landed_next[0] = landed_next; a.freed_prev[0] = freed_prev;
+    cudaError_t e = cerar::launch_ring_rounds(a, 1, false, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "fused rank rounds launch");
+    return CERAR_OK;
+}
+
 cerar_status_t cerar_allreduce_fused(cerar_plan_t* P, const float* grads, int64_t grads_stride, float* out,
                                      int64_t out_stride, int64_t d, float scale, cerar_stream_t stream) {
     int64_t p;
@@ -538,6 +623,8 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "tc_kc") cerar::g_tune_tc_kc = value;
     else if (n == "tc_stages") cerar::g_tune_tc_stages = value;
     else if (n == "tc_variant") cerar::g_tune_tc_variant = value;
+    else if (n == "ring_wait_ms") cerar::g_tune_ring_wait_ms = value;
+    else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;
 }

@@ -44,6 +44,24 @@ struct RankRoundArgs {
     int slot_prev, slot_cancel, slot_add, slot_land;   // filled in by the launcher (-1 = term absent)
 };
 
+// All L rounds of up to RING_MAX_WORKERS workers in one launch (blockIdx.y = index into the arrays).
+constexpr int RING_MAX_WORKERS = 32;
+struct RingFusedArgs {
+    const float* ws[RING_MAX_WORKERS];            // the worker's own workspace ((c+N+1) x p)
+    float* peer_ws[RING_MAX_WORKERS];             // the next worker's workspace (may be peer memory)
+    const unsigned* landed_local[RING_MAX_WORKERS];   // per tile: last message that has landed here
+    const unsigned* freed_local[RING_MAX_WORKERS];    // per tile: last round the next worker has finished
+    unsigned* landed_next[RING_MAX_WORKERS];      // the next worker's landed counters (written here)
+    unsigned* freed_prev[RING_MAX_WORKERS];       // the previous worker's freed counters (written here)
+    int N, c;
+    int64_t p;
+    int64_t tile, ntiles;                          // positions per tile (a multiple of 4), tiles per worker
+    unsigned base;                                 // counters of this aggregation are base + k
+    int vec;                                       // 1: p % 4 == 0 and 16-byte aligned workspaces
+    int* status;
+    unsigned long long limit_ns;
+};
+
 enum { KERNEL_AUTO = 0, KERNEL_REF = 1, KERNEL_STAGED = 2, KERNEL_TC = 3 };
 
 // Returns cudaSuccess or the launch error.  *launches is incremented by the
@@ -56,12 +74,16 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
 bool tc_pair_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
-extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant;
+extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant,
+           g_tune_ring_wait_ms, g_tune_ring_tile;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
 // Slots of the per-worker layout that round k reads (-1 = term absent) and the landing slot
 // in the neighbour's workspace; the one definition that launcher and callers share.
 void rank_round_slots(int N, int c, int k, int* slot_prev, int* slot_cancel, int* slot_add, int* slot_land);
 cudaError_t launch_rank_round(RankRoundArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
+// cooperative = true when the launch serves workers that wait on one another (all on this GPU).
+cudaError_t launch_ring_rounds(const RingFusedArgs& a, int nworkers, bool cooperative, int num_sms, cudaStream_t s,
+                               uint64_t* launches);
 // A kernel whose bounded wait is made to run out (nothing arrives on its barrier).
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, cudaStream_t s);
 // Whole protocol in one launch with the slots in shared memory (small N (c+N) only).

@@ -11,8 +11,10 @@ LocalRing         all N workers in this process on one GPU, each with its own
                   what the GPU tests and the single-GPU measurements run.
 DistributedRing   one worker per process and GPU (torch.distributed, NCCL): the
                   workspace lives in symmetric memory, the neighbour's copy is a
-                  peer-mapped tensor, and a device-side barrier on the stream
-                  separates the rounds.  Needs N GPUs with peer access.
+                  peer-mapped tensor, and either a device-side barrier on the stream
+                  separates the rounds or (fused=True) one kernel runs all rounds
+                  and orders itself against the neighbours tile by tile through
+                  counters in symmetric memory.  Needs N GPUs with peer access.
 """
 from __future__ import annotations
 
@@ -39,6 +41,9 @@ class LocalRing:
         self.N, self.c, self.L = plan.N, plan.c, plan.L
         n = plan.rank_workspace_bytes(d) // 4
         self.ws = [torch.empty(n, dtype=torch.float32, device=device) for _ in range(self.N)]
+        # tile counters of the fused rounds: [worker][landed | freed][tile], zero once, never reset
+        self.counters = torch.zeros(2 * self.N * plan.ring_tiles(d), dtype=torch.int32, device=device)
+        self.epoch = 0
 
     def grad_view(self, i):
         """The D rows of worker i's workspace as a length-d tensor (in-place use)."""
@@ -54,14 +59,22 @@ class LocalRing:
         for i in range(self.N):
             self.plan.rank_round(i, self.ws[i], self.ws[(i + 1) % self.N], self.d, k, stream)
 
+    def rounds_fused(self, stream=0):
+        """All L rounds of all N workers in one cooperative launch, ordered per tile by counters."""
+        self.plan.ring_rounds_fused_local(self.ws, self.counters, self.d, self.epoch, stream)
+        self.epoch += 1
+
     def decode(self, outs, scale=1.0, stream=0):
         for i in range(self.N):
             self.plan.rank_decode(i, self.ws[i], outs[i], self.d, scale, stream)
 
-    def allreduce(self, grads, outs, scale=1.0, stream=0):
+    def allreduce(self, grads, outs, scale=1.0, stream=0, fused=False):
         self.encode(grads, stream)
-        for k in range(1, self.L + 1):
-            self.round(k, stream)
+        if fused:
+            self.rounds_fused(stream)
+        else:
+            for k in range(1, self.L + 1):
+                self.round(k, stream)
         self.decode(outs, scale, stream)
 
 
@@ -86,17 +99,37 @@ class DistributedRing:
         self._hdl = symm_mem.rendezvous(self.ws, group)
         self.peer_ws = self._hdl.get_buffer((self.rank + 1) % self.N, (n,), torch.float32)
         self.barrier_timeout_ms = 10000
+        # tile counters of the fused rounds, [landed | freed][tile], in symmetric memory as well
+        nt = plan.ring_tiles(d)
+        self.counters = symm_mem.empty(2 * nt, dtype=torch.int32, device=self.ws.device)
+        self.counters.zero_()
+        self._chdl = symm_mem.rendezvous(self.counters, group)
+        nxt, prv = (self.rank + 1) % self.N, (self.rank - 1) % self.N
+        self._landed_next = self._chdl.get_buffer(nxt, (nt,), torch.int32, 0)
+        self._freed_prev = self._chdl.get_buffer(prv, (nt,), torch.int32, nt)
+        self._nt = nt
+        self.epoch = 0
 
     def _barrier(self):
         # on the current stream: all kernels of the round before, on every rank, are
         # complete and visible before anything after it starts
         self._hdl.barrier(channel=0, timeout_ms=self.barrier_timeout_ms)
 
-    def allreduce(self, grad, out, scale=1.0, stream=0):
-        """grad, out: this rank's length-d device tensors; `stream` must be torch's current stream."""
+    def allreduce(self, grad, out, scale=1.0, stream=0, fused=False):
+        """grad, out: this rank's length-d device tensors; `stream` must be torch's current stream.
+        fused=True: one kernel for all rounds, ordered against the neighbours per tile by counters
+        in symmetric memory, instead of one kernel and one barrier per round."""
         self._barrier()                      # the neighbours are done reading the previous call's slots
         self.plan.rank_encode(self.rank, grad, self.ws, self.d, stream)
-        for k in range(1, self.L + 1):
-            self.plan.rank_round(self.rank, self.ws, self.peer_ws, self.d, k, stream)
-            self._barrier()
+        if fused:
+            # no further barrier: a message only ever lands in a slot whose owner has either not used
+            # it yet in this aggregation (slots 0..N) or has reported its last read of it (`freed`)
+            self.plan.rank_rounds_fused(self.rank, self.ws, self.peer_ws, self.counters,
+                                        self.counters[self._nt:], self._landed_next, self._freed_prev,
+                                        self.d, self.epoch, stream)
+            self.epoch += 1
+        else:
+            for k in range(1, self.L + 1):
+                self.plan.rank_round(self.rank, self.ws, self.peer_ws, self.d, k, stream)
+                self._barrier()
         self.plan.rank_decode(self.rank, self.ws, out, self.d, scale, stream)

@@ -166,8 +166,9 @@ def ring_table(args, exps, peak, free, stream):
     """The rank-level calls on one GPU: same algorithmic bytes, N launches per step instead of one."""
     import torch
     from . import cerar, inputs, ring
-    print("| N | c | d | pipeline ms | rank-level ms | rank-level GB/s | frac of measured HBM | launches |")
-    print("|---|---|---|---|---|---|---|---|")
+    print("| N | c | d | pipeline ms | rank-level ms (launches) | rank-level GB/s | frac | fused-rounds ms (launches) | "
+          "fused GB/s | frac |")
+    print("|---|---|---|---|---|---|---|---|---|---|")
     for (N, c) in ((4, 16), (8, 32), (8, 64)):
         rng = np.random.default_rng(0)
         L = c + N - 2
@@ -196,10 +197,12 @@ def ring_table(args, exps, peak, free, stream):
                 return float(np.median(ts))
             t_pipe = med(lambda: plan.allreduce_sim(g, d, out, d, ws, d, 1.0 / N, stream))
             t_ring = med(lambda: r.allreduce(grads, outs, 1.0 / N, stream))
+            t_fus = med(lambda: r.allreduce(grads, outs, 1.0 / N, stream, fused=True))
             plan.device_status(stream)
             ab = 4 * N * p * (8 * c + 3 * N - 8)
-            print(f"| {N} | {c} | 2^{e} | {t_pipe:.3f} | {t_ring:.3f} | {ab / t_ring / 1e6:.0f} | "
-                  f"{ab / t_ring / 1e6 / peak:.2f} | {N * (L + 2)} |", flush=True)
+            print(f"| {N} | {c} | 2^{e} | {t_pipe:.3f} | {t_ring:.3f} ({N * (L + 2)}) | {ab / t_ring / 1e6:.0f} | "
+                  f"{ab / t_ring / 1e6 / peak:.2f} | {t_fus:.3f} ({2 * N + 1}) | {ab / t_fus / 1e6:.0f} | "
+                  f"{ab / t_fus / 1e6 / peak:.2f} |", flush=True)
             del g, out, ws, r, grads, outs
             torch.cuda.empty_cache()
         plan.destroy()

@@ -102,3 +102,81 @@ def test_one_call_form_and_argument_checks(mods):
     with pytest.raises(cerar.CerarError):
         plan.rank_decode(0, r.ws[0], outs[0], d + 1, 1.0, s)
     assert plan.rank_workspace_bytes(d) == 4 * (c + N + 1) * p
+
+
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192 * 3 + 260), (8, 32, 8192 * 5 + 4), (2, 2, 8192 + 8), (3, 5, 20001),
+                                   (16, 16, 8192 * 2), (5, 9, 7)])
+def test_fused_rounds_one_launch_equals_round_by_round(mods, N, c, p):
+    """All L rounds of all workers in one cooperative launch, ordered per tile by counters:
+    same slots bit for bit as one launch per worker and round; several aggregations on the
+    same counters (the epoch moves on, nothing is reset)."""
+    import torch
+    cerar, inputs, ring = mods
+    d = c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(3 * N + c))
+    plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+    s = torch.cuda.current_stream().cuda_stream
+    ra, rb = ring.LocalRing(plan, d), ring.LocalRing(plan, d)
+    assert plan.ring_tiles(d) == -(-p // 8192)
+    rows = c + N + 1
+    ys = ring.y_slots(plan)
+    for rep in range(3):
+        g = inputs.gradients_numpy(N, d, "normal", seed=20 + rep)
+        grads = [torch.from_numpy(g[i]).cuda() for i in range(N)]
+        for r in (ra, rb):
+            r.encode(grads, s)
+        for k in range(1, plan.L + 1):
+            ra.round(k, s)
+        rb.rounds_fused(s)
+        torch.cuda.synchronize()
+        plan.device_status(s)
+        for i in range(N):
+            a = ra.ws[i].view(rows, p)[ys]
+            b = rb.ws[i].view(rows, p)[ys]
+            assert torch.equal(a, b), (rep, i)
+    # and the whole aggregation through the fused form against the oracle
+    ora = run_oracle(des.U, des.R, g, 0.5)
+    outs = [torch.empty(d, device="cuda") for _ in range(N)]
+    rb.allreduce(grads, outs, 0.5, s, fused=True)
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    assert max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
+
+
+def test_fused_rounds_give_up_when_a_neighbour_never_answers(mods):
+    """One worker's kernel alone: nobody moves its counters, so round 2 cannot start.  The
+    waits run out after the (shortened) limit, the status word says so, nothing hangs and
+    the device keeps working."""
+    import time
+    import torch
+    cerar, inputs, ring = mods
+    N, c, p = 4, 8, 8192 * 4
+    d = c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(1))
+    plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+    s = torch.cuda.current_stream().cuda_stream
+    n = plan.rank_workspace_bytes(d) // 4
+    ws, peer = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+    nt = plan.ring_tiles(d)
+    mine, nxt, prv = (torch.zeros(2 * nt, dtype=torch.int32, device="cuda") for _ in range(3))
+    assert cerar.cerar_set_tuning("ring_wait_ms", 50) == 0
+    try:
+        t0 = time.time()
+        plan.rank_rounds_fused(1, ws, peer, mine, mine[nt:], nxt, prv[nt:], d, 0, s)
+        with pytest.raises(cerar.CerarError) as e:
+            plan.device_status(s)
+        assert e.value.status == 8                      # CERAR_ERR_TIMEOUT
+        assert time.time() - t0 < 10.0
+    finally:
+        cerar.cerar_set_tuning("ring_wait_ms", 0)
+    assert int(nxt[:nt].min()) == 1 and int(prv[nt:].min()) == 1      # round 1 was done and published
+    plan.device_status(s)
+    r = ring.LocalRing(plan, d)
+    g = inputs.gradients_numpy(N, d, "normal", seed=1)
+    grads = [torch.from_numpy(g[i]).cuda() for i in range(N)]
+    outs = [torch.empty(d, device="cuda") for _ in range(N)]
+    r.allreduce(grads, outs, 1.0, s, fused=True)
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    ora = run_oracle(des.U, des.R, g, 1.0)
+    assert max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
