@@ -1,7 +1,7 @@
 """Mutation check of the oracle pins (run by hand: python tests/oracle_mutation_check.py).
 Applies one plausible mistake at a time to the oracle source (restored afterwards),
 runs the CPU oracle tests and expects at least one of them to fail: a mutation that
-survives means a pin is missing.  20 of 20 mutations are killed."""
+survives means a pin is missing.  24 of 24 mutations are killed."""
 import subprocess, shutil, sys, os
 ROOT=os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 muts=[
@@ -25,6 +25,10 @@ muts=[
  ('oracle/designs.py','F[j, k] = (-1) ** (j - k) * comb(j, k)','F[j, k] = (-1) ** (j + k + 1) * comb(j, k)'),
  ('oracle/designs.py','(i - 1 - k) % N, c) for i in range(N)], axis=1)','(i - k) % N, c) for i in range(N)], axis=1)'),
  ('oracle/designs.py','b0 = a0 * kappa_max / np.sqrt(N)','b0 = a0 * kappa_max'),
+ ('oracle/designs.py','blocks = [B * h ** j for j in range(beta)]','blocks = [B * h ** (j + 1) for j in range(beta)]'),
+ ('oracle/designs.py','E = [(l + t) % N for t in range(s)]','E = [(l - t) % N for t in range(s)]'),
+ ('oracle/designs.py','blocks.append((B * h ** beta)[E, :])','blocks.append((B * h ** (beta - 1))[E, :])'),
+ ('oracle/designs.py','compute_uv=False)[-1]) for l in range(N))','compute_uv=False)[0]) for l in range(N))'),
 ]
 def main():
     survived=[]
