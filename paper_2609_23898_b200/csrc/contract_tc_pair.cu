@@ -125,26 +125,9 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
         const int64_t t_begin = (w == w_first) ? g_begin - (int64_t)w * T : 0;
         const int64_t t_end = (w == w_last) ? g_end - (int64_t)w * T : T;
         {
-            // coefficients of this worker, split into tf32 hi / lo, in the only layout the tensor
-            // core takes for an MN-major 32-bit operand (128-byte swizzle, 32-byte atoms):
-            // block nb (32 outputs) | row k (128 B) | 32-byte chunk ^ (k & 3)
-            const float* cf = a.coef + (size_t)w * a.K * a.J;
-            uint32_t* bhi = reinterpret_cast<uint32_t*>(smem_al);
-            uint32_t* blo = reinterpret_cast<uint32_t*>(smem_al + b_bytes);
-            for (int idx = threadIdx.x; idx < K_pad * Npad; idx += blockDim.x) {
-                const int k = idx / Npad, j = idx - k * Npad;
-                // physical input row k -> coefficient row (skipped rows are not part of Y: zero)
-                int src = -1;
-                if (k < a.skip_row) src = k; else if (k >= a.skip_row + a.skip_count) src = k - a.skip_count;
-                float v = 0.f;
-                if (src >= 0 && src < a.K && j < a.J) v = cf[(size_t)src * a.J + j];
-                const uint32_t hi = tf32_bits(v);
-                const uint32_t lo = tf32_bits(v - __uint_as_float(hi));
-                const int nb = j >> 5, jj = j & 31;
-                const int off = nb * (K_pad * 32) + k * 32 + ((((jj >> 3) ^ (k & 3)) << 3) | (jj & 7));
-                bhi[off] = hi;
-                blo[off] = lo;
-            }
+            // coefficients of this worker as the tensor core's B operand (tf32 hi and lo copies)
+            split_coefficients(a, w, K_pad, Npad, reinterpret_cast<uint32_t*>(smem_al),
+                               reinterpret_cast<uint32_t*>(smem_al + b_bytes));
             fence_proxy_async_smem();
         }
         __syncthreads();

@@ -5,6 +5,7 @@
 
 #include <cstdint>
 
+#include "kernels.cuh"
 #include "ptx.cuh"
 
 namespace cerar {
@@ -109,6 +110,29 @@ __device__ __forceinline__ void tc_dealloc(uint32_t base, uint32_t cols) {
 // instruction descriptor: D = f32, A = B = tf32, A from TMEM (K-major), B MN-major, N = n, M = 128
 __device__ __forceinline__ uint32_t idesc_tf32_ts(uint32_t n) {
     return (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+// Worker w's K x J coefficient matrix, split into tf32 hi / lo copies, in the only layout the
+// tensor core takes for an MN-major 32-bit B operand (128-byte swizzle with 32-byte atoms):
+// block nb (32 outputs) | row k (128 B) | 32-byte chunk ^ (k & 3).  Physical input rows that are
+// not part of the contraction (a.skip_row ..) and the padding up to K_pad x Npad are zero.
+// All threads of the CTA take part; the caller fences (async proxy) and synchronises.
+__device__ __forceinline__ void split_coefficients(const ContractArgs& a, int w, int K_pad, int Npad, uint32_t* bhi,
+                                                   uint32_t* blo) {
+    const float* cf = a.coef + (size_t)w * a.K * a.J;
+    for (int idx = threadIdx.x; idx < K_pad * Npad; idx += blockDim.x) {
+        const int k = idx / Npad, j = idx - k * Npad;
+        int src = -1;                      // physical input row k -> coefficient row
+        if (k < a.skip_row) src = k; else if (k >= a.skip_row + a.skip_count) src = k - a.skip_count;
+        float v = 0.f;
+        if (src >= 0 && src < a.K && j < a.J) v = cf[(size_t)src * a.J + j];
+        const uint32_t hi = tf32_bits(v);
+        const uint32_t lo = tf32_bits(v - __uint_as_float(hi));
+        const int nb = j >> 5, jj = j & 31;
+        const int off = nb * (K_pad * 32) + k * 32 + ((((jj >> 3) ^ (k & 3)) << 3) | (jj & 7));
+        bhi[off] = hi;
+        blo[off] = lo;
+    }
 }
 
 // ---- host side: tensor maps over [N workers][rows][p positions] fp32 arrays
