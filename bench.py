@@ -144,7 +144,7 @@ def oracle_step(des, g_sub, scale):
     return P.allreduce([x for x in g_sub], des.U, des.R, scale)
 
 
-def cpu_baseline(cfg, des, p_sample, seed=0):
+def cpu_baseline(cfg, des, p_sample, seed=0, one_thread=False):
     """Times the oracle, as it stands, on the first p_sample positions of the
     workload (all N workers, all c chunks)."""
     from paper_2609_23898_b200 import inputs
@@ -160,9 +160,24 @@ def cpu_baseline(cfg, des, p_sample, seed=0):
         thr = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     except Exception:
         thr = os.cpu_count() or 1
-    return {"value": ab / dt / 1e9, "unit": UNIT, "cores": int(thr), "kind": "oracle",
-            "sample": f"first {p_sample} of p={cfg['d'] // c} positions, all {N} workers and {c} chunks; "
-                      f"{dt:.2f} s of numpy fp64", "seconds": dt}
+    res = {"value": ab / dt / 1e9, "unit": UNIT, "cores": int(thr), "kind": "oracle",
+           "sample": f"first {p_sample} of p={cfg['d'] // c} positions, all {N} workers and {c} chunks; "
+                     f"{dt:.2f} s of numpy fp64", "seconds": dt}
+    if one_thread:
+        # the same oracle held to one BLAS thread, on an eighth of the sample
+        try:
+            from threadpoolctl import threadpool_limits
+            p1 = max(1, p_sample // 8)
+            g1 = inputs.gradients_numpy(N, c * p1, cfg["workload"], seed=seed, **kw).astype(np.float64)
+            with threadpool_limits(limits=1):
+                t0 = time.perf_counter()
+                oracle_step(des, g1, 1.0 / N)
+                dt1 = time.perf_counter() - t0
+            res["value_1_thread"] = algorithmic_bytes(N, c, p1)["total"] / dt1 / 1e9
+            res["sample_1_thread"] = f"first {p1} positions, {dt1:.2f} s"
+        except Exception:
+            pass
+    return res
 
 
 def run_reference(args, cfg):
@@ -321,6 +336,7 @@ def main():
         traffic = NCU_ROUND_TRAFFIC_OVER_ALGORITHMIC * dom_bytes
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                "frac_of_nominal_8TBps": achieved / 8000.0, "whole_path_frac_of_nominal_8TBps": value / world / 8000.0,
                 "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": dom_ms,
                 "per_kernel": {
                     "encode": {"ms": enc_ms, "GBps": ab["encode"] / enc_ms / 1e6, "launches_per_step": 1},
@@ -387,7 +403,7 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         if des is None:
             des = build_design_oracle(cfg, B)
-        line["cpu_baseline"] = cpu_baseline(cfg, des, min(p, args.ref_positions))
+        line["cpu_baseline"] = cpu_baseline(cfg, des, min(p, args.ref_positions), one_thread=True)
 
     if rank == 0:
         print(json.dumps(line))
