@@ -144,7 +144,7 @@ def test_fused_rounds_one_launch_equals_round_by_round(mods, N, c, p):
 
 
 def test_fused_rounds_give_up_when_a_neighbour_never_answers(mods):
-    """One worker's kernel alone: nobody moves its counters, so round 2 cannot start.  The
+    """One worker's kernel alone: nobody moves its counters, so ring round k = 2 cannot start.  The
     waits run out after the (shortened) limit, the status word says so, nothing hangs and
     the device keeps working."""
     import time
@@ -169,7 +169,7 @@ def test_fused_rounds_give_up_when_a_neighbour_never_answers(mods):
         assert time.time() - t0 < 10.0
     finally:
         cerar.cerar_set_tuning("ring_wait_ms", 0)
-    assert int(nxt[:nt].min()) == 1 and int(prv[nt:].min()) == 1      # round 1 was done and published
+    assert int(nxt[:nt].min()) == 1 and int(prv[nt:].min()) == 1      # ring round k = 1 was done and published
     plan.device_status(s)
     r = ring.LocalRing(plan, d)
     g = inputs.gradients_numpy(N, d, "normal", seed=1)
