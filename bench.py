@@ -357,6 +357,22 @@ def main():
                        "buffers": "out of place: grads, workspace and output are separate device buffers"},
             "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks}
 
+    # ---- the same K aggregations through the one-call entry point, one event pair around all of
+    # them: no event between the launches, so consecutive kernels overlap their launch with the
+    # previous kernel's tail (what a caller of cerar_allreduce_sim gets; matters below ~1 ms)
+    sync_all()
+    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    o0.record()
+    for _ in range(K):
+        plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
+    o1.record()
+    sync_all()
+    plan.device_status(stream)
+    ms_one = max_over_ranks(o0.elapsed_time(o1), world, dev) / K
+    line["one_call"] = {"ms_per_step": ms_one, "value": whole_job_value(ab["total"], world, ms_one), "unit": UNIT,
+                        "frac": whole_job_value(ab["total"], world, ms_one) / world / peak,
+                        "note": "cerar_allreduce_sim, events around the K calls only"}
+
     des = None
 
     # ---- end to end through the host-buffer entry point (pinned host memory)

@@ -131,6 +131,9 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
             fence_proxy_async_smem();
         }
         __syncthreads();
+        // up to here only the plan's constant coefficients were read: that may overlap the tail of the
+        // kernel before this one in the stream; the data may not be touched before that kernel is done
+        if (w == w_first) grid_dependency_wait();
 
         if (failed) {
             // a wait of this warp ran out in an earlier segment: only keep the CTA barriers company
@@ -299,6 +302,9 @@ contract_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap_in, const __gri
         while (global_ns() - t0 < 2000000ull) { }      // let async work that is in flight finish
     }
     // ---------------- tear-down: every warp arrives here (all waits above are bounded)
+    // (only now may the next kernel of the stream be scheduled next to this CTA: blocks that arrive
+    // early and wait for this grid to finish were measured to slow it down by 10 %)
+    grid_dependents_may_launch();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -315,8 +321,7 @@ cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const Con
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    kern<<<grid, NUM_THREADS, smem, s>>>(tin, tout, a, tp);
-    return cudaGetLastError();
+    return launch_pdl(kern, dim3((unsigned)grid), dim3(NUM_THREADS), smem, s, tin, tout, a, tp);
 }
 
 }  // namespace

@@ -21,6 +21,8 @@ using namespace ptx;
 __global__ void contract_ref_kernel(const ContractArgs a) {
     const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int w = blockIdx.y;
+    grid_dependents_may_launch();
+    grid_dependency_wait();
     if (q >= a.p) return;
     float acc[REF_MAX_J];
     for (int j = 0; j < a.J; ++j) acc[j] = 0.f;
@@ -80,6 +82,9 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
         }
     }
     __syncthreads();
+    // everything above reads only the plan's constant coefficients: it may overlap the tail of the
+    // kernel before this one; the data rows may not
+    grid_dependency_wait();
 
     uint32_t it = 0;            // chunk counter, same sequence in producer and consumers
     bool failed = false;
@@ -206,6 +211,10 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
     constexpr int VW = sizeof(VT) / 4;
     const int64_t nv = a.p / VW;
     const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    // Programmatic dependent launch: the next launch in the stream may be scheduled while this grid
+    // drains, and this grid touches memory only after the grid before it has completed.
+    grid_dependents_may_launch();
+    grid_dependency_wait();
     if (v >= nv) return;
     const int N = a.N, c = a.c, k = a.k;
     const int64_t pv = a.p / VW;                               // row pitch in vectors
@@ -273,14 +282,13 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
     if (per_worker < 1) per_worker = 1;
     if (per_worker > a.tiles_per_worker) per_worker = a.tiles_per_worker;
     dim3 grid((unsigned)per_worker, (unsigned)a.N);
-    kern<<<grid, threads, smem, s>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(kern, grid, dim3(threads), smem, s, a);
 }
 
 }  // namespace
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
-int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0;
+int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0;
 
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0 || a.N <= 0) return cudaSuccess;
@@ -344,7 +352,7 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     if (a.J > REF_MAX_J) return cudaErrorInvalidValue;
     const int threads = 128;
     dim3 grid((unsigned)((a.p + threads - 1) / threads), (unsigned)a.N);
-    contract_ref_kernel<<<grid, threads, 0, s>>>(a);
+    { cudaError_t el = launch_pdl(contract_ref_kernel, grid, dim3(threads), 0, s, a); if (el != cudaSuccess) return el; }
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
@@ -358,16 +366,16 @@ cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_n
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0) return cudaSuccess;
     const int threads = 256;
+    cudaError_t e;
     if (a.p % 4 == 0 && aligned16(a.ws)) {
         const int64_t nv = a.p / 4;
         const unsigned blocks = (unsigned)((nv + threads - 1) / threads);
         // plain loads and stores, 4 workers in flight per thread: streaming cache hints, 512-thread
         // blocks and 8 workers per group were all measured and are not faster at d = 1.4e9
-        round_kernel<float4, 4><<<blocks, threads, 0, s>>>(a);
+        e = launch_pdl(round_kernel<float4, 4>, dim3(blocks), dim3(threads), 0, s, a);
     } else {
-        round_kernel<float, 4><<<(unsigned)((a.p + threads - 1) / threads), threads, 0, s>>>(a);
+        e = launch_pdl(round_kernel<float, 4>, dim3((unsigned)((a.p + threads - 1) / threads)), dim3(threads), 0, s, a);
     }
-    cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }

@@ -75,7 +75,7 @@ bool tc_pair_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
 extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant,
-           g_tune_ring_wait_ms, g_tune_ring_tile;
+           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
 // Slots of the per-worker layout that round k reads (-1 = term absent) and the landing slot
 // in the neighbour's workspace; the one definition that launcher and callers share.
@@ -91,5 +91,19 @@ bool fused_supported(int N, int c);
 cudaError_t launch_fused(const float* grads, int64_t grads_stride, float* out, int64_t out_stride, const float* U,
                          const float* R, int N, int c, int64_t p, float scale, int num_sms, cudaStream_t s,
                          uint64_t* launches);
+
+// Launch with programmatic stream serialization (programmatic dependent launch): the kernel may be
+// scheduled while the previous kernel of the stream is still draining, so it must execute
+// ptx::grid_dependency_wait() before its first access to global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_tune_pdl_off ? 0 : 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 }  // namespace cerar

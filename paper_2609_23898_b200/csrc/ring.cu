@@ -13,6 +13,7 @@
 // landing slot through `peer_ws`, which may be a peer-mapped pointer into another
 // GPU's memory: plain coalesced 16-byte stores, no TMA and no multicast.
 #include "kernels.cuh"
+#include "ptx.cuh"
 
 namespace cerar {
 namespace {
@@ -29,6 +30,8 @@ template <typename VT>
 __global__ void __launch_bounds__(256) rank_round_kernel(const RankRoundArgs a) {
     constexpr int VW = sizeof(VT) / 4;
     const int64_t nv = a.p / VW;
+    ptx::grid_dependents_may_launch();
+    ptx::grid_dependency_wait();
     const VT* ws = reinterpret_cast<const VT*>(a.ws);
     VT* land = reinterpret_cast<VT*>(a.peer_ws) + (int64_t)a.slot_land * nv;
     const VT* prev = ws + (int64_t)a.slot_prev * nv;
@@ -62,9 +65,8 @@ cudaError_t launch_rank_round(RankRoundArgs a, int num_sms, cudaStream_t s, uint
     int64_t blocks = (nv + 255) / 256;
     const int64_t cap = (int64_t)num_sms * 16;         // grid-stride beyond 16 resident-size waves
     if (blocks > cap) blocks = cap;
-    if (vec) rank_round_kernel<float4><<<(unsigned)blocks, 256, 0, s>>>(a);
-    else rank_round_kernel<float><<<(unsigned)blocks, 256, 0, s>>>(a);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = vec ? launch_pdl(rank_round_kernel<float4>, dim3((unsigned)blocks), dim3(256), 0, s, a)
+                        : launch_pdl(rank_round_kernel<float>, dim3((unsigned)blocks), dim3(256), 0, s, a);
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }
