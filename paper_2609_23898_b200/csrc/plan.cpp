@@ -1,6 +1,8 @@
 // Host-side builder of the CERAR coefficient matrices (fp64 results; extended
 // precision inside where the windows A_l are ill-conditioned by construction).
 #include "plan.hpp"
+#include <atomic>
+#include <thread>
 #include <algorithm>
 
 #include <cmath>
@@ -322,22 +324,37 @@ double kappa_M_max(const HostPlan& P) {
 // U_k into [a0, b0] (sqrt(N) b0 / a0 = C guarantees the constraint), least
 // squares in R with U fixed.  Started from an epsilon-construction.
 
+// The N solves of an ALS step are independent (each writes only its own matrix): one thread each,
+// up to the host's core count.  The result does not depend on the number of threads.
+template <class F>
+static void parallel_for(int n, int c, F fn) {
+    unsigned hw = std::thread::hardware_concurrency();
+    int nt = (int)std::min<unsigned>(hw ? hw : 1u, (unsigned)n);
+    if (c < 24) nt = 1;                 // small solves: starting threads costs more than it saves
+    if (nt <= 1) { for (int i = 0; i < n; ++i) fn(i); return; }
+    std::vector<std::thread> th;
+    std::atomic<int> next(0);
+    for (int t = 0; t < nt; ++t)
+        th.emplace_back([&]() { for (int i = next.fetch_add(1); i < n; i = next.fetch_add(1)) fn(i); });
+    for (auto& x : th) x.join();
+}
+
 static void ls_R(HostPlan& P) {
     const int N = P.N, c = P.c, L = P.L;
     MatD T(N * c, c);
     for (int r = 0; r < N; ++r)
         for (int a = 0; a < c; ++a) T(r * c + a, a) = 1.0;
-    for (int i = 0; i < N; ++i) {
+    parallel_for(N, c, [&](int i) {
         MatD X;
         la::lstsq(m_matrix(P, i), T, X);
         for (int l = 0; l <= L; ++l)
             for (int j = 0; j < c; ++j) P.R[i][(size_t)l * c + j] = X(l, j);
-    }
+    });
 }
 
 static void ls_U(HostPlan& P) {
     const int N = P.N, c = P.c;
-    for (int k = 0; k < N; ++k) {
+    parallel_for(N, c, [&](int k) {
         // U_k [W_{s_0}(R_0) ... W_{s_{N-1}}(R_{N-1})] ~ [I ... I], s_i = (i-1-k) mod N;
         // transposed: rows of P^T are the columns of the windows.
         MatD Pt(N * c, c), Tt(N * c, c);
@@ -351,12 +368,12 @@ static void ls_U(HostPlan& P) {
         la::lstsq(Pt, Tt, X);
         for (int a = 0; a < c; ++a)
             for (int b = 0; b < c; ++b) P.U[k][(size_t)a * c + b] = X(b, a);
-    }
+    });
 }
 
 static void project(HostPlan& P, double a0, double b0) {
     const int c = P.c;
-    for (int k = 0; k < P.N; ++k) {
+    parallel_for(P.N, c, [&](int k) {
         MatD Uo, V;
         std::vector<double> s;
         la::svd_jacobi(mat_of(P.U[k], c, c), Uo, s, V);
@@ -367,7 +384,7 @@ static void project(HostPlan& P, double a0, double b0) {
                 for (int t = 0; t < c; ++t) acc += Uo(a, t) * s[t] * V(b, t);
                 P.U[k][(size_t)a * c + b] = acc;
             }
-    }
+    });
 }
 
 int build_kappa(int N, int c, double kappa_max, const double* B, const double* h, double eps_init,
