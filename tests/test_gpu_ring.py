@@ -180,3 +180,36 @@ def test_fused_rounds_give_up_when_a_neighbour_never_answers(mods):
     plan.device_status(s)
     ora = run_oracle(des.U, des.R, g, 1.0)
     assert max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
+
+
+def test_randomised_ring_shapes(mods):
+    """Seeded random (N, c, p): the rank-level path, round by round and with the fused rounds
+    (tile size forced small for some, so that short jobs have several tiles), against the oracle."""
+    import torch
+    cerar, inputs, ring = mods
+    rng = np.random.default_rng(31)
+    s = torch.cuda.current_stream().cuda_stream
+    try:
+        for trial in range(16):
+            N = int(rng.integers(2, 13))
+            c = max(N, int(rng.choice([N, N + 2, 2 * N, 16, 32, 48, 64])))
+            p = int(rng.choice([1, 4, 131, 516, 2052, 4104, 9000]))
+            tile = int(rng.choice([0, 64, 256, 1024]))
+            cerar.cerar_set_tuning("ring_tile", tile)
+            d = c * p
+            des = Dz.custom_orthogonal(N, c, np.random.default_rng(trial))
+            g = inputs.gradients_numpy(N, d, "normal", seed=200 + trial)
+            plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+            scale = float(rng.choice([1.0, 1.0 / N]))
+            ora = run_oracle(des.U, des.R, g, scale)
+            r = ring.LocalRing(plan, d)
+            grads = [torch.from_numpy(g[i]).cuda() for i in range(N)]
+            outs = [torch.empty(d, device="cuda") for _ in range(N)]
+            for fused in (False, True, True):
+                r.allreduce(grads, outs, scale, s, fused=fused)
+                torch.cuda.synchronize()
+                plan.device_status(s)
+                worst = max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N))
+                assert worst < 1e-5, (N, c, p, tile, fused, worst)
+    finally:
+        cerar.cerar_set_tuning("ring_tile", 0)
