@@ -30,7 +30,6 @@ template <typename VT>
 __global__ void __launch_bounds__(256) rank_round_kernel(const RankRoundArgs a) {
     constexpr int VW = sizeof(VT) / 4;
     const int64_t nv = a.p / VW;
-    ptx::grid_dependents_may_launch();
     ptx::grid_dependency_wait();
     const VT* ws = reinterpret_cast<const VT*>(a.ws);
     VT* land = reinterpret_cast<VT*>(a.peer_ws) + (int64_t)a.slot_land * nv;
