@@ -7,6 +7,8 @@
  * length-p messages (problem statement, Sec. I; protocol, Sec. II).  In this
  * library the N logical workers live in one GPU's memory and a ring hand-off
  * is a store into the neighbour's buffer; there is no inter-GPU transport.
+ * (The cerar_rank_* calls further down are the one-worker-per-GPU form of the
+ * same protocol, with the neighbour's buffer given as a pointer.)
  *
  * Conventions for every call
  *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA
@@ -245,7 +247,8 @@ cerar_status_t cerar_rank_decode(cerar_plan_t* plan, int rank, const float* ws, 
                                  float scale, cerar_stream_t stream);
 
 /* All L rounds in one launch per worker, ordered tile by tile instead of round by round.
- * The positions are cut into tiles of CERAR_RING_TILE; per tile a worker keeps two 32-bit
+ * The positions are cut into cerar_ring_tiles(plan, d) tiles (CERAR_RING_TILE positions each,
+ * four times that from p = 2^23); per tile a worker keeps two 32-bit
  * counters in its OWN memory that its neighbours write: `landed` (the previous worker has
  * stored message k of that tile here: value epoch (L+1) + k) and `freed` (the next worker
  * has finished round k on that tile, so the slot that message k+1 overwrites may be
@@ -328,13 +331,17 @@ cerar_status_t cerar_selftest_wait_timeout(cerar_plan_t* plan, int limit_ms, cer
  * back.  Returns the previous value. */
 int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
 
-/* Process-wide tuning knobs of the staged kernel, for experiments: name is one of
- * "kc" (input rows per pipeline stage), "stages", "jt" (outputs per thread: 4, 8
- * or 16), "slabs" (position slabs per CTA), "tc_kc" / "tc_stages" (rows per stage and
- * stages of the tensor-core kernel), "tc_variant" (1 = always tiles of 128 positions;
- * by default c <= 64 runs on tiles of 256 positions;
- * 2 / 3 = tiles of 256 wherever they fit, with one / two MMA issuers per half), "ring_wait_ms"
- * (limit of the waits of the fused ring rounds, default 2000); value 0 restores the default.
+/* Process-wide tuning knobs, for experiments and tests; value 0 restores the default.
+ *   "kc", "stages", "jt", "slabs"   staged FMA kernel: input rows per pipeline stage, stages,
+ *                                   outputs per thread (4, 8 or 16), position slabs per CTA
+ *   "tc_kc", "tc_stages"            tensor-core kernels: rows per stage, stages
+ *   "tc_variant"                    1 = always tiles of 128 positions (default: tiles of 256
+ *                                   positions for c <= 64); 2 / 3 = tiles of 256 with one /
+ *                                   two MMA issuers per half
+ *   "ring_wait_ms"                  limit of the waits of the fused ring rounds (default 2000)
+ *   "ring_tile"                     positions per tile of the fused ring rounds (a multiple of 4;
+ *                                   default 8192, 32768 from p = 2^23); set before sizing counters
+ *   "pdl_off"                       1 = launch without programmatic stream serialization
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 
