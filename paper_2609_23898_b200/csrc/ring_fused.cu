@@ -99,18 +99,20 @@ __global__ void __launch_bounds__(256) ring_rounds_kernel(const RingFusedArgs a)
                 float4* l4 = reinterpret_cast<float4*>(peer) + (int64_t)sl * pv;
                 for (int64_t v = q0 / 4 + threadIdx.x; v < q1 / 4; v += blockDim.x) {
                     float4 y = make_float4(0.f, 0.f, 0.f, 0.f), dc = y, da = y;
-                    if (sp >= 0) y = w4[(int64_t)sp * pv + v];
-                    if (sc >= 0) dc = w4[(int64_t)sc * pv + v];
-                    if (sa >= 0) da = w4[(int64_t)sa * pv + v];
+                    // .cg loads: a slot is read again two rounds after the neighbour has overwritten it,
+                    // and this kernel never ends in between, so nothing may be served from this SM's L1
+                    if (sp >= 0) y = __ldcg(w4 + (int64_t)sp * pv + v);
+                    if (sc >= 0) dc = __ldcg(w4 + (int64_t)sc * pv + v);
+                    if (sa >= 0) da = __ldcg(w4 + (int64_t)sa * pv + v);
                     l4[v] = comb4(y, dc, da);
                 }
             } else {
                 float* l1 = peer + (int64_t)sl * p;
                 for (int64_t q = q0 + threadIdx.x; q < q1; q += blockDim.x) {
                     float y = 0.f, dc = 0.f, da = 0.f;
-                    if (sp >= 0) y = ws[(int64_t)sp * p + q];
-                    if (sc >= 0) dc = ws[(int64_t)sc * p + q];
-                    if (sa >= 0) da = ws[(int64_t)sa * p + q];
+                    if (sp >= 0) y = __ldcg(ws + (int64_t)sp * p + q);
+                    if (sc >= 0) dc = __ldcg(ws + (int64_t)sc * p + q);
+                    if (sa >= 0) da = __ldcg(ws + (int64_t)sa * p + q);
                     l1[q] = (y - dc) + da;
                 }
             }
