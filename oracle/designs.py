@@ -7,8 +7,9 @@ A_l are extremely ill-conditioned by design (Remark after Theorem 1,
 Corollary 1), so a plain fp64 inverse would not be a trustworthy reference.
 The condition-number-constrained design is an fp64 iteration (numpy).
 
-PARITY UNPINNED: kappa_constrained (no published U, R to compare with; only
-its invariants are tested).
+PARITY UNPINNED: kappa_constrained for c > N (no published U, R to compare with;
+only its invariants are tested; for c = N, where the optimum Phi = 0 is known, it is
+checked to reach it).
 """
 from __future__ import annotations
 

@@ -356,3 +356,22 @@ def test_surrogate_is_well_conditioned():
     des = Dz.custom_orthogonal(4, 8, np.random.default_rng(0))
     for u in des.U:
         assert P.kappa2(u) == pytest.approx(1.0, abs=1e-9)
+
+
+@pytest.mark.parametrize("N,C", [(3, 1e6), (4, 1e4)])
+def test_kappa_constrained_reaches_the_known_optimum_when_c_equals_N(N, C):
+    """c = N is the exactly solvable case (Lemma 1 only forbids Phi = 0 for c > N; the classic
+    ring all-reduce is an exact solution): with a loose bound the constrained problem has
+    optimum Phi = 0, and the heuristic must get there from its O(eps^2) start, with the
+    decoded sum exact."""
+    c = N
+    B = _rng_B(N, c, 12)
+    des = Dz.kappa_constrained(N, c, C, B, iters=200)
+    hist = des.info["phi_history"]
+    assert hist[0] > 1e-4 and hist[-1] < 1e-18
+    assert max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N)) <= C
+    rng = np.random.default_rng(0)
+    g = [rng.standard_normal(c * 5) for _ in range(N)]
+    res = P.allreduce(g, des.U, des.R, 1.0)
+    for i in range(N):
+        assert P.rel_l2(res["out"][i], P.exact_sum(g)) < 1e-9

@@ -191,3 +191,14 @@ def test_tradeoff_report_runs_on_the_host(capsys, monkeypatch):
     assert "gamma(B, H)" in out and out.count("\n|---|") == 2
     rows = [ln for ln in out.splitlines() if ln.startswith("| 0.001 |")]
     assert len(rows) == 1 and "nan" not in rows[0]
+
+
+def test_library_kappa_design_reaches_phi_zero_when_c_equals_N():
+    """The exactly solvable case c = N: the library's ALS must end at Phi ~ 0 within its bound,
+    as the oracle's does."""
+    from paper_2609_23898_b200 import cerar, inputs
+    for N, C in [(3, 1e6), (4, 1e4)]:
+        B = inputs.base_matrix(N, N, 0)
+        p = cerar.Plan.create(N, N, cerar.KAPPA, C, B=B, host_only=True)
+        info = p.info()
+        assert info["phi"] < 1e-18 and info["kappa_M_max"] <= C
