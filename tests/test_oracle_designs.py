@@ -362,11 +362,11 @@ def test_surrogate_is_well_conditioned():
 def test_kappa_constrained_reaches_the_known_optimum_when_c_equals_N(N, C):
     """c = N is the exactly solvable case (Lemma 1 only forbids Phi = 0 for c > N; the classic
     ring all-reduce is an exact solution): with a loose bound the constrained problem has
-    optimum Phi = 0, and the heuristic must get there from its O(eps^2) start, with the
-    decoded sum exact."""
+    optimum Phi = 0 wherever the projection interval [a0, b0] does not bind (true for this B),
+    and the heuristic must get there from its O(eps^2) start, with the decoded sum exact."""
     c = N
     B = _rng_B(N, c, 12)
-    des = Dz.kappa_constrained(N, c, C, B, iters=200)
+    des = Dz.kappa_constrained(N, c, C, B, iters=1000, tol=1e-30)
     hist = des.info["phi_history"]
     assert hist[0] > 1e-4 and hist[-1] < 1e-18
     assert max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N)) <= C

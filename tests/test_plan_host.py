@@ -199,6 +199,6 @@ def test_library_kappa_design_reaches_phi_zero_when_c_equals_N():
     from paper_2609_23898_b200 import cerar, inputs
     for N, C in [(3, 1e6), (4, 1e4)]:
         B = inputs.base_matrix(N, N, 0)
-        p = cerar.Plan.create(N, N, cerar.KAPPA, C, B=B, host_only=True)
+        p = cerar.Plan.create(N, N, cerar.KAPPA, C, B=B, als_iters=1000, als_tol=1e-30, host_only=True)
         info = p.info()
         assert info["phi"] < 1e-18 and info["kappa_M_max"] <= C
