@@ -2,31 +2,42 @@
 //
 //   out[j][q] = scale * sum_k coef[k][j] * in[k][q],   j < J (= c),  k < K rows,  q < p
 //
-// is a skinny GEMM with M = positions (128 per tile), N = J, K = input rows.  At
-// c >= 32 the FP32 FMA pipe cannot keep up with HBM (c/4 flop per byte), so the
-// products run on the 5th-generation tensor cores as 3 x TF32: every fp32 value
-// is split into hi = tf32(x) and lo = tf32(x - hi) and
+// is a skinny GEMM with M = positions, N = J, K = input rows.  At c >= 32 the FP32 FMA pipe
+// cannot keep up with HBM (c/4 flop per byte), so the products run on the 5th-generation
+// tensor cores as 3 x TF32: every fp32 value is split into hi = tf32(x), lo = tf32(x - hi) and
 //   x*y ~ lo_x*hi_y + hi_x*lo_y + hi_x*hi_y           (relative error ~ 2^-22),
 // accumulated in fp32 in tensor memory.
 //
-// One CTA of 11 warps per SM, persistent over the 128-position tiles of one worker:
-//   warp 0      producer: one TMA load per chunk ([KC rows] x [128 positions], row-major)
-//   warps 6-9   splitter: thread = position; reads its column of the chunk from shared
-//               memory, splits it, and writes hi | lo into tensor memory (tcgen05.st),
-//               where they are the A operand (rows = positions, columns = k)
-//   warps 1,10  MMA issuers (one lane each, even / odd tiles, so that one can issue while
-//               the other drains): tcgen05.mma kind::tf32, A from TMEM, B = the
-//               coefficient matrix (hi and lo copies) resident in shared memory,
-//               M=128, N=Npad, K=8 per instruction; warp 1 owns the TMEM allocation
-//   warps 2-5   epilogue: tcgen05.ld of the accumulator, scale, transpose through a
-//               shared-memory tile, one TMA store per 32 output rows
-// So the data tile is read from shared memory exactly once, and global memory is
-// touched only by TMA in rows of 512 contiguous bytes.  Every wait is bounded.
+// A tile is HALVES UMMA tiles of M = 128 positions ("halves").  HALVES = 2 (c <= 64): global
+// memory is read and written in rows of 1 KB, which HBM serves measurably better than 512 B;
+// half h belongs to the MMA issuers of half h for the whole run.  HALVES = 1 (c <= 128): the
+// four accumulators of two halves would not leave room for the A operand in the 512 TMEM
+// columns, and two coefficient copies of c = 128 leave shared memory for 128-position stages
+// only.
+//
+// One CTA of 21 warps per SM.  The tiles of all workers form one list that is cut into one
+// contiguous range per CTA, so every SM is busy whatever N is; a range that crosses a worker
+// boundary is processed in two segments (the coefficients are per worker).
+//   warp 0        producer: one TMA load per chunk ([KC rows] x [tile positions])
+//   warps 11-18   splitter: thread = position (of every half); the two warps of a lane
+//                 quadrant take one half of the chunk's rows each; values are split into
+//                 tf32 hi | lo and written to tensor memory (tcgen05.st), where they are
+//                 the A operand of their half: shared memory is read once per element
+//   warps 1, 2    MMA issuers (one lane each) for half 0 / 1, even tiles; warps 19, 20 the
+//                 same for the odd tiles when a tile has more than four k-steps (an issuing
+//                 thread is limited by its own instruction stream, not by the tensor pipe):
+//                 tcgen05.mma kind::tf32, A from TMEM, B = the coefficients (hi and lo
+//                 copies) in shared memory, M=128, N=Npad, K=8; two accumulators per half,
+//                 so that the epilogue of one tile overlaps the products of the next;
+//                 warp 1 owns the TMEM allocation
+//   warps 3-10    epilogue: tcgen05.ld (16 of every 32 output rows per warp), scale,
+//                 transpose through a shared-memory tile, one TMA store per 32 output rows
+// Every wait is bounded; a wait that runs out sets the status word and the CTA leaves
+// through the common exit, where tensor memory is freed.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
-#include <cstdio>
 
 #include "kernels.cuh"
 #include "tc_common.cuh"
@@ -34,218 +45,265 @@
 namespace cerar {
 namespace {
 
-constexpr int TILE_M = 128;          // positions per tile = UMMA M
-constexpr int NUM_THREADS = 32 * 11;
-constexpr int OUT_ROWS = 32;         // output rows per TMA store
-
 using namespace tc;
 
-struct TcParams {
+constexpr int HALF_M = 128;              // UMMA M
+constexpr int OUT_ROWS = 32;             // output rows per TMA store
+constexpr int NUM_WARPS = 21;
+constexpr int NUM_THREADS = 32 * NUM_WARPS;
+constexpr int WARP_EPI0 = 3, WARP_SPLIT0 = 11, WARP_MMA2 = 19;
+
+struct PairParams {
     int K_rows;        // physical input rows that carry data; rows beyond read as zero (TMA fill)
     int K_pad;         // K_rows rounded up to a multiple of KC
     int stages;        // shared-memory stages of raw chunks
-    int NA;            // A (hi|lo) chunk buffers in tensor memory
+    int NAh;           // A (hi|lo) chunk buffers per half in tensor memory
     int Npad;          // J rounded up to 32
-    int tmem_cols;     // power of two >= 2*Npad + NA*2*KC
+    int tmem_cols;     // power of two >= HALVES * (2*Npad + NAh*2*KC)
+    int four_issuers;  // 1: every half has one issuer per accumulator (even / odd tiles)
+    int64_t tiles_per_worker;
+    int64_t total_tiles;
 };
 
 // shared memory (1024-aligned): B_hi | B_lo | raw stages | 2 output tiles | barriers | tmem slot
-template <int KC>
+template <int KC, int HALVES>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
-                   const __grid_constant__ ContractArgs a, const __grid_constant__ TcParams tp) {
+                   const __grid_constant__ ContractArgs a, const __grid_constant__ PairParams tp) {
+    constexpr int TILE_W = HALVES * HALF_M;      // positions per tile
     extern __shared__ unsigned char smem_dyn[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int w = blockIdx.y;
-    const int stages = tp.stages, NA = tp.NA, Npad = tp.Npad, K_pad = tp.K_pad;
+    const int stages = tp.stages, Npad = tp.Npad, K_pad = tp.K_pad;
+    const uint32_t NAh = (uint32_t)tp.NAh;
     const int nkc = K_pad / KC;
     const int nblk = Npad / 32;
-    const uint32_t NAh = (uint32_t)NA / 2u;      // A buffers per MMA issuer
+    static_assert(KC % 8 == 0, "a chunk is a whole number of k-steps");
+    constexpr int KG = KC / 2;           // rows of a chunk per splitter warp of a quadrant (a multiple of 4)
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* smem_al = smem_dyn + (smem_base - smem_u32(smem_dyn));
     const uint32_t b_bytes = (uint32_t)K_pad * Npad * 4u;            // one of B_hi / B_lo
-    constexpr uint32_t chunk_bytes = (uint32_t)KC * TILE_M * 4u;
-    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * TILE_M * 4u;
+    constexpr uint32_t chunk_bytes = (uint32_t)KC * TILE_W * 4u;
+    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * TILE_W * 4u;
     const uint32_t bhi_u32 = smem_base, blo_u32 = smem_base + b_bytes;
     const uint32_t raw_u32 = smem_base + 2u * b_bytes;
     const uint32_t out_u32 = raw_u32 + (uint32_t)stages * chunk_bytes;
     const uint32_t bar_u32 = out_u32 + 2u * out_bytes;
     const uint32_t raw_full = bar_u32, raw_empty = raw_full + 8u * stages;
-    const uint32_t a_full = raw_empty + 8u * stages, a_empty = a_full + 8u * NA;
-    const uint32_t acc_full = a_empty + 8u * NA, acc_empty = acc_full + 16u;
-    const uint32_t out_full = acc_empty + 16u, out_free = out_full + 16u;
+    // "A buffer filled": one barrier per (half, tile parity, buffer), so that each has ONE waiter
+    // (the issuer of that half and parity) who sees all of its phases in order; a barrier that two
+    // issuers took turns on could be two phases ahead of one of them, which a parity wait cannot tell
+    const uint32_t a_full = raw_empty + 8u * stages;                 // [half][parity][NAh]
+    const uint32_t a_empty = a_full + 16u * HALVES * NAh;            // [half][NAh]
+    const uint32_t acc_full = a_empty + 8u * HALVES * NAh;           // [half][2]
+    const uint32_t acc_empty = acc_full + 32u;
+    const uint32_t out_full = acc_empty + 32u, out_free = out_full + 16u;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem_al + (out_free + 16u - smem_base));
     const float* raw_s = reinterpret_cast<const float*>(smem_al + (raw_u32 - smem_base));
     float* out_s = reinterpret_cast<float*>(smem_al + (out_u32 - smem_base));
 
     // ---------------- set-up
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) { mbar_init(raw_full + 8u * s, 1); mbar_init(raw_empty + 8u * s, 4); }
-        for (int b = 0; b < NA; ++b) { mbar_init(a_full + 8u * b, 4); mbar_init(a_empty + 8u * b, 1); }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, 4);
-            mbar_init(out_full + 8u * b, 4); mbar_init(out_free + 8u * b, 1);
-        }
+        for (int s = 0; s < stages; ++s) { mbar_init(raw_full + 8u * s, 1); mbar_init(raw_empty + 8u * s, 8); }
+        for (uint32_t b = 0; b < 2u * HALVES * NAh; ++b) mbar_init(a_full + 8u * b, 8);
+        for (uint32_t b = 0; b < HALVES * NAh; ++b) mbar_init(a_empty + 8u * b, 1);
+        for (int b = 0; b < 2 * HALVES; ++b) { mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(out_full + 8u * b, 8); mbar_init(out_free + 8u * b, 1); }
         mbar_init_fence();
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)tp.tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    {
-        // coefficients of this worker as the tensor core's B operand (tf32 hi and lo copies)
-        split_coefficients(a, w, K_pad, Npad, reinterpret_cast<uint32_t*>(smem_al),
-                           reinterpret_cast<uint32_t*>(smem_al + b_bytes));
-        fence_proxy_async_smem();
-    }
+    if (warp == 1) tc_alloc(smem_u32(tmem_slot), (uint32_t)tp.tmem_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    // the set-up above reads only the plan's constant coefficients and may overlap the tail of the
-    // kernel before this one in the stream; the data may not be touched before that kernel is done
-    grid_dependency_wait();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t a_col0 = 2u * (uint32_t)Npad;            // A buffers start after the two accumulators
+    const uint32_t a_col0 = 2u * HALVES * (uint32_t)Npad;   // A buffers start after the accumulators (two per half)
 
-    const int64_t ntiles = a.tiles_per_worker;
+    // this CTA's contiguous range of the tile list (worker-major), cut at worker boundaries
+    const int64_t T = tp.tiles_per_worker;
+    const int64_t g_begin = tp.total_tiles * blockIdx.x / gridDim.x;
+    const int64_t g_end = tp.total_tiles * (blockIdx.x + 1) / gridDim.x;
+    const int w_first = (int)(g_begin / T);
+    const int w_last = g_end > g_begin ? (int)((g_end - 1) / T) : w_first - 1;
+
     bool failed = false;
+    uint32_t it = 0, tc = 0, oc = 0;      // chunks, tiles and output blocks this CTA has gone through (all roles count alike)
+    uint32_t afull_ph = 0;                // issuers: next phase parity of their "filled" barriers, bit = 4 * parity + buffer
 
-    if (warp == 0) {
-        // ================= producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x) {
-                const int q0 = (int)(t * TILE_M);
-                for (int kc = 0; kc < nkc; ++kc, ++it) {
-                    const uint32_t s = it % stages, ph = (it / stages) & 1u;
-                    if (!mbar_wait_bounded(raw_empty + 8u * s, ph ^ 1u)) { failed = true; break; }
-                    mbar_arrive_expect_tx(raw_full + 8u * s, chunk_bytes);
-                    tma_load_3d(raw_u32 + s * chunk_bytes, &tmap_in, q0, kc * KC, w, raw_full + 8u * s);
+    for (int w = w_first; w <= w_last; ++w) {
+        const int64_t t_begin = (w == w_first) ? g_begin - (int64_t)w * T : 0;
+        const int64_t t_end = (w == w_last) ? g_end - (int64_t)w * T : T;
+        {
+            // coefficients of this worker as the tensor core's B operand (tf32 hi and lo copies)
+            split_coefficients(a, w, K_pad, Npad, reinterpret_cast<uint32_t*>(smem_al),
+                               reinterpret_cast<uint32_t*>(smem_al + b_bytes));
+            fence_proxy_async_smem();
+        }
+        __syncthreads();
+        // up to here only the plan's constant coefficients were read: that may overlap the tail of the
+        // kernel before this one in the stream; the data may not be touched before that kernel is done
+        if (w == w_first) grid_dependency_wait();
+
+        if (failed) {
+            // a wait of this warp ran out in an earlier segment: only keep the CTA barriers company
+        } else if (warp == 0) {
+            // ================= producer
+            if (lane == 0) {
+                for (int64_t t = t_begin; t < t_end && !failed; ++t) {
+                    const int q0 = (int)(t * TILE_W);
+                    for (int kc = 0; kc < nkc; ++kc, ++it) {
+                        const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                        if (!mbar_wait_bounded(raw_empty + 8u * s, ph ^ 1u)) { failed = true; break; }
+                        mbar_arrive_expect_tx(raw_full + 8u * s, chunk_bytes);
+                        tma_load_3d(raw_u32 + s * chunk_bytes, &tmap_in, q0, kc * KC, w, raw_full + 8u * s);
+                    }
                 }
             }
-        }
-    } else if (warp == 1 || warp == 10) {
-        // ================= MMA issuers: issuer m takes tiles m, m+2, ... into accumulator m
-        if (lane == 0) {
-            const uint32_t m = (warp == 1) ? 0u : 1u;
-            // instruction descriptor: D=f32, A=B=tf32, A from TMEM (K-major), B MN-major, N=Npad, M=128
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | (1u << 16) |
-                                   ((uint32_t)(Npad >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
-            const uint32_t b_lbo = (uint32_t)K_pad * 128u;
-            const uint64_t bhi0 = make_desc(bhi_u32, b_lbo, 512u), blo0 = make_desc(blo_u32, b_lbo, 512u);
-            const uint32_t d_tmem = tmem_base + m * (uint32_t)Npad;
-            uint32_t tc = m;
-            for (int64_t t = blockIdx.x + (int64_t)m * gridDim.x; t < ntiles && !failed; t += 2 * (int64_t)gridDim.x, tc += 2) {
-                const uint32_t aph = (tc >> 1) & 1u;
-                if (!mbar_wait_bounded(acc_empty + 8u * m, aph ^ 1u)) { failed = true; break; }
-                tc_fence_after();
-                for (int kc = 0; kc < nkc; ++kc) {
-                    const uint32_t seq = (tc >> 1) * (uint32_t)nkc + (uint32_t)kc;
-                    const uint32_t ab = m * NAh + seq % NAh, ph = (seq / NAh) & 1u;
-                    if (!mbar_wait_bounded(a_full + 8u * ab, ph)) { failed = true; break; }
+        } else if (warp == 1 || warp == 2 || warp >= WARP_MMA2) {
+            // ================= MMA issuer of half m: accumulators 2m, 2m+1 alternate by tile.
+            // With four issuers, warps 1, 2 take the even tiles and warps 19, 20 the odd ones
+            // (an issuing thread is limited by its own instruction stream, not by the tensor pipe).
+            const bool odd_only = warp >= WARP_MMA2;
+            const uint32_t m = (uint32_t)(odd_only ? warp - WARP_MMA2 : warp - 1);
+            if (lane == 0 && m < (uint32_t)HALVES && (tp.four_issuers || !odd_only)) {
+                const uint32_t idesc = idesc_tf32_ts((uint32_t)Npad);
+                const uint32_t b_lbo = (uint32_t)K_pad * 128u;
+                const uint64_t bhi0 = make_desc(bhi_u32, b_lbo, 512u), blo0 = make_desc(blo_u32, b_lbo, 512u);
+                for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                    const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
+                    if (tp.four_issuers && (buf != 0u) != odd_only) continue;
+                    const uint32_t d_tmem = tmem_base + (2u * m + buf) * (uint32_t)Npad;
+                    if (!mbar_wait_bounded(acc_empty + 8u * (2u * m + buf), aph ^ 1u)) { failed = true; break; }
                     tc_fence_after();
-                    const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
-                    int ksteps = KC / 8;
-                    const int rows_left = tp.K_rows - kc * KC;               // rows with data in this chunk
-                    if (rows_left < KC) ksteps = (rows_left + 7) / 8;
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        // descriptor start address advances by 8 rows x 128 B (in 16-byte units)
-                        const uint64_t boff = (uint64_t)(((kc * KC + ks * 8) * 128) >> 4);
-                        tc_mma_tf32_ts(d_tmem, a_lo + ks * 8u, bhi0 + boff, idesc, (kc | ks) != 0);
-                        tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, blo0 + boff, idesc, 1u);
-                        tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, bhi0 + boff, idesc, 1u);
-                    }
-                    tc_commit(a_empty + 8u * ab);      // the A buffer is free once these MMAs have read it
-                }
-                if (failed) break;
-                tc_commit(acc_full + 8u * m);          // the accumulator is complete
-            }
-        }
-    } else if (warp < 6) {
-        // ================= epilogue (warps 2..5; TMEM lanes 32*(warp%4) ..)
-        const int qd = warp & 3;
-        const int pos = qd * 32 + lane;
-        uint32_t tc = 0, oc = 0;
-        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++tc) {
-            const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
-            if (!warp_wait(acc_full + 8u * buf, aph)) { failed = true; break; }
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + buf * (uint32_t)Npad;
-            for (int nb = 0; nb < nblk; ++nb, ++oc) {
-                float v[32];
-                tc_ld32(taddr + (uint32_t)nb * 32u, v);
-                if (nb == nblk - 1) {
-                    // everything is in registers: hand the accumulator back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(acc_empty + 8u * buf);
-                }
-                const uint32_t ob = oc & 1u, oph = (oc >> 1) & 1u;
-                if (!warp_wait(out_free + 8u * ob, oph ^ 1u)) { failed = true; break; }
-                float* o = out_s + (size_t)ob * (OUT_ROWS * TILE_M) + pos;
-#pragma unroll
-                for (int j = 0; j < 32; ++j) o[j * TILE_M] = v[j] * a.scale;
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(out_full + 8u * ob);
-                if (warp == 2 && lane == 0) {
-                    if (!mbar_wait_bounded(out_full + 8u * ob, oph)) {
-                        failed = true;
-                    } else {
-                        // rows beyond J and positions beyond p are clipped by the tensor map
-                        tma_store_3d(&tmap_out, (int)(t * TILE_M), nb * OUT_ROWS, w, out_u32 + ob * out_bytes);
-                        bulk_commit();
-                        if (oc >= 1) {                 // the store before this one has read its tile: free it
-                            bulk_wait_read_1();
-                            mbar_arrive(out_free + 8u * (ob ^ 1u));
+                    for (int kc = 0; kc < nkc; ++kc) {
+                        const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
+                        const uint32_t b = seq % NAh, ab = m * NAh + b;
+                        const uint32_t bit = 4u * buf + b, ph = (afull_ph >> bit) & 1u;
+                        if (!mbar_wait_bounded(a_full + 8u * ((2u * m + buf) * NAh + b), ph)) { failed = true; break; }
+                        afull_ph ^= 1u << bit;
+                        tc_fence_after();
+                        const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
+                        int ksteps = KC / 8;
+                        const int rows_left = tp.K_rows - kc * KC;               // rows with data in this chunk
+                        if (rows_left < KC) ksteps = (rows_left + 7) / 8;
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            // descriptor start address advances by 8 rows x 128 B (in 16-byte units)
+                            const uint64_t boff = (uint64_t)(((kc * KC + ks * 8) * 128) >> 4);
+                            tc_mma_tf32_ts(d_tmem, a_lo + ks * 8u, bhi0 + boff, idesc, (kc | ks) != 0);
+                            tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, blo0 + boff, idesc, 1u);
+                            tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, bhi0 + boff, idesc, 1u);
                         }
+                        tc_commit(a_empty + 8u * ab);      // the A buffer is free once these MMAs have read it
+                    }
+                    if (failed) break;
+                    tc_commit(acc_full + 8u * (2u * m + buf));          // the accumulator is complete
+                }
+            }
+        } else if (warp < WARP_SPLIT0) {
+            // ================= epilogue (TMEM lanes 32*(warp%4) ..; group g takes rows 16g..16g+15 of every 32)
+            const int qd = warp & 3, g = (warp - WARP_EPI0) >> 2;
+            const int pos = qd * 32 + lane;
+            for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
+                for (int nb = 0; nb < nblk && !failed; ++nb, ++oc) {
+                    const uint32_t ob = oc & 1u, oph = (oc >> 1) & 1u;
+                    if (!warp_wait(out_free + 8u * ob, oph ^ 1u)) { failed = true; break; }
+                    float* o = out_s + (size_t)ob * (OUT_ROWS * TILE_W) + (size_t)(g * 16) * TILE_W + pos;
+#pragma unroll
+                    for (int h = 0; h < HALVES; ++h) {
+                        const uint32_t acc = 2u * h + buf;
+                        if (nb == 0 && !warp_wait(acc_full + 8u * acc, aph)) { failed = true; break; }
+                        tc_fence_after();
+                        float v[16];
+                        tc_ld16(tmem_base + ((uint32_t)(qd * 32) << 16) + acc * (uint32_t)Npad + (uint32_t)(nb * 32 + g * 16), v);
+                        if (nb == nblk - 1) {
+                            // this warp's part of the accumulator is in registers: hand it back
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(acc_empty + 8u * acc);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) o[j * TILE_W + h * HALF_M] = v[j] * a.scale;
+                    }
+                    if (failed) break;
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(out_full + 8u * ob);
+                    if (warp == WARP_EPI0) {
+                        if (lane == 0) {
+                            if (!mbar_wait_bounded(out_full + 8u * ob, oph)) {
+                                failed = true;
+                            } else {
+                                // rows beyond J and positions beyond p are clipped by the tensor map
+                                tma_store_3d(&tmap_out, (int)(t * TILE_W), nb * OUT_ROWS, w, out_u32 + ob * out_bytes);
+                                bulk_commit();
+                                if (oc >= 1) {                 // the store before this one has read its tile: free it
+                                    bulk_wait_read_1();
+                                    mbar_arrive(out_free + 8u * (ob ^ 1u));
+                                }
+                            }
+                        }
+                        failed = __any_sync(0xffffffffu, failed ? 1 : 0) != 0;
                     }
                 }
-                if (warp == 2) failed = __any_sync(0xffffffffu, failed ? 1 : 0) != 0;
-                if (failed) break;
+            }
+        } else {
+            // ================= splitter (TMEM lanes 32*(warp%4) ..; group g takes rows [g*KG, (g+1)*KG) of the chunk)
+            const int qd = warp & 3, g = (warp - WARP_SPLIT0) >> 2;
+            const int pos = qd * 32 + lane;
+            const int r0 = g * KG;
+            for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                for (int kc = 0; kc < nkc && !failed; ++kc, ++it) {
+                    const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                    const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
+                    const uint32_t abi = seq % NAh, pa = (seq / NAh) & 1u;
+                    if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
+                    const float* col = raw_s + (size_t)s * (KC * TILE_W) + (size_t)r0 * TILE_W + pos;
+                    // rows of this chunk that some product reads (the last chunk may be short): rounded up
+                    // to the k-step, rows beyond the data are zero (TMA fill)
+                    const int rows_left = tp.K_rows - kc * KC;
+                    const int kuse = ((rows_left < KC ? rows_left : KC) + 7) / 8 * 8 - r0;   // relative to r0
+#pragma unroll
+                    for (int h = 0; h < HALVES; ++h) {
+                        uint32_t hi[KG], lo[KG];
+#pragma unroll
+                        for (int k = 0; k < KG; ++k) {
+                            if ((k & ~3) < kuse) {
+                                const float x = col[k * TILE_W + h * HALF_M];
+                                hi[k] = tf32_bits(x);
+                                lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
+                            }
+                        }
+                        if (h == HALVES - 1) {
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(raw_empty + 8u * s);        // the whole chunk is in registers
+                        }
+                        const uint32_t ab = (uint32_t)h * NAh + abi;
+                        if (!warp_wait(a_empty + 8u * ab, pa ^ 1u)) { failed = true; break; }
+                        tc_fence_after();
+                        const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC) + (uint32_t)r0;
+#pragma unroll
+                        for (int k4 = 0; k4 < KG / 4; ++k4) {
+                            if (4 * k4 < kuse) {               // uniform over the warp
+                                tc_st4(ta + 4u * k4, hi + 4 * k4);
+                                tc_st4(ta + KC + 4u * k4, lo + 4 * k4);
+                            }
+                        }
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(a_full + 8u * ((2u * (uint32_t)h + (tc & 1u)) * NAh + abi));
+                    }
+                }
             }
         }
-        if (warp == 2 && lane == 0) bulk_wait_all();   // all output has left shared memory and is written
-    } else {
-        // ================= splitter (warps 6..9): thread = position
-        const int qd = warp & 3;
-        const int pos = qd * 32 + lane;
-        uint32_t it = 0, tc = 0;
-        for (int64_t t = blockIdx.x; t < ntiles && !failed; t += gridDim.x, ++tc) {
-            for (int kc = 0; kc < nkc; ++kc, ++it) {
-                const uint32_t s = it % stages, ph = (it / stages) & 1u;
-                // A buffers are split between the two MMA issuers: tile parity picks the half
-                const uint32_t seq = (tc >> 1) * (uint32_t)nkc + (uint32_t)kc;
-                const uint32_t ab = (tc & 1u) * NAh + seq % NAh, pa = (seq / NAh) & 1u;
-                if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
-                const float* col = raw_s + (size_t)s * (KC * TILE_M) + pos;
-                uint32_t hi[KC], lo[KC];
-#pragma unroll
-                for (int k = 0; k < KC; ++k) {
-                    const float x = col[k * TILE_M];
-                    hi[k] = tf32_bits(x);
-                    lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(raw_empty + 8u * s);        // the values are in registers
-                if (!warp_wait(a_empty + 8u * ab, pa ^ 1u)) { failed = true; break; }
-                tc_fence_after();
-                const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC);
-#pragma unroll
-                for (int k8 = 0; k8 < KC / 8; ++k8) {
-                    tc_st8(ta + 8u * k8, hi + 8 * k8);
-                    tc_st8(ta + KC + 8u * k8, lo + 8 * k8);
-                }
-                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(a_full + 8u * ab);
-            }
-        }
+        // ---------------- end of segment: all products that read these coefficients are done
+        // (the epilogue has waited for every accumulator) before the next worker's overwrite them
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
     }
 
+    if (warp == WARP_EPI0 && lane == 0) bulk_wait_all();   // all output has left shared memory and is written
     if (failed) {
         if (lane == 0) atomicExch(a.status, 2);
         const unsigned long long t0 = global_ns();
@@ -259,19 +317,62 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)tp.tmem_cols) : "memory");
+        tc_dealloc(tmem_base, (uint32_t)tp.tmem_cols);
     }
 }
 
-template <int KC>
-cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a, const TcParams& tp,
-                      size_t smem, dim3 grid, cudaStream_t s) {
-    auto kern = contract_tc_kernel<KC>;
+template <int KC, int HALVES>
+cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a, const PairParams& tp,
+                      size_t smem, int grid, cudaStream_t s) {
+    auto kern = contract_tc_kernel<KC, HALVES>;
     {   // per device and cheap: set on every launch rather than cached
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    return launch_pdl(kern, grid, dim3(NUM_THREADS), smem, s, tin, tout, a, tp);
+    return launch_pdl(kern, dim3((unsigned)grid), dim3(NUM_THREADS), smem, s, tin, tout, a, tp);
+}
+
+template <int HALVES>
+cudaError_t launch_halves(int KC, const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a,
+                          const PairParams& tp, size_t smem, int grid, cudaStream_t s) {
+    switch (KC) {
+        case 40: return launch_kc<40, HALVES>(tin, tout, a, tp, smem, grid, s);
+        case 32: return launch_kc<32, HALVES>(tin, tout, a, tp, smem, grid, s);
+        case 24: return launch_kc<24, HALVES>(tin, tout, a, tp, smem, grid, s);
+        default: return launch_kc<16, HALVES>(tin, tout, a, tp, smem, grid, s);
+    }
+}
+
+// Rows per chunk (0 if nothing fits): as few chunks as possible, then as few padded rows as
+// possible, with at least 3 stages in the shared memory that the coefficient copies and the
+// output tiles leave and at least two A buffers per half in the tensor memory that the
+// accumulators leave.
+int choose_chunk(const ContractArgs& a, int halves, PairParams* tp) {
+    const int tile_w = halves * HALF_M;
+    tp->K_rows = a.K + a.skip_count;                        // decode: physical rows that are not part of Y
+    tp->Npad = ((a.J + 31) / 32) * 32;
+    const size_t budget = 227 * 1024 - 1024;
+    const int cands[4] = {40, 32, 24, 16};
+    int best_kc = 0, best_pad = 1 << 30, best_stages = 0, best_nk = 1 << 30;
+    for (int ci = 0; ci < 4; ++ci) {
+        const int kc = cands[ci];
+        if (g_tune_tc_kc && kc != g_tune_tc_kc) continue;
+        if (halves * (2 * tp->Npad + 2 * 2 * kc) > 512) continue;
+        const int kpad = ((tp->K_rows + kc - 1) / kc) * kc;
+        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp->Npad * 4 + 2 * (size_t)OUT_ROWS * tile_w * 4 + 512;
+        const size_t stage_c = (size_t)kc * tile_w * 4;
+        if (fixed_c + 3 * stage_c > budget) continue;
+        int st = (int)((budget - fixed_c) / stage_c);
+        if (st > 8) st = 8;
+        if (g_tune_tc_stages && g_tune_tc_stages < st) st = g_tune_tc_stages;
+        if (st < 2) continue;
+        // fewest chunks first (every chunk costs a round of barrier hand-offs), then fewest padded rows
+        const int nk = kpad / kc;
+        if (nk < best_nk || (nk == best_nk && kpad < best_pad)) { best_nk = nk; best_pad = kpad; best_kc = kc; best_stages = st; }
+    }
+    tp->K_pad = best_pad;
+    tp->stages = best_stages;
+    return best_kc;
 }
 
 }  // namespace
@@ -287,56 +388,37 @@ bool tc_eligible(const ContractArgs& a) {
 }
 
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches) {
-    TcParams tp;
-    tp.K_rows = a.K + a.skip_count;                         // decode: physical rows that are not part of Y
-    tp.Npad = ((a.J + 31) / 32) * 32;
-    // rows per chunk: as few padded rows as possible, then as large as possible, with at
-    // least 3 stages in the shared memory that the two coefficient copies leave
-    const size_t budget = 227 * 1024 - 1024;
-    const int cands[4] = {40, 32, 24, 16};
-    int best_kc = 0, best_pad = 1 << 30, best_stages = 0;
-    for (int ci = 0; ci < 4; ++ci) {
-        const int kc = cands[ci];
-        if (g_tune_tc_kc && kc != g_tune_tc_kc) continue;
-        if (2 * tp.Npad + 2 * 2 * kc > 512) continue;       // two accumulators + at least two A buffers
-        const int kpad = ((tp.K_rows + kc - 1) / kc) * kc;
-        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp.Npad * 4 + 2 * OUT_ROWS * TILE_M * 4 + 512;
-        const size_t stage_c = (size_t)kc * TILE_M * 4;
-        if (fixed_c + 3 * stage_c > budget) continue;
-        int st = (int)((budget - fixed_c) / stage_c);
-        if (st > 8) st = 8;
-        if (g_tune_tc_stages && g_tune_tc_stages < st) st = g_tune_tc_stages;
-        if (st < 2) continue;
-        if (kpad < best_pad) { best_pad = kpad; best_kc = kc; best_stages = st; }
-    }
-    if (!best_kc) return cudaErrorInvalidConfiguration;
-    const int KC = best_kc;
-    tp.K_pad = best_pad;
-    tp.stages = best_stages;
-    tp.NA = (512 - 2 * tp.Npad) / (2 * KC);
-    if (tp.NA > 4) tp.NA = 4;
-    tp.NA -= tp.NA % 2;                                   // one half per MMA issuer
+    // tiles of 256 positions where four accumulators fit next to the A operand (c <= 64) and the
+    // coefficient copies leave room for 256-position stages; tc_variant 1 forces tiles of 128
+    PairParams tp;
+    int halves = (a.J <= 64 && g_tune_tc_variant != 1) ? 2 : 1;
+    int KC = choose_chunk(a, halves, &tp);
+    if (!KC && halves == 2) { halves = 1; KC = choose_chunk(a, halves, &tp); }
+    if (!KC) return cudaErrorInvalidConfiguration;
+    const int tile_w = halves * HALF_M;
+    tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
+    if (tp.NAh > 4) tp.NAh = 4;
+    // Measured on B200 at c = 32: a second issuer per half pays once a tile has more than 4 k-steps
+    // (decode +8 .. +25 %), and costs 2 % below that (encode).  With one half per tile two issuers
+    // (even / odd tiles) are the minimum that keeps one issuing while the other drains.
+    tp.four_issuers = ((tp.K_rows + 7) / 8 > 4 || halves == 1) ? 1 : 0;
+    if (g_tune_tc_variant == 2) tp.four_issuers = 0;
+    if (g_tune_tc_variant == 3) tp.four_issuers = 1;
     tp.tmem_cols = 32;
-    while (tp.tmem_cols < 2 * tp.Npad + tp.NA * 2 * KC) tp.tmem_cols *= 2;
-    const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * TILE_M * 4 +
-                        2 * OUT_ROWS * TILE_M * 4 + 512;
+    while (tp.tmem_cols < halves * (2 * tp.Npad + tp.NAh * 2 * KC)) tp.tmem_cols *= 2;
+    const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * tile_w * 4 +
+                        2 * (size_t)OUT_ROWS * tile_w * 4 + 512;
 
     CUtensorMap tin, tout;
-    if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, TILE_M, KC)) return cudaErrorInvalidValue;
-    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, TILE_M, OUT_ROWS)) return cudaErrorInvalidValue;
+    if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, tile_w, KC)) return cudaErrorInvalidValue;
+    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, tile_w, OUT_ROWS)) return cudaErrorInvalidValue;
 
-    a.tiles_per_worker = (int)((a.p + TILE_M - 1) / TILE_M);
-    int64_t per_worker = num_sms / a.N;
-    if (per_worker < 1) per_worker = 1;
-    if (per_worker > a.tiles_per_worker) per_worker = a.tiles_per_worker;
-    dim3 grid((unsigned)per_worker, (unsigned)a.N);
-    cudaError_t e;
-    switch (KC) {
-        case 40: e = launch_kc<40>(tin, tout, a, tp, smem, grid, s); break;
-        case 32: e = launch_kc<32>(tin, tout, a, tp, smem, grid, s); break;
-        case 24: e = launch_kc<24>(tin, tout, a, tp, smem, grid, s); break;
-        default: e = launch_kc<16>(tin, tout, a, tp, smem, grid, s); break;
-    }
+    tp.tiles_per_worker = (a.p + tile_w - 1) / tile_w;
+    tp.total_tiles = tp.tiles_per_worker * a.N;
+    int grid = num_sms;
+    if ((int64_t)grid > tp.total_tiles) grid = (int)tp.total_tiles;
+    cudaError_t e = halves == 2 ? launch_halves<2>(KC, tin, tout, a, tp, smem, grid, s)
+                                : launch_halves<1>(KC, tin, tout, a, tp, smem, grid, s);
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }

@@ -296,10 +296,6 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     if (mode == KERNEL_TC && !tc_eligible(a)) return cudaErrorInvalidValue;
     // automatic choice: the FMA kernel is HBM-bound below c ~ 32; from there on only the tensor cores keep up
     if (mode == KERNEL_TC || (mode == KERNEL_AUTO && a.J >= 32 && tc_eligible(a))) {
-        // tc_variant: 0 = tiles of 256 positions where they fit (c <= 64; measured faster than tiles of
-        // 128 inside the pipeline for every shape tried), 1 = always tiles of 128
-        const bool pair = g_tune_tc_variant != 1 && tc_pair_eligible(a);
-        if (pair) return launch_contract_tc_pair(a, num_sms, s, launches);
         return launch_contract_tc(a, num_sms, s, launches);
     }
     if (mode == KERNEL_STAGED && !can_stage) return cudaErrorInvalidValue;

@@ -70,9 +70,6 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
 // Tensor-core (tcgen05, 3 x TF32) contraction; tc_eligible says whether the shape fits it.
 bool tc_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
-// The same contraction on tiles of 256 positions (1 KB rows in global memory), for c <= 64.
-bool tc_pair_eligible(const ContractArgs& a);
-cudaError_t launch_contract_tc_pair(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
 extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant,
            g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off;
