@@ -19,7 +19,7 @@ import pytest
 
 from oracle import designs as Dz
 from oracle import protocol as P
-from tests._harness import rel_l2, run_library, run_oracle
+from tests._harness import rel_l2, run_library, run_oracle, torch_stream
 
 pytestmark = pytest.mark.gpu
 
@@ -430,3 +430,40 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_survives(cerar_mod):
     _check_stages(res, ora, OUT_TOL, N)
     with pytest.raises(cerar_mod.CerarError):
         plan.selftest_wait_timeout(0)
+
+
+def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
+    """Seeded random (N, c, p, tiling): chunk counts, A-buffer counts, segment boundaries and
+    tails of the tensor-core kernel vary with all of them; its result must stay within 3 x TF32
+    accuracy of the FMA kernel's (checked against the oracle elsewhere), with nothing left
+    unwritten."""
+    import torch
+    rng = np.random.default_rng(2024)
+    s = torch_stream()
+    try:
+        for trial in range(48):
+            N = int(rng.integers(2, 17))
+            c = max(N, int(rng.choice([32, 36, 40, 48, 56, 64, 72, 96, 128])))
+            p = int(rng.choice([4, 128, 132, 256, 260, 1028, 4104, 20000, 65540]))
+            variant = int(rng.choice([0, 0, 1, 2, 3]))
+            d = c * p
+            des = Dz.custom_orthogonal(N, c, np.random.default_rng(trial))
+            g = torch.randn(N * d, device="cuda")
+            outs = {}
+            for mode, v in ((cerar_mod.KERNEL_TC, variant), (cerar_mod.KERNEL_STAGED, 0)):
+                cerar_mod.cerar_set_tuning("tc_variant", v)
+                plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+                plan.set_kernel_mode(mode)
+                ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
+                out = torch.full((N * d,), float("nan"), device="cuda")
+                for _ in range(2):
+                    plan.allreduce_sim(g, d, out, d, ws, d, 0.5, s)
+                torch.cuda.synchronize()
+                plan.device_status(s)
+                outs[mode] = out
+                plan.destroy()
+            a, b = outs[cerar_mod.KERNEL_TC], outs[cerar_mod.KERNEL_STAGED]
+            assert bool(torch.isfinite(a).all()), (N, c, p, variant)
+            assert float((a - b).norm() / b.norm()) < 3e-6, (N, c, p, variant)
+    finally:
+        cerar_mod.cerar_set_tuning("tc_variant", 0)
