@@ -69,3 +69,53 @@ def test_config4_full_size_sampled():
     print("\n[cfg4 full size]", res)
     assert res["rel_l2_Y"] < 2e-6
     assert res["rel_l2_out_max"] < max(1e-4, 4 * kap * U32)
+
+
+def test_config3_full_size_one_worker_per_rank_fused_rounds():
+    """Config 3 at full size through the one-worker-per-rank calls, in place (eight separate
+    45 + 13 GB workspaces; the rounds in one cooperative launch, ordered per tile by counters):
+    the observations and the outputs on sampled positions against the oracle."""
+    import torch
+    from paper_2609_23898_b200 import cerar, inputs, ring
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70e9:
+        pytest.skip("needs 70 GB of device memory")
+    cfg = dict(inputs.CONFIGS["cfg3"])
+    N, c, d = cfg["N"], cfg["c"], cfg["d"]
+    p, L = d // c, c + N - 2
+    B = inputs.base_matrix(N, c, 0)
+    des = Dz.epsilon(N, c, cfg["param"], B)
+    plan = cerar.Plan.create(N, c, cerar.EPSILON, cfg["param"], B=B)
+    r = ring.LocalRing(plan, d)
+    grads = [r.grad_view(i) for i in range(N)]
+    inputs.fill_gradients_torch(grads, cfg["workload"], seed=0, std=cfg["std"]) if "std" in cfg else \
+        inputs.fill_gradients_torch(grads, cfg["workload"], seed=0)
+    # sampled positions: a few tiles of the counters' grid, first and last included
+    rng = np.random.default_rng(5)
+    tile = 256
+    starts = sorted({0, p - tile} | {int(x) for x in rng.integers(0, p - tile, 6)})
+    idx = torch.from_numpy(np.concatenate([np.arange(a, a + tile) for a in starts])).cuda()
+    rows = c + N + 1
+    g_sub = np.stack([r.ws[i].view(rows, p)[N + 1:N + 1 + c][:, idx].reshape(-1).cpu().numpy() for i in range(N)])
+    s = torch.cuda.current_stream().cuda_stream
+    r.encode(grads, s)
+    r.rounds_fused(s)
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    ys = ring.y_slots(plan)
+    Y_dev = np.stack([r.ws[i].view(rows, p)[ys][:, idx].cpu().numpy() for i in range(N)])
+    r.decode(grads, 1.0 / N, s)                       # in place: the D rows receive the result
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    out_dev = np.stack([grads[i].view(c, p)[:, idx].reshape(-1).cpu().numpy() for i in range(N)])
+    ora = P.allreduce([x.astype(np.float64) for x in g_sub], des.U, des.R, 1.0 / N)
+    Y_ora = np.stack([ora["Y"][i].T for i in range(N)])
+    kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+    err_y = P.rel_l2(Y_dev, Y_ora)
+    err_out = max(P.rel_l2(out_dev[i], ora["out"][i]) for i in range(N))
+    print("\n[cfg3 full size, rank-level, fused rounds]", {"positions": int(idx.numel()), "rel_l2_Y": err_y,
+                                                            "rel_l2_out_max": err_out, "kappa_M": kap})
+    assert err_y < 2e-6
+    assert err_out < 4 * kap * U32
+    del r, grads
+    torch.cuda.empty_cache()
