@@ -189,7 +189,9 @@ def run_reference(args, cfg):
     N, c, d = cfg["N"], cfg["c"], cfg["d"]
     B = inputs.base_matrix(N, c, 0)
     des = build_design_oracle(cfg, B)
-    p_sample = min(d // c, args.ref_positions)
+    # a bounded sample per step, sized so that the whole run (K steps + W short warm-ups) stays
+    # within a few minutes whatever K is: about ten steps' worth of --ref-positions in total
+    p_sample = min(d // c, args.ref_positions, max(4096, (10 * args.ref_positions) // max(1, args.steps)))
     for _ in range(args.warmup):
         cpu_baseline(cfg, des, max(1, p_sample // 8))
     times, base = [], None
@@ -232,8 +234,8 @@ def workload_name(key, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3")
     ap.add_argument("--d", type=int, default=0, help="override d per worker (multiple of c)")
