@@ -213,3 +213,56 @@ def test_randomised_ring_shapes(mods):
                 assert worst < 1e-5, (N, c, p, tile, fused, worst)
     finally:
         cerar.cerar_set_tuning("ring_tile", 0)
+
+
+def test_rank_level_kernels_on_symmetric_memory_allocations(mods):
+    """DistributedRing keeps workspaces and counters in torch's symmetric memory.  With one GPU
+    the peer mapping cannot be exercised, but the allocations can: a one-rank NCCL group,
+    every worker's workspace and the counters from symm_mem.empty + rendezvous (as the driver
+    does, buffers taken through the handle), then the rank-level kernels and the fused rounds
+    on them, against the oracle."""
+    import os
+    import torch
+    import torch.distributed as dist
+    cerar, inputs, ring = mods
+    try:
+        import torch.distributed._symmetric_memory as symm_mem
+    except Exception as e:                                    # pragma: no cover
+        pytest.skip(f"no symmetric memory in this torch: {e}")
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29541")
+    created = not dist.is_initialized()
+    if created:
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        N, c, p = 4, 8, 8192 * 2 + 516
+        d = c * p
+        des = Dz.custom_orthogonal(N, c, np.random.default_rng(8))
+        plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+        g = inputs.gradients_numpy(N, d, "normal", seed=9)
+        ora = run_oracle(des.U, des.R, g, 1.0)
+        s = torch.cuda.current_stream().cuda_stream
+        n, nt = plan.rank_workspace_bytes(d) // 4, plan.ring_tiles(d)
+        dev = torch.device("cuda", 0)
+        r = ring.LocalRing(plan, d)
+        keep = []
+        for i in range(N):
+            t = symm_mem.empty(n, dtype=torch.float32, device=dev)
+            h = symm_mem.rendezvous(t, dist.group.WORLD)
+            r.ws[i] = h.get_buffer(0, (n,), torch.float32)
+            keep.append((t, h))
+        cnt = symm_mem.empty(2 * N * nt, dtype=torch.int32, device=dev)
+        cnt.zero_()
+        hc = symm_mem.rendezvous(cnt, dist.group.WORLD)
+        r.counters = hc.get_buffer(0, (2 * N * nt,), torch.int32)
+        grads = [torch.from_numpy(g[i]).cuda() for i in range(N)]
+        outs = [torch.empty(d, device="cuda") for _ in range(N)]
+        for fused in (False, True, True):
+            r.allreduce(grads, outs, 1.0, s, fused=fused)
+            keep[0][1].barrier(channel=0, timeout_ms=5000)     # the driver's stream barrier, one rank
+            torch.cuda.synchronize()
+            plan.device_status(s)
+            assert max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
+    finally:
+        if created:
+            dist.destroy_process_group()
