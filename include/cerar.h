@@ -214,7 +214,7 @@ cerar_status_t cerar_allreduce_fused(cerar_plan_t* plan, const float* grads, int
 int            cerar_fused_supported(const cerar_plan_t* plan);
 
 /* ---- One worker per GPU (the ring the paper runs between machines, Sec. II and
- * Algorithm 1; its Sec. V names the fused compute/transfer form as future work).
+ * Algorithm 1; its Sec. IV names the fused compute/transfer form as future work).
  * Each call serves ONE worker `rank` in 0..N-1, whose state is its own workspace of
  * cerar_rank_workspace_bytes(plan, d) = (c+N+1) (d/c) 4 bytes on this GPU: row
  * ("slot") k-1 receives message k, slot N+j holds delta_{rank,j}.  The one row more
