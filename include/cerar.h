@@ -18,6 +18,10 @@
  *     data-path calls (encode, ring_round, decode, allreduce_sim).
  *   - Data-path calls are asynchronous on the given stream and report
  *     argument and launch errors only.  Nothing throws across this boundary.
+ *   - A plan is not synchronised internally: calls on the SAME plan from several
+ *     host threads must be serialised by the caller (its round state, counters and
+ *     status word are per plan); different plans are independent.  The tuning
+ *     knobs (cerar_set_tuning) are process-wide and meant to be set before use.
  *   - All matrices are row-major.  Gradients are fp32 on the device; the
  *     coefficient matrices are built in fp64 on the host and rounded to fp32
  *     for the device.
