@@ -289,33 +289,46 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    for _ in range(args.warmup):
-        plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
-    torch.cuda.synchronize()
-    plan.device_status(stream)
-    if sampler:
-        sampler.wait_first_sample()
-
-    # ---- timed region: K steps, each the C-ABI sequence encode, rounds 1..L, decode
     K = args.steps
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 3)] for _ in range(K)]
-    sync_all()
-    launches0 = plan.launch_count()
-    for s in range(K):
-        e = ev[s]
-        e[0].record()
-        plan.encode(grads, d, ws, d, stream)
-        e[1].record()
-        for k in range(1, L + 1):
-            plan.ring_round(ws, d, k, stream)
-            e[1 + k].record()
-        plan.decode(ws, out, d, d, scale, stream)
-        e[L + 2].record()
-    sync_all()
-    launches = plan.launch_count() - launches0
-    clocks = sampler.stop() if sampler else None
-    plan.device_status(stream)
+    THERMAL = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+
+    def measure():
+        """W warm-ups, then the timed region: K steps, each the C-ABI sequence encode, rounds 1..L,
+        decode, with a CUDA event after every call and the clocks sampled alongside."""
+        sampler = ClockSampler(local_rank) if rank == 0 else None
+        for _ in range(args.warmup):
+            plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
+        torch.cuda.synchronize()
+        plan.device_status(stream)
+        if sampler:
+            sampler.wait_first_sample()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 3)] for _ in range(K)]
+        sync_all()
+        launches0 = plan.launch_count()
+        for s in range(K):
+            e = ev[s]
+            e[0].record()
+            plan.encode(grads, d, ws, d, stream)
+            e[1].record()
+            for k in range(1, L + 1):
+                plan.ring_round(ws, d, k, stream)
+                e[1 + k].record()
+            plan.decode(ws, out, d, d, scale, stream)
+            e[L + 2].record()
+        sync_all()
+        launches = plan.launch_count() - launches0
+        clocks = sampler.stop() if sampler else None
+        plan.device_status(stream)
+        return ev, launches, clocks
+
+    ev, launches, clocks = measure()
+    remeasured = False
+    if clocks and THERMAL & set(clocks.get("reasons", [])) and world == 1:
+        # a thermal or hardware slowdown during the timed region: the number is not usable; once more
+        first = clocks
+        ev, launches, clocks = measure()
+        clocks["first_attempt_reasons"] = first["reasons"]
+        remeasured = True
     total_ms = ev[0][0].elapsed_time(ev[K - 1][L + 2])
     enc_ms = float(np.mean([ev[s][0].elapsed_time(ev[s][1]) for s in range(K)]))
     dec_ms = float(np.mean([ev[s][L + 1].elapsed_time(ev[s][L + 2]) for s in range(K)]))
@@ -357,7 +370,7 @@ def main():
                        "scale": "1/N", "replicas": world, "l2": "inputs larger than L2" if ab["total"] / (L + 2) > 2.6e8
                        else "working set may be L2 resident",
                        "buffers": "out of place: grads, workspace and output are separate device buffers"},
-            "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks}
+            "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks, "remeasured": remeasured}
 
     # ---- the same K aggregations through the one-call entry point, one event pair around all of
     # them: no event between the launches, so consecutive kernels overlap their launch with the
