@@ -346,6 +346,7 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "ring_tile"                     positions per tile of the fused ring rounds (a multiple of 4;
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters
  *   "pdl_off"                       1 = launch without programmatic stream serialization
+ *   "serpentine_off"                1 = every ring round walks the positions upwards
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

@@ -287,7 +287,7 @@ cerar_status_t cerar_ring_round(cerar_plan_t* P, float* ws, int64_t d, int k, ce
     if (!ws) return fail(CERAR_ERR_INVALID_ARG, "ws is NULL");
     if (!P->encoded || d != P->cur_d) return fail(CERAR_ERR_STATE, "encode (with the same d) must come first");
     if (k != P->rounds_done + 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "rounds must run in order 1..L");
-    cerar::RoundArgs a{ws, p, P->host.N, P->host.c, k};
+    cerar::RoundArgs a{ws, p, P->host.N, P->host.c, k, 0};
     cudaError_t e = cerar::launch_round(a, (cudaStream_t)stream, &P->launches);
     if (e != cudaSuccess) return cuda_fail(e, "round launch");
     P->rounds_done = k;
@@ -625,6 +625,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "tc_variant") cerar::g_tune_tc_variant = value;
     else if (n == "ring_wait_ms") cerar::g_tune_ring_wait_ms = value;
     else if (n == "pdl_off") cerar::g_tune_pdl_off = value;
+    else if (n == "serpentine_off") cerar::g_tune_serpentine_off = value;
     else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;
