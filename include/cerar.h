@@ -141,6 +141,14 @@ cerar_status_t cerar_plan_info(cerar_plan_t* plan, cerar_plan_info_t* out);
 cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, const double* h,
                                   double* gamma_out);
 
+/* Smallest d' >= d that is a multiple of 4c.  The protocol needs c | d (the caller pads the
+ * gradient with zeros, Sec. II); the fast kernels additionally need rows of p = d/c values to
+ * start on 16-byte boundaries, i.e. 4 | p.  With c | d but p not a multiple of 4 every call
+ * still works, through kernels with plain 4-byte accesses at about half the speed for
+ * c <= 32 and less beyond (no tensor cores there): pad to this length instead (zeros in, the
+ * padded tail of the result is zero as well). */
+int64_t        cerar_padded_length(const cerar_plan_t* plan, int64_t d);
+
 /* Bytes of the device workspace for gradient length d: 4 * N * (c+N) * (d/c);
  * 0 if c does not divide d. */
 size_t cerar_workspace_bytes(const cerar_plan_t* plan, int64_t d);

@@ -70,6 +70,8 @@ lib.cerar_plan_get_R.argtypes = [_vp, C.c_int, C.POINTER(C.c_double)]
 lib.cerar_plan_info.argtypes = [_vp, C.POINTER(PlanInfo)]
 lib.cerar_design_gamma.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.c_uint64, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double)]
+lib.cerar_padded_length.argtypes = [_vp, _i64]
+lib.cerar_padded_length.restype = _i64
 lib.cerar_workspace_bytes.argtypes = [_vp, _i64]
 lib.cerar_workspace_bytes.restype = C.c_size_t
 lib.cerar_encode.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _vp]
@@ -203,6 +205,10 @@ class Plan:
         s = PlanInfo()
         _check(lib.cerar_plan_info(self._h, C.byref(s)))
         return {f: getattr(s, f) for f, _ in PlanInfo._fields_}
+
+    def padded_length(self, d: int) -> int:
+        """Smallest d' >= d with 4c | d' (what the fast kernels want; pad the gradient with zeros)."""
+        return int(lib.cerar_padded_length(self._h, d))
 
     def workspace_bytes(self, d: int) -> int:
         return lib.cerar_workspace_bytes(self._h, d)

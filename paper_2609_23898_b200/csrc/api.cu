@@ -256,6 +256,12 @@ cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, 
     return CERAR_OK;
 }
 
+int64_t cerar_padded_length(const cerar_plan_t* P, int64_t d) {
+    if (!P || d <= 0) return 0;
+    const int64_t q = 4 * (int64_t)P->host.c;
+    return (d + q - 1) / q * q;
+}
+
 size_t cerar_workspace_bytes(const cerar_plan_t* P, int64_t d) {
     if (!P || d <= 0 || d % P->host.c != 0) return 0;
     return (size_t)4 * P->host.N * (size_t)(P->host.c + P->host.N) * (size_t)(d / P->host.c);

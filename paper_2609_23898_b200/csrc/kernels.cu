@@ -36,6 +36,58 @@ __global__ void contract_ref_kernel(const ContractArgs a) {
     for (int j = 0; j < a.J; ++j) out[(int64_t)j * a.out_rstride] = acc[j] * a.scale;
 }
 
+// ------------------------------------------------------------------ tiled contraction, any alignment
+//
+// For shapes whose rows do not start on 16-byte boundaries (p not a multiple of 4), where
+// neither vector loads nor bulk copies apply.  A block stages all K input rows of its TP
+// positions in shared memory with plain coalesced 4-byte loads, then every thread (one
+// position) forms the J outputs eight at a time from shared memory; the coefficients sit
+// in shared memory too, padded to a multiple of 8 columns so that they are read as two
+// 16-byte broadcasts per input row.  All inputs of the tile are read before its first
+// output is stored, so in-place use stays safe.
+__global__ void __launch_bounds__(256) contract_tile_kernel(const ContractArgs a) {
+    extern __shared__ __align__(16) float tile_smem[];
+    const int TP = blockDim.x;
+    const int Jpad = (a.J + 7) / 8 * 8;
+    float* coef_s = tile_smem;                        // K x Jpad
+    float* in_s = tile_smem + (size_t)a.K * Jpad;     // K x TP
+    const int w = blockIdx.y;
+    const int64_t q = (int64_t)blockIdx.x * TP + threadIdx.x;
+    const float* cf = a.coef + (size_t)w * a.K * a.J;
+    for (int idx = threadIdx.x; idx < a.K * Jpad; idx += TP) {
+        const int k = idx / Jpad, j = idx - k * Jpad;
+        coef_s[idx] = (j < a.J) ? cf[(size_t)k * a.J + j] : 0.f;
+    }
+    grid_dependency_wait();                           // the coefficients above are constants of the plan
+    if (q < a.p) {
+        const float* in = a.in + (int64_t)w * a.in_wstride + q;
+        for (int k = 0; k < a.K; ++k) {
+            const int row = (k < a.skip_row) ? k : k + a.skip_count;
+            in_s[(size_t)k * TP + threadIdx.x] = in[(int64_t)row * a.in_rstride];
+        }
+    }
+    __syncthreads();
+    if (q >= a.p) return;
+    float* out = a.out + (int64_t)w * a.out_wstride + q;
+    for (int jc = 0; jc < a.J; jc += 8) {
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        for (int k = 0; k < a.K; ++k) {
+            const float x = in_s[(size_t)k * TP + threadIdx.x];
+            const float4 c0 = *reinterpret_cast<const float4*>(coef_s + (size_t)k * Jpad + jc);
+            const float4 c1 = *reinterpret_cast<const float4*>(coef_s + (size_t)k * Jpad + jc + 4);
+            acc[0] = fmaf(c0.x, x, acc[0]); acc[1] = fmaf(c0.y, x, acc[1]);
+            acc[2] = fmaf(c0.z, x, acc[2]); acc[3] = fmaf(c0.w, x, acc[3]);
+            acc[4] = fmaf(c1.x, x, acc[4]); acc[5] = fmaf(c1.y, x, acc[5]);
+            acc[6] = fmaf(c1.z, x, acc[6]); acc[7] = fmaf(c1.w, x, acc[7]);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (jc + j < a.J) out[(int64_t)(jc + j) * a.out_rstride] = acc[j] * a.scale;
+    }
+}
+
 // ------------------------------------------------------------------ staged contraction
 //
 // grid = (CTAs per worker, N).  CTA (b, w) walks tiles b, b+gridDim.x, ... of
@@ -347,6 +399,20 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
         }
     }
     if (mode == KERNEL_STAGED) return cudaErrorInvalidConfiguration;
+    if (mode != KERNEL_REF) {
+        // unaligned rows: positions tiled through shared memory with plain loads
+        int tp = 256;
+        size_t smem = ((size_t)a.K * ((a.J + 7) / 8 * 8) + (size_t)a.K * tp) * sizeof(float);
+        while (smem > 200 * 1024 && tp > 32) { tp /= 2; smem = ((size_t)a.K * ((a.J + 7) / 8 * 8) + (size_t)a.K * tp) * sizeof(float); }
+        if (smem <= 200 * 1024) {
+            cudaError_t es = cudaFuncSetAttribute(contract_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (es != cudaSuccess) return es;
+            dim3 grid((unsigned)((a.p + tp - 1) / tp), (unsigned)a.N);
+            es = launch_pdl(contract_tile_kernel, grid, dim3(tp), smem, s, a);
+            if (es == cudaSuccess && launches) ++*launches;
+            return es;
+        }
+    }
     if (a.J > REF_MAX_J) return cudaErrorInvalidValue;
     const int threads = 128;
     dim3 grid((unsigned)((a.p + threads - 1) / threads), (unsigned)a.N);

@@ -202,3 +202,13 @@ def test_library_kappa_design_reaches_phi_zero_when_c_equals_N():
         p = cerar.Plan.create(N, N, cerar.KAPPA, C, B=B, als_iters=1000, als_tol=1e-30, host_only=True)
         info = p.info()
         assert info["phi"] < 1e-18 and info["kappa_M_max"] <= C
+
+
+def test_padded_length():
+    from oracle import designs as Dz
+    from paper_2609_23898_b200 import cerar
+    des = Dz.custom_orthogonal(4, 12, np.random.default_rng(0))
+    plan = cerar.Plan.create_custom(4, 12, des.U, des.R, host_only=True)
+    assert plan.padded_length(1_414_647_808) == 1_414_647_840 and 1_414_647_840 % 48 == 0
+    assert plan.padded_length(48) == 48 and plan.padded_length(49) == 96 and plan.padded_length(1) == 48
+    assert plan.padded_length(0) == 0
