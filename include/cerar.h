@@ -355,6 +355,7 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters
  *   "pdl_off"                       1 = launch without programmatic stream serialization
  *   "serpentine_off"                1 = every ring round walks the positions upwards
+ *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24)
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

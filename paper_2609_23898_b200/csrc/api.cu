@@ -632,6 +632,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "ring_wait_ms") cerar::g_tune_ring_wait_ms = value;
     else if (n == "pdl_off") cerar::g_tune_pdl_off = value;
     else if (n == "serpentine_off") cerar::g_tune_serpentine_off = value;
+    else if (n == "tc_min_c") cerar::g_tune_tc_min_c = value;
     else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;

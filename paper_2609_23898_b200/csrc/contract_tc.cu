@@ -2,7 +2,7 @@
 //
 //   out[j][q] = scale * sum_k coef[k][j] * in[k][q],   j < J (= c),  k < K rows,  q < p
 //
-// is a skinny GEMM with M = positions, N = J, K = input rows.  At c >= 32 the FP32 FMA pipe
+// is a skinny GEMM with M = positions, N = J, K = input rows.  From c ~ 24 on the FP32 FMA pipe
 // cannot keep up with HBM (c/4 flop per byte), so the products run on the 5th-generation
 // tensor cores as 3 x TF32: every fp32 value is split into hi = tf32(x), lo = tf32(x - hi) and
 //   x*y ~ lo_x*hi_y + hi_x*lo_y + hi_x*hi_y           (relative error ~ 2^-22),
@@ -377,10 +377,12 @@ int choose_chunk(const ContractArgs& a, int halves, PairParams* tp) {
 
 }  // namespace
 
-int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_variant = 0;
+int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_variant = 0, g_tune_tc_min_c = 0;
 
 bool tc_eligible(const ContractArgs& a) {
-    if (a.J < 32 || a.J > 128) return false;      // N = J padded to 32; two coefficient copies must fit in smem
+    // N = J padded to 32 (rows beyond J are clipped by the output map); measured against the FMA kernel
+    // on B200: +40 % at c = 28, +5 % at c = 24, -15 % at c = 20.  Two coefficient copies must fit in smem.
+    if (a.J < (g_tune_tc_min_c > 0 ? g_tune_tc_min_c : 24) || a.J > 128) return false;
     if (a.p % 4 != 0 || a.p >= (int64_t)1 << 31) return false;
     if ((reinterpret_cast<uintptr_t>(a.in) & 15u) || (a.in_rstride % 4) || (a.in_wstride % 4)) return false;
     if ((reinterpret_cast<uintptr_t>(a.out) & 15u) || (a.out_rstride % 4) || (a.out_wstride % 4)) return false;

@@ -349,8 +349,8 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     bool can_stage = (a.p % 4 == 0) && aligned16(a.in) && aligned16(a.out) && (a.in_wstride % 4 == 0) &&
                      (a.out_wstride % 4 == 0) && (a.in_rstride % 4 == 0) && (a.out_rstride % 4 == 0);
     if (mode == KERNEL_TC && !tc_eligible(a)) return cudaErrorInvalidValue;
-    // automatic choice: the FMA kernel is HBM-bound below c ~ 32; from there on only the tensor cores keep up
-    if (mode == KERNEL_TC || (mode == KERNEL_AUTO && a.J >= 32 && tc_eligible(a))) {
+    // automatic choice: the FMA kernel is HBM-bound below c ~ 24; from there on only the tensor cores keep up
+    if (mode == KERNEL_TC || (mode == KERNEL_AUTO && tc_eligible(a))) {
         return launch_contract_tc(a, num_sms, s, launches);
     }
     if (mode == KERNEL_STAGED && !can_stage) return cudaErrorInvalidValue;

@@ -4,7 +4,7 @@ element on the same seeded inputs.
 Tolerances.  The device computes in fp32: encode and decode are dot products
 of length c and L+1, the rounds add at most N terms.  With unit roundoff
 u = 2^-24 the relative L2 deviation of a well-conditioned stage is a few u
-(observed ~1e-7 with the FMA kernel); for c >= 32 the products run on the
+(observed ~1e-7 with the FMA kernel); for c >= 24 the products run on the
 tensor cores as 3 x TF32 (per-product error about 2^-22, fp32 accumulation;
 observed 2.4e-7 at c=32 up to 9e-7 at c=128).  The tests allow 2e-6 for every
 stage taken alone (encode
@@ -102,7 +102,7 @@ def test_staged_kernel_is_what_runs(cerar_mod):
 
 def test_tensor_core_kernel_is_what_runs(cerar_mod):
     """Forcing the tensor-core kernel works on an eligible shape (so that 'auto' at
-    c >= 32 is not silently the FMA kernel), agrees with the FMA kernel to TF32x3
+    c >= 24 is not silently the FMA kernel), agrees with the FMA kernel to TF32x3
     accuracy, and refuses shapes it cannot take."""
     N, c, p = 8, 32, 2048 + 132
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(3))

@@ -66,7 +66,7 @@ def test_local_ring_matches_oracle_and_batched_pipeline(mods, N, c, p, inplace):
     ref = run_library(cerar.Plan.create_custom(N, c, des.U, des.R), g, 0.5)
     assert np.array_equal(delta, ref["Delta"])
     assert np.array_equal(Y, ref["Y"])
-    if c < 32:
+    if c < 24:
         assert np.array_equal(out, ref["out"])
     else:
         # tensor-core decode: the two spent rows shift which inputs share a K = 8 product, and the
