@@ -229,8 +229,12 @@ def test_rank_level_kernels_on_symmetric_memory_allocations(mods):
         import torch.distributed._symmetric_memory as symm_mem
     except Exception as e:                                    # pragma: no cover
         pytest.skip(f"no symmetric memory in this torch: {e}")
+    import socket
     os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-    os.environ.setdefault("MASTER_PORT", "29541")
+    if "MASTER_PORT" not in os.environ:
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            os.environ["MASTER_PORT"] = str(sk.getsockname()[1])
     created = not dist.is_initialized()
     if created:
         dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
