@@ -345,7 +345,7 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
 
 /* Process-wide tuning knobs, for experiments and tests; value 0 restores the default.
  *   "kc", "stages", "jt", "slabs"   staged FMA kernel: input rows per pipeline stage, stages,
- *                                   outputs per thread (4, 8 or 16), position slabs per CTA
+ *                                   outputs per thread (4, 8, 16 or 20), position slabs per CTA
  *   "tc_kc", "tc_stages"            tensor-core kernels: rows per stage, stages
  *   "tc_variant"                    1 = always tiles of 128 positions (default: tiles of 256
  *                                   positions for c <= 64); 2 / 3 = tiles of 256 with one /
