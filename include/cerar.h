@@ -189,6 +189,15 @@ cerar_status_t cerar_encode(cerar_plan_t* plan, const float* grads, int64_t grad
                             float* ws, int64_t d, cerar_stream_t stream);
 cerar_status_t cerar_ring_round(cerar_plan_t* plan, float* ws, int64_t d, int k,
                                 cerar_stream_t stream);
+/* Rounds k_first .. k_last (k_first must follow the last completed round) in ONE launch: a thread
+ * owns its positions for all N workers, so it runs their rounds one after the other without any
+ * ordering against other threads.  Same stores into the neighbours' slots, same results bit for
+ * bit, same counters; but a message may be read back from cache instead of HBM, so for a
+ * workspace larger than the L2 this is not the HBM hand-off that cerar_ring_round performs.
+ * cerar_allreduce_sim uses it on its own for workspaces up to 64 MB, which never leave the L2
+ * and are bound by the L launches otherwise. */
+cerar_status_t cerar_ring_rounds(cerar_plan_t* plan, float* ws, int64_t d, int k_first, int k_last,
+                                 cerar_stream_t stream);
 cerar_status_t cerar_decode(cerar_plan_t* plan, const float* ws, float* out, int64_t out_stride,
                             int64_t d, float scale, cerar_stream_t stream);
 cerar_status_t cerar_allreduce_sim(cerar_plan_t* plan, const float* grads, int64_t grads_stride,
@@ -356,6 +365,7 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "pdl_off"                       1 = launch without programmatic stream serialization
  *   "serpentine_off"                1 = every ring round walks the positions upwards
  *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24)
+ *   "rounds_one_launch_off"         1 = cerar_allreduce_sim always launches round by round
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

@@ -76,6 +76,7 @@ lib.cerar_workspace_bytes.argtypes = [_vp, _i64]
 lib.cerar_workspace_bytes.restype = C.c_size_t
 lib.cerar_encode.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _vp]
 lib.cerar_ring_round.argtypes = [_vp, _f32p, _i64, C.c_int, _vp]
+lib.cerar_ring_rounds.argtypes = [_vp, _f32p, _i64, C.c_int, C.c_int, _vp]
 lib.cerar_decode.argtypes = [_vp, _f32p, _f32p, _i64, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
 lib.cerar_allreduce_sim_host.argtypes = [_vp, _f32p, _i64, _f32p, _i64, _f32p, _i64, C.c_float, _vp]
@@ -236,6 +237,10 @@ class Plan:
 
     def ring_round(self, ws, d, k, stream=0):
         _check(lib.cerar_ring_round(self._h, _ptr(ws), d, k, stream))
+
+    def ring_rounds(self, ws, d, k_first, k_last, stream=0):
+        """cerar_ring_rounds: rounds k_first..k_last in one launch."""
+        _check(lib.cerar_ring_rounds(self._h, _ptr(ws), d, k_first, k_last, stream))
 
     def decode(self, ws, out, out_stride, d, scale=1.0, stream=0):
         _check(lib.cerar_decode(self._h, _ptr(ws), _ptr(out), out_stride, d, scale, stream))

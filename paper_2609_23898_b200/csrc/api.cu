@@ -102,6 +102,9 @@ cerar_status_t finish_create(cerar_plan* P, bool host_only, cerar_plan_t** out) 
     return CERAR_OK;
 }
 
+// cerar_allreduce_sim runs all rounds in one launch up to this workspace size (half of the 126 MB L2)
+constexpr size_t kOneLaunchRoundsBytes = (size_t)64 << 20;
+
 cerar_status_t check_data_call(const cerar_plan* P, int64_t d, int64_t* p_out) {
     if (!P) return fail(CERAR_ERR_INVALID_ARG, "plan is NULL");
     if (!P->on_device) return fail(CERAR_ERR_CUDA, "plan has no device copies (no CUDA device, or host_only)");
@@ -301,6 +304,23 @@ cerar_status_t cerar_ring_round(cerar_plan_t* P, float* ws, int64_t d, int k, ce
     return CERAR_OK;
 }
 
+cerar_status_t cerar_ring_rounds(cerar_plan_t* P, float* ws, int64_t d, int k_first, int k_last,
+                                 cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws) return fail(CERAR_ERR_INVALID_ARG, "ws is NULL");
+    if (!P->encoded || d != P->cur_d) return fail(CERAR_ERR_STATE, "encode (with the same d) must come first");
+    if (k_first != P->rounds_done + 1 || k_last < k_first || k_last > P->host.L)
+        return fail(CERAR_ERR_STATE, "rounds must run in order 1..L");
+    cerar::RoundArgs a{ws, p, P->host.N, P->host.c, k_first, 0};
+    cudaError_t e = cerar::launch_rounds_multi(a, k_last, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rounds launch");
+    P->rounds_done = k_last;
+    P->bytes_forwarded += (uint64_t)4 * (uint64_t)p * (uint64_t)(k_last - k_first + 1);
+    return CERAR_OK;
+}
+
 cerar_status_t cerar_decode(cerar_plan_t* P, const float* ws, float* out, int64_t out_stride, int64_t d,
                             float scale, cerar_stream_t stream) {
     int64_t p;
@@ -328,8 +348,14 @@ cerar_status_t cerar_allreduce_sim(cerar_plan_t* P, const float* grads, int64_t 
                                    int64_t out_stride, float* ws, int64_t d, float scale, cerar_stream_t stream) {
     cerar_status_t st = cerar_encode(P, grads, grads_stride, ws, d, stream);
     if (st != CERAR_OK) return st;
-    for (int k = 1; k <= P->host.L; ++k)
-        if ((st = cerar_ring_round(P, ws, d, k, stream)) != CERAR_OK) return st;
+    // A state that lives in the L2 anyway (hand-offs never reach HBM in either form) is bound by the
+    // L launches of the round-by-round form: run its rounds in one launch.
+    if (cerar_workspace_bytes(P, d) <= kOneLaunchRoundsBytes && !cerar::g_tune_rounds_one_launch_off) {
+        if ((st = cerar_ring_rounds(P, ws, d, 1, P->host.L, stream)) != CERAR_OK) return st;
+    } else {
+        for (int k = 1; k <= P->host.L; ++k)
+            if ((st = cerar_ring_round(P, ws, d, k, stream)) != CERAR_OK) return st;
+    }
     return cerar_decode(P, ws, out, out_stride, d, scale, stream);
 }
 
@@ -633,6 +659,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "pdl_off") cerar::g_tune_pdl_off = value;
     else if (n == "serpentine_off") cerar::g_tune_serpentine_off = value;
     else if (n == "tc_min_c") cerar::g_tune_tc_min_c = value;
+    else if (n == "rounds_one_launch_off") cerar::g_tune_rounds_one_launch_off = value;
     else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;

@@ -257,24 +257,10 @@ __device__ __forceinline__ float4 combine(float4 y, float4 dc, float4 da) {
     return make_float4((y.x - dc.x) + da.x, (y.y - dc.y) + da.y, (y.z - dc.z) + da.z, (y.w - dc.w) + da.w);
 }
 
+// One round k for the position vector at `base` (all N workers), as described above.
 template <typename VT, int WG>
-__global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
-    constexpr int VW = sizeof(VT) / 4;
-    const int64_t nv = a.p / VW;
-    // Even rounds walk the positions downwards: what the round before wrote last is read first,
-    // while it is still in L2 (measured: +0.7 % at p = 2.2e7, +3 % at p = 4e6, nothing lost below).
-    const int64_t blk = a.reverse ? (int64_t)gridDim.x - 1 - blockIdx.x : (int64_t)blockIdx.x;
-    const int64_t v = blk * blockDim.x + threadIdx.x;
-    // Programmatic dependent launch: this grid may be scheduled while the grid before it drains and
-    // touches memory only after that grid has completed.  (Letting the NEXT grid in early, with an
-    // explicit trigger at the top, gained nothing and cost 8 % at N = 16, c = 128.)
-    grid_dependency_wait();
-    if (v >= nv) return;
-    const int N = a.N, c = a.c, k = a.k;
-    const int64_t pv = a.p / VW;                               // row pitch in vectors
-    const int64_t wstride = (int64_t)(c + N) * pv;
+__device__ __forceinline__ void round_body(VT* base, int64_t pv, int64_t wstride, int N, int c, int k) {
     const bool has_prev = k >= 2, has_cancel = (k - 1) >= N, has_add = k <= c;
-    VT* base = reinterpret_cast<VT*>(a.ws) + v;
     const int64_t off_prev = (int64_t)(k - 2) * pv, off_land = (int64_t)(k - 1) * pv,
                   off_add = (int64_t)(N - 1 + k) * pv;
     VT carry = vzero<VT>();
@@ -301,6 +287,41 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
             }
         }
     }
+}
+
+template <typename VT, int WG>
+__global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
+    constexpr int VW = sizeof(VT) / 4;
+    const int64_t nv = a.p / VW;
+    // Even rounds walk the positions downwards: what the round before wrote last is read first,
+    // while it is still in L2 (measured: +0.7 % at p = 2.2e7, +3 % at p = 4e6, nothing lost below).
+    const int64_t blk = a.reverse ? (int64_t)gridDim.x - 1 - blockIdx.x : (int64_t)blockIdx.x;
+    const int64_t v = blk * blockDim.x + threadIdx.x;
+    // Programmatic dependent launch: this grid may be scheduled while the grid before it drains and
+    // touches memory only after that grid has completed.  (Letting the NEXT grid in early, with an
+    // explicit trigger at the top, gained nothing and cost 8 % at N = 16, c = 128.)
+    grid_dependency_wait();
+    if (v >= nv) return;
+    const int64_t pv = a.p / VW;                               // row pitch in vectors
+    round_body<VT, WG>(reinterpret_cast<VT*>(a.ws) + v, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, a.k);
+}
+
+// Rounds k .. k_last in one launch.  A thread owns its positions for all N workers, and a round
+// touches nothing else, so the rounds of one position need no ordering against other threads:
+// each thread simply runs them one after the other (its own stores are visible to its own later
+// loads).  Every message is still stored into the neighbour's slot and read back from there in
+// the next round, but that read may be served from cache, so this form is for states that live
+// in L2 anyway, where the L launches of the round-by-round form cost more than the data movement.
+template <typename VT, int WG>
+__global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, int k_last) {
+    constexpr int VW = sizeof(VT) / 4;
+    const int64_t nv = a.p / VW;
+    const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    grid_dependency_wait();
+    if (v >= nv) return;
+    const int64_t pv = a.p / VW;
+    VT* base = reinterpret_cast<VT*>(a.ws) + v;
+    for (int k = a.k; k <= k_last; ++k) round_body<VT, WG>(base, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, k);
 }
 
 // Nothing ever arrives on this barrier: the bounded wait runs out after limit_ns and the
@@ -342,7 +363,8 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 }  // namespace
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
-int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0;
+int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
+    g_tune_rounds_one_launch_off = 0;
 
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0 || a.N <= 0) return cudaSuccess;
@@ -446,6 +468,29 @@ cudaError_t launch_round(const RoundArgs& a_in, cudaStream_t s, uint64_t* launch
         e = launch_pdl(round_kernel<float4, 4>, dim3(blocks), dim3(threads), 0, s, a);
     } else {
         e = launch_pdl(round_kernel<float, 4>, dim3((unsigned)((a.p + threads - 1) / threads)), dim3(threads), 0, s, a);
+    }
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+cudaError_t launch_rounds_multi(const RoundArgs& a, int k_last, cudaStream_t s, uint64_t* launches) {
+    if (a.p <= 0 || k_last < a.k) return cudaSuccess;
+    // this form is latency-bound (L dependent rounds per thread): spread a small job over all SMs
+    // with narrower accesses and smaller blocks rather than leave most of them idle
+    int threads = 256;
+    const bool vec = (a.p % 4 == 0 && aligned16(a.ws));
+    bool use_vec = vec;
+    if (vec && a.p / 4 >= (int64_t)148 * 256 * 4) threads = 256;
+    else if (vec && a.p / 4 >= (int64_t)148 * 64 * 4) threads = 64;
+    else { use_vec = false; threads = (a.p >= (int64_t)148 * 128 * 2) ? 128 : 64; }
+    cudaError_t e;
+    if (use_vec) {
+        const int64_t nv = a.p / 4;
+        e = launch_pdl(rounds_multi_kernel<float4, 4>, dim3((unsigned)((nv + threads - 1) / threads)), dim3(threads), 0, s,
+                       a, k_last);
+    } else {
+        e = launch_pdl(rounds_multi_kernel<float, 4>, dim3((unsigned)((a.p + threads - 1) / threads)), dim3(threads), 0,
+                       s, a, k_last);
     }
     if (e == cudaSuccess && launches) ++*launches;
     return e;

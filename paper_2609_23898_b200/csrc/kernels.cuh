@@ -73,8 +73,11 @@ bool tc_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
 extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant,
-           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off, g_tune_serpentine_off, g_tune_tc_min_c;
+           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off, g_tune_serpentine_off, g_tune_tc_min_c,
+           g_tune_rounds_one_launch_off;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
+// Rounds a.k .. k_last in one launch (for states that are cache-resident anyway).
+cudaError_t launch_rounds_multi(const RoundArgs& a, int k_last, cudaStream_t s, uint64_t* launches);
 // Slots of the per-worker layout that round k reads (-1 = term absent) and the landing slot
 // in the neighbour's workspace; the one definition that launcher and callers share.
 void rank_round_slots(int N, int c, int k, int* slot_prev, int* slot_cancel, int* slot_add, int* slot_land);

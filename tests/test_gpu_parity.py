@@ -467,3 +467,49 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
             assert float((a - b).norm() / b.norm()) < 3e-6, (N, c, p, variant)
     finally:
         cerar_mod.cerar_set_tuning("tc_variant", 0)
+
+
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (3, 5, 1031), (16, 16, 1028), (2, 2, 4)])
+def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
+    """cerar_ring_rounds (what cerar_allreduce_sim uses for cache-resident states) leaves exactly
+    the slots of L calls of cerar_ring_round, in one go or in pieces, with the same counters."""
+    import torch
+    d = c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(N + c))
+    g = torch.randn(N * d, device="cuda")
+    s = torch_stream()
+    L = c + N - 2
+    res = []
+    for how in ("each", "all", "pieces"):
+        plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+        ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
+        plan.encode(g, d, ws, d, s)
+        if how == "each":
+            for k in range(1, L + 1):
+                plan.ring_round(ws, d, k, s)
+        elif how == "all":
+            plan.ring_rounds(ws, d, 1, L, s)
+        else:
+            cut = max(1, L // 3)
+            plan.ring_rounds(ws, d, 1, cut, s)
+            if cut < L:
+                plan.ring_round(ws, d, cut + 1, s)
+            if cut + 1 < L:
+                plan.ring_rounds(ws, d, cut + 2, L, s)
+            with pytest.raises(cerar_mod.CerarError):
+                plan.ring_rounds(ws, d, 1, L, s)                 # out of order
+        torch.cuda.synchronize()
+        plan.device_status(s)
+        res.append((ws.clone(), plan.counters()))
+    for w, cnt in res[1:]:
+        assert torch.equal(torch.nan_to_num(w, nan=-1.0), torch.nan_to_num(res[0][0], nan=-1.0))
+        assert cnt == res[0][1]
+    # and through the one-call entry point: one launch for the rounds of this small state
+    plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+    out = torch.empty(N * d, device="cuda")
+    ws = torch.empty(N * (c + N) * p, device="cuda")
+    n0 = plan.launch_count()
+    plan.allreduce_sim(g, d, out, d, ws, d, 1.0, s)
+    assert plan.launch_count() - n0 == 3
+    ora = run_oracle(des.U, des.R, g.view(N, d).cpu().numpy(), 1.0)
+    assert max(rel_l2(out.view(N, d)[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
