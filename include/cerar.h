@@ -264,6 +264,12 @@ cerar_status_t cerar_rank_encode(cerar_plan_t* plan, int rank, const float* grad
                                  cerar_stream_t stream);
 cerar_status_t cerar_rank_round(cerar_plan_t* plan, int rank, const float* ws, float* peer_ws, int64_t d, int k,
                                 cerar_stream_t stream);
+/* Same message as cerar_rank_round, but written to `msg`, a device buffer of d/c floats of the
+ * caller's, instead of the neighbour's memory: for a transport that moves it itself (a
+ * send/receive pair between GPUs without peer access, as in the paper's own runs over PCIe);
+ * the receiver takes it straight into slot k-1 of its workspace (a contiguous row). */
+cerar_status_t cerar_rank_round_msg(cerar_plan_t* plan, int rank, const float* ws, float* msg, int64_t d, int k,
+                                    cerar_stream_t stream);
 cerar_status_t cerar_rank_decode(cerar_plan_t* plan, int rank, const float* ws, float* out, int64_t d,
                                  float scale, cerar_stream_t stream);
 

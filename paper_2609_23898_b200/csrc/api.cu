@@ -471,6 +471,21 @@ cerar_status_t cerar_rank_round(cerar_plan_t* P, int rank, const float* ws, floa
     return CERAR_OK;
 }
 
+cerar_status_t cerar_rank_round_msg(cerar_plan_t* P, int rank, const float* ws, float* msg, int64_t d, int k,
+                                    cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !msg) return fail(CERAR_ERR_INVALID_ARG, "ws or msg is NULL");
+    if (rank < 0 || rank >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    if (k < 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "round index outside 1..L");
+    cerar::RankRoundArgs a{};
+    a.ws = ws; a.peer_ws = msg; a.p = p; a.N = P->host.N; a.c = P->host.c; a.k = k; a.to_message = 1;
+    cudaError_t e = cerar::launch_rank_round(a, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rank round (message) launch");
+    return CERAR_OK;
+}
+
 cerar_status_t cerar_rank_decode(cerar_plan_t* P, int rank, const float* ws, float* out, int64_t d, float scale,
                                  cerar_stream_t stream) {
     int64_t p;

@@ -43,6 +43,7 @@ struct RankRoundArgs {
     int64_t p;
     int N, c, k;            // round k in 1..L
     int slot_prev, slot_cancel, slot_add, slot_land;   // filled in by the launcher (-1 = term absent)
+    int to_message;         // 1: peer_ws is a plain p-float message buffer (row 0), not a workspace
 };
 
 // All L rounds of up to RING_MAX_WORKERS workers in one launch (blockIdx.y = index into the arrays).

@@ -58,6 +58,7 @@ void rank_round_slots(int N, int c, int k, int* slot_prev, int* slot_cancel, int
 cudaError_t launch_rank_round(RankRoundArgs a, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0) return cudaSuccess;
     rank_round_slots(a.N, a.c, a.k, &a.slot_prev, &a.slot_cancel, &a.slot_add, &a.slot_land);
+    if (a.to_message) a.slot_land = 0;          // the message goes to a buffer of its own, for a transport to send
     const bool vec = (a.p % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.ws) & 15u) == 0) &&
                      ((reinterpret_cast<uintptr_t>(a.peer_ws) & 15u) == 0);
     const int64_t nv = vec ? a.p / 4 : a.p;

@@ -15,6 +15,11 @@ DistributedRing   one worker per process and GPU (torch.distributed, NCCL): the
                   separates the rounds or (fused=True) one kernel runs all rounds
                   and orders itself against the neighbours tile by tile through
                   counters in symmetric memory.  Needs N GPUs with peer access.
+SendRecvRing      one worker per process without peer access (the paper's own setting:
+                  GPUs on PCIe, one process each): the message of a round is formed in a
+                  local buffer and moved by a batched send / receive pair of
+                  torch.distributed (NCCL between GPUs), received straight into the
+                  landing slot of the workspace.
 """
 from __future__ import annotations
 
@@ -132,4 +137,40 @@ class DistributedRing:
             for k in range(1, self.L + 1):
                 self.plan.rank_round(self.rank, self.ws, self.peer_ws, self.d, k, stream)
                 self._barrier()
+        self.plan.rank_decode(self.rank, self.ws, out, self.d, scale, stream)
+
+
+class SendRecvRing:
+    """One worker per rank, messages moved by torch.distributed send / receive."""
+
+    def __init__(self, plan, d: int, group=None, device=None):
+        import torch
+        import torch.distributed as dist
+        self.group = group if group is not None else dist.group.WORLD
+        self.rank, world = dist.get_rank(self.group), dist.get_world_size(self.group)
+        if world != plan.N:
+            raise ValueError(f"the plan is for N={plan.N} workers, the group has {world} ranks")
+        if d % plan.c:
+            raise ValueError("d must be a multiple of c")
+        self.plan, self.d, self.p = plan, d, d // plan.c
+        self.N, self.c, self.L = plan.N, plan.c, plan.L
+        dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        self.ws = torch.empty(plan.rank_workspace_bytes(d) // 4, dtype=torch.float32, device=dev)
+        self.msg = torch.empty(self.p, dtype=torch.float32, device=dev)
+        self.schedule = round_schedule(plan)
+        self.nxt = dist.get_global_rank(self.group, (self.rank + 1) % self.N)
+        self.prv = dist.get_global_rank(self.group, (self.rank - 1) % self.N)
+
+    def allreduce(self, grad, out, scale=1.0, stream=0):
+        """grad, out: this rank's length-d tensors; `stream` must be torch's current stream (the
+        send and the receive are ordered against it by torch.distributed)."""
+        import torch.distributed as dist
+        self.plan.rank_encode(self.rank, grad, self.ws, self.d, stream)
+        rows = self.ws.view(self.c + self.N + 1, self.p)
+        for k, _prev, _cancel, _add, land in self.schedule:
+            self.plan.rank_round_msg(self.rank, self.ws, self.msg, self.d, k, stream)
+            ops = [dist.P2POp(dist.isend, self.msg, self.nxt, self.group),
+                   dist.P2POp(dist.irecv, rows[land], self.prv, self.group)]
+            for req in dist.batch_isend_irecv(ops):
+                req.wait()
         self.plan.rank_decode(self.rank, self.ws, out, self.d, scale, stream)

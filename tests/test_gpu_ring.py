@@ -215,6 +215,48 @@ def test_randomised_ring_shapes(mods):
         cerar.cerar_set_tuning("ring_tile", 0)
 
 
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192 + 260), (3, 5, 1031), (2, 2, 4), (8, 32, 4100), (5, 7, 3)])
+def test_round_into_a_message_buffer_equals_the_peer_store(mods, N, c, p):
+    """cerar_rank_round_msg forms the same message as cerar_rank_round, bit for bit, but leaves
+    it in the caller's buffer; moving the buffers by hand into the neighbours' landing slots (what a
+    send / receive pair does) gives the same workspaces, and an unaligned buffer takes the
+    scalar path with the same bits."""
+    import torch
+    cerar, inputs, ring = mods
+    d = c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(3 * N + c))
+    g = inputs.gradients_numpy(N, d, "normal", seed=9)
+    plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+    s = torch.cuda.current_stream().cuda_stream
+    a, b = ring.LocalRing(plan, d), ring.LocalRing(plan, d)
+    grads = [torch.from_numpy(g[i]).cuda() for i in range(N)]
+    for r in (a, b):
+        for w in r.ws:
+            w.fill_(float("nan"))
+        r.encode(grads, s)
+    rows = c + N + 1
+    raw = torch.full((N, p + 1), float("nan"), device="cuda")
+    for k, _prev, _cancel, _add, land in ring.round_schedule(plan):
+        a.round(k, s)
+        off = k % 2                                       # odd rounds: a buffer that is not 16-byte aligned
+        for i in range(N):
+            plan.rank_round_msg(i, b.ws[i], raw[i, off:off + p], d, k, s)
+        for i in range(N):                                # every message formed before any lands
+            b.ws[(i + 1) % N].view(rows, p)[land].copy_(raw[i, off:off + p])
+        for i in range(N):
+            assert torch.equal(a.ws[i].view(rows, p)[land], b.ws[i].view(rows, p)[land]), (k, i)
+    outs = [torch.empty(d, device="cuda") for _ in range(N)]
+    b.decode(outs, 1.0 / N, s)
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    ora = run_oracle(des.U, des.R, g, 1.0 / N)
+    assert max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
+    with pytest.raises(cerar.CerarError):
+        plan.rank_round_msg(0, b.ws[0], raw[0, :p], d, 0, s)
+    with pytest.raises(cerar.CerarError):
+        plan.rank_round_msg(N, b.ws[0], raw[0, :p], d, 1, s)
+
+
 def test_rank_level_kernels_on_symmetric_memory_allocations(mods):
     """DistributedRing keeps workspaces and counters in torch's symmetric memory.  With one GPU
     the peer mapping cannot be exercised, but the allocations can: a one-rank NCCL group,

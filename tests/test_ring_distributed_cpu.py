@@ -70,6 +70,9 @@ class _CpuPlan:
     def ring_tiles(self, d):
         return self.real.ring_tiles(d)
 
+    def rank_round_slots(self, k):
+        return self.real.rank_round_slots(k)
+
     def _rows(self, ws, d):
         return ws.view(self.c + self.N + 1, d // self.c)
 
@@ -95,6 +98,12 @@ class _CpuPlan:
         land, x = self._message(self._rows(ws, d), k, 0, p)
         self._rows(peer_ws, d)[land] = x
         self.calls.append(("round", rank, k))
+
+    def rank_round_msg(self, rank, ws, msg, d, k, stream=0):
+        p = d // self.c
+        _land, x = self._message(self._rows(ws, d), k, 0, p)
+        msg.copy_(x)
+        self.calls.append(("round_msg", rank, k))
 
     def rank_rounds_fused(self, rank, ws, peer_ws, landed_local, freed_local, landed_next, freed_prev, d, epoch,
                           stream=0):
@@ -199,3 +208,51 @@ def test_distributed_ring_driver_with_two_gloo_ranks(fused):
             assert epoch == 2 and calls == ["encode", "fused", "decode"] * 2
         else:
             assert calls == (["encode"] + ["round"] * L + ["decode"]) * 2
+
+
+def _worker_sendrecv(rank, world, port, c, p, q):
+    sys.path.insert(0, ROOT)
+    import torch
+    import torch.distributed as dist
+    from oracle import designs as Dz
+    from oracle import protocol as P
+    from paper_2609_23898_b200 import cerar, ring
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    N, d = world, c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(6))
+    plan = _CpuPlan(cerar.Plan.create_custom(N, c, des.U, des.R, host_only=True))
+    r = ring.SendRecvRing(plan, d, device=torch.device("cpu"))
+    errs = []
+    for rep in range(2):
+        rng = np.random.default_rng(300 + rep)
+        grads = [rng.standard_normal(d).astype(np.float32) for _ in range(N)]
+        out = torch.empty(d)
+        r.allreduce(torch.from_numpy(grads[rank]), out, 1.0 / N, 0)
+        ora = P.allreduce([g.astype(np.float64) for g in grads], des.U, des.R, 1.0 / N)
+        errs.append(P.rel_l2(out.numpy(), ora["out"][rank]))
+    dist.barrier()
+    dist.destroy_process_group()
+    q.put((rank, errs, [c_[0] for c_ in plan.calls]))
+
+
+@pytest.mark.parametrize("N,c", [(2, 3), (3, 4)])
+def test_send_receive_ring_driver_with_gloo_ranks(N, c):
+    import torch.multiprocessing as mp
+    sys.path.insert(0, ROOT)
+    p = 37
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker_sendrecv, args=(r, N, port, c, p, q)) for r in range(N)]
+    for pr in procs:
+        pr.start()
+    res = sorted(q.get(timeout=240) for _ in procs)
+    for pr in procs:
+        pr.join(timeout=60)
+        assert pr.exitcode == 0
+    L = c + N - 2
+    for rank, errs, calls in res:
+        assert max(errs) < 5e-6, errs
+        assert calls == (["encode"] + ["round_msg"] * L + ["decode"]) * 2
