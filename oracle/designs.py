@@ -7,9 +7,12 @@ A_l are extremely ill-conditioned by design (Remark after Theorem 1,
 Corollary 1), so a plain fp64 inverse would not be a trustworthy reference.
 The condition-number-constrained design is an fp64 iteration (numpy).
 
-PARITY UNPINNED: kappa_constrained for c > N (no published U, R to compare with;
-only its invariants are tested; for c = N, where the optimum Phi = 0 is known, it is
-checked to reach it).
+kappa_constrained: every step of an iteration is pinned to the property that defines
+it (the U-step and the R-step are stationary minimisers of the brute-force Phi, the
+projection is the Frobenius-nearest matrix with singular values in the interval), the
+invariants of the whole iteration are tested, and for c = N, where the optimum Phi = 0 is
+known, it is checked to reach it.  PARITY UNPINNED for the end point at c > N only: the
+paper prints no U, R or Phi of this heuristic to compare with.
 """
 from __future__ import annotations
 

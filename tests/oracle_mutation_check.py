@@ -1,7 +1,7 @@
 """Mutation check of the oracle pins (run by hand: python tests/oracle_mutation_check.py).
 Applies one plausible mistake at a time to the oracle source (restored afterwards),
 runs the CPU oracle tests and expects at least one of them to fail: a mutation that
-survives means a pin is missing.  24 of 24 mutations are killed."""
+survives means a pin is missing.  28 of 28 mutations are killed.  Indices on the command line run only those."""
 import subprocess, shutil, sys, os
 ROOT=os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 muts=[
@@ -29,10 +29,16 @@ muts=[
  ('oracle/designs.py','E = [(l + t) % N for t in range(s)]','E = [(l - t) % N for t in range(s)]'),
  ('oracle/designs.py','blocks.append((B * h ** beta)[E, :])','blocks.append((B * h ** (beta - 1))[E, :])'),
  ('oracle/designs.py','compute_uv=False)[-1]) for l in range(N))','compute_uv=False)[0]) for l in range(N))'),
+ ('oracle/designs.py','U.append(Uk_T.T)','U.append(Uk_T)'),
+ ('oracle/designs.py','out.append((X * np.clip(s, a0, b0)) @ Zt)','out.append((X * np.clip(s, a0, b0)) @ Zt.T)'),
+ ('oracle/designs.py','return [np.linalg.lstsq(protocol.m_matrix(U, i), T, rcond=None)[0] for i in range(N)]','return [np.linalg.lstsq(protocol.m_matrix(U, (i + 1) % N), T, rcond=None)[0] for i in range(N)]'),
+ ('oracle/designs.py','Tk = np.concatenate([np.eye(c)] * N, axis=1)','Tk = np.concatenate([np.eye(c)] * (N - 1) + [np.zeros((c, c))], axis=1)'),
 ]
 def main():
     survived=[]
+    only=[int(a) for a in sys.argv[1:]]
     for idx,(f,old,new) in enumerate(muts):
+        if only and idx not in only: continue
         path=os.path.join(ROOT,f); src=open(path).read()
         if old not in src:
             print(idx,'PATTERN NOT FOUND',f,old[:40]); continue

@@ -352,6 +352,86 @@ def test_kappa_constrained_invariants():
     assert 1e-3 < err < 0.1
 
 
+# The three steps of one iteration (Sec. II-D), each against the property that defines it.  Phi is
+# evaluated from the M_i matrices (pinned by brute force in test_oracle_protocol.py), so a step that
+# solved for the wrong blocks, or transposed its result, is not a minimiser of THIS Phi.
+
+def _phi_slope_and_rise(U, R, perturb, t=1e-3):
+    """Phi is quadratic along any line: central difference = exact slope, Phi(+t) + Phi(-t) - 2 Phi(0) = 2 t^2 curvature."""
+    f0 = P.phi(U, R)
+    fp = P.phi(*perturb(U, R, +t))
+    fm = P.phi(*perturb(U, R, -t))
+    return (fp - fm) / (2 * t), fp + fm - 2 * f0, f0
+
+
+@pytest.mark.parametrize("N,c", [(3, 5), (4, 6), (2, 5)])
+def test_als_U_step_and_R_step_are_stationary_minimisers_of_phi(N, c):
+    rng = np.random.default_rng(N * 10 + c)
+    L = c + N - 2
+    # U-step: R arbitrary, U = argmin_U Phi(U, R)
+    R = [rng.standard_normal((L + 1, c)) for _ in range(N)]
+    U = Dz._ls_U(R, N, c)
+    for trial in range(12):
+        k = trial % N
+        E = rng.standard_normal((c, c))
+
+        def perturb(U_, R_, t, k=k, E=E):
+            V = [u.copy() for u in U_]
+            V[k] = V[k] + t * E
+            return V, R_
+        slope, rise, f0 = _phi_slope_and_rise(U, R, perturb)
+        assert abs(slope) < 1e-7 * max(1.0, f0), (k, slope)
+        assert rise > 0
+    # and it is not a minimiser by accident of the test: a U that is not the step's has a slope
+    V = [u + 0.1 * rng.standard_normal((c, c)) for u in U]
+    E = rng.standard_normal((c, c))
+    slope, _, f0 = _phi_slope_and_rise(V, R, lambda U_, R_, t: ([U_[0] + t * E] + list(U_[1:]), R_))
+    assert abs(slope) > 1e-3
+    # R-step: U arbitrary, R = argmin_R Phi(U, R)
+    U = [rng.standard_normal((c, c)) for _ in range(N)]
+    R = Dz._ls_R(U, N, c)
+    for trial in range(12):
+        i = trial % N
+        E = rng.standard_normal((L + 1, c))
+
+        def perturb(U_, R_, t, i=i, E=E):
+            Q = [r.copy() for r in R_]
+            Q[i] = Q[i] + t * E
+            return U_, Q
+        slope, rise, f0 = _phi_slope_and_rise(U, R, perturb)
+        assert abs(slope) < 1e-7 * max(1.0, f0), (i, slope)
+        assert rise > 0
+
+
+def test_als_projection_is_the_nearest_matrix_with_singular_values_in_the_interval():
+    """Clamping the singular values is the Frobenius-nearest point of {sigma(X) in [a, b]}
+    (Mirsky's inequality: ||A - X||_F >= ||sigma(A) - sigma(X)||_2, attained with A's singular vectors).
+    Checked against that bound, against feasible competitors, and on matrices it must not change."""
+    rng = np.random.default_rng(4)
+    c, a, b = 5, 0.5, 2.0
+    for trial in range(6):
+        A = rng.standard_normal((c, c)) * rng.choice([0.3, 1.0, 3.0])
+        Pj = Dz._project([A], a, b)[0]
+        sA = np.linalg.svd(A, compute_uv=False)
+        sP = np.linalg.svd(Pj, compute_uv=False)
+        assert sP[-1] >= a * (1 - 1e-12) and sP[0] <= b * (1 + 1e-12)
+        best = np.linalg.norm(sA - np.clip(sA, a, b))
+        assert np.linalg.norm(A - Pj) == pytest.approx(best, rel=1e-10, abs=1e-13)
+        for _ in range(200):                               # no feasible competitor is nearer
+            X, _ = np.linalg.qr(rng.standard_normal((c, c)))
+            Z, _ = np.linalg.qr(rng.standard_normal((c, c)))
+            mix = rng.uniform(0, 0.2)
+            Xc, s0, Zc = np.linalg.svd(A)
+            Xn, _ = np.linalg.qr(Xc + mix * X)
+            Zn, _ = np.linalg.qr(Zc.T + mix * Z)
+            comp = (Xn * rng.uniform(a, b, c)) @ Zn.T
+            assert np.linalg.norm(A - comp) >= np.linalg.norm(A - Pj) * (1 - 1e-12)
+    inside = (np.linalg.qr(rng.standard_normal((c, c)))[0] * rng.uniform(a, b, c)) @ np.linalg.qr(rng.standard_normal((c, c)))[0]
+    assert np.allclose(Dz._project([inside], a, b)[0], inside, atol=1e-13)
+    once = Dz._project([A], a, b)
+    assert np.allclose(Dz._project(once, a, b)[0], once[0], atol=1e-13)
+
+
 def test_surrogate_is_well_conditioned():
     des = Dz.custom_orthogonal(4, 8, np.random.default_rng(0))
     for u in des.U:
