@@ -194,8 +194,9 @@ cerar_status_t cerar_ring_round(cerar_plan_t* plan, float* ws, int64_t d, int k,
  * ordering against other threads.  Same stores into the neighbours' slots, same results bit for
  * bit, same counters; but a message may be read back from cache instead of HBM, so for a
  * workspace larger than the L2 this is not the HBM hand-off that cerar_ring_round performs.
- * cerar_allreduce_sim uses it on its own for workspaces up to 64 MB, which never leave the L2
- * and are bound by the L launches otherwise. */
+ * cerar_allreduce_sim uses it on its own where it is the faster form: for workspaces up to 64 MB,
+ * which never leave the L2 and are bound by the L launches otherwise, and for N <= 4 (with d/c a
+ * multiple of 4) at every size. */
 cerar_status_t cerar_ring_rounds(cerar_plan_t* plan, float* ws, int64_t d, int k_first, int k_last,
                                  cerar_stream_t stream);
 cerar_status_t cerar_decode(cerar_plan_t* plan, const float* ws, float* out, int64_t out_stride,
@@ -372,6 +373,8 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "serpentine_off"                1 = every ring round walks the positions upwards
  *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24)
  *   "rounds_one_launch_off"         1 = cerar_allreduce_sim always launches round by round
+ *   "rounds_one_launch_mb"          largest workspace (MB) whose rounds cerar_allreduce_sim runs in
+ *                                   one launch, for every N (default: 64, and no limit for N <= 4)
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

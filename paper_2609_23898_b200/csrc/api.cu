@@ -348,9 +348,16 @@ cerar_status_t cerar_allreduce_sim(cerar_plan_t* P, const float* grads, int64_t 
                                    int64_t out_stride, float* ws, int64_t d, float scale, cerar_stream_t stream) {
     cerar_status_t st = cerar_encode(P, grads, grads_stride, ws, d, stream);
     if (st != CERAR_OK) return st;
-    // A state that lives in the L2 anyway (hand-offs never reach HBM in either form) is bound by the
-    // L launches of the round-by-round form: run its rounds in one launch.
-    if (cerar_workspace_bytes(P, d) <= kOneLaunchRoundsBytes && !cerar::g_tune_rounds_one_launch_off) {
+    // One launch for all rounds where that is the faster form (measured): a state that lives in L2 anyway
+    // (hand-offs never reach HBM in either form, and L launches cost more than the data movement), and
+    // any state with N <= 4, where a thread has all loads of a round in flight at once and the message
+    // it has just stored is read back from cache.
+    const size_t one_launch_limit = cerar::g_tune_rounds_one_launch_mb > 0
+                                        ? (size_t)cerar::g_tune_rounds_one_launch_mb << 20 : kOneLaunchRoundsBytes;
+    const bool one_launch = (cerar_workspace_bytes(P, d) <= one_launch_limit ||
+                             (P->host.N <= 4 && (d / P->host.c) % 4 == 0 && cerar::g_tune_rounds_one_launch_mb == 0)) &&
+                            !cerar::g_tune_rounds_one_launch_off;
+    if (one_launch) {
         if ((st = cerar_ring_rounds(P, ws, d, 1, P->host.L, stream)) != CERAR_OK) return st;
     } else {
         for (int k = 1; k <= P->host.L; ++k)
@@ -675,6 +682,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "serpentine_off") cerar::g_tune_serpentine_off = value;
     else if (n == "tc_min_c") cerar::g_tune_tc_min_c = value;
     else if (n == "rounds_one_launch_off") cerar::g_tune_rounds_one_launch_off = value;
+    else if (n == "rounds_one_launch_mb") cerar::g_tune_rounds_one_launch_mb = value;
     else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;

@@ -310,8 +310,11 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
 // touches nothing else, so the rounds of one position need no ordering against other threads:
 // each thread simply runs them one after the other (its own stores are visible to its own later
 // loads).  Every message is still stored into the neighbour's slot and read back from there in
-// the next round, but that read may be served from cache, so this form is for states that live
-// in L2 anyway, where the L launches of the round-by-round form cost more than the data movement.
+// the next round, but that read may be served from cache.  Measured on B200: always faster for states
+// that live in L2 (the L launches cost more than the data movement), and at every size for N <= 4
+// (one group of workers per round: +4 .. +25 %); for larger N it loses up to 20 % once the state
+// exceeds L2 (several dependent groups per round and L dependent rounds per thread).  Groups of 8
+// workers, 8-byte accesses and fewer resident threads were measured too and are slower.
 template <typename VT, int WG>
 __global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, int k_last) {
     constexpr int VW = sizeof(VT) / 4;
@@ -364,7 +367,7 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
 int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
-    g_tune_rounds_one_launch_off = 0;
+    g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0;
 
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0 || a.N <= 0) return cudaSuccess;

@@ -94,12 +94,17 @@ def main():
                     if rep >= 3:
                         times.append(e0.elapsed_time(e1))
                 plan.device_status(stream)
+                n0 = plan.launch_count()
+                plan.allreduce_sim(dptr, wstride, dptr, wstride, ws, d, 1.0 / N, stream)
+                torch.cuda.synchronize()
+                launches = plan.launch_count() - n0
                 ms = float(np.median(times))
                 ab = 4 * N * p * (8 * c + 3 * N - 8)
                 gbs = ab / ms / 1e6
                 l2 = "L2-resident" if ws_bytes < 100e6 else ""
-                row = dict(N=N, c=c, d=d, state_mb=ws_bytes / 1e6, ms=ms, gbps=gbs, frac=gbs / peak,
-                           note=", ".join(x for x in (note, l2) if x))
+                one = "rounds in one launch" if launches == 3 else ""
+                row = dict(N=N, c=c, d=d, state_mb=ws_bytes / 1e6, ms=ms, gbps=gbs, frac=gbs / peak, launches=launches,
+                           note=", ".join(x for x in (note, l2, one) if x))
                 rows.append(row)
                 print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | {ms:.3f} | {gbs:.0f} | {gbs / peak:.2f} | {row['note']} |",
                       flush=True)
