@@ -189,14 +189,16 @@ cerar_status_t cerar_encode(cerar_plan_t* plan, const float* grads, int64_t grad
                             float* ws, int64_t d, cerar_stream_t stream);
 cerar_status_t cerar_ring_round(cerar_plan_t* plan, float* ws, int64_t d, int k,
                                 cerar_stream_t stream);
-/* Rounds k_first .. k_last (k_first must follow the last completed round) in ONE launch: a thread
- * owns its positions for all N workers, so it runs their rounds one after the other without any
- * ordering against other threads.  Same stores into the neighbours' slots, same results bit for
- * bit, same counters; but a message may be read back from cache instead of HBM, so for a
- * workspace larger than the L2 this is not the HBM hand-off that cerar_ring_round performs.
- * cerar_allreduce_sim uses it on its own where it is the faster form: for workspaces up to 64 MB,
- * which never leave the L2 and are bound by the L launches otherwise, and for N <= 4 (with d/c a
- * multiple of 4) at every size. */
+/* Rounds k_first .. k_last (k_first must follow the last completed round) in ONE launch: a block
+ * of N warps owns 32 (x 4) positions, warp i plays worker i; every message is stored into the
+ * neighbour's slot as in cerar_ring_round and, besides, handed to the neighbour's warp through
+ * shared memory, so a round costs a block barrier instead of a launch and the operands of the
+ * next round are already in flight.  Same slots afterwards bit for bit, same counters; but the
+ * receiver takes the message from shared memory, not from its slot, so this is not the in-HBM
+ * hand-off that cerar_ring_round performs (per steady round 2 reads + 1 write reach memory
+ * instead of 3 + 1).  (N > 32: one thread per position runs its N workers in turn.)
+ * cerar_allreduce_sim uses it on its own (it measured faster than L launches at every shape
+ * tried), except for N <= 32 with d/c > 65536 not a multiple of 4 and a workspace above 64 MB. */
 cerar_status_t cerar_ring_rounds(cerar_plan_t* plan, float* ws, int64_t d, int k_first, int k_last,
                                  cerar_stream_t stream);
 cerar_status_t cerar_decode(cerar_plan_t* plan, const float* ws, float* out, int64_t out_stride,
@@ -373,8 +375,13 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "serpentine_off"                1 = every ring round walks the positions upwards
  *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24)
  *   "rounds_one_launch_off"         1 = cerar_allreduce_sim always launches round by round
- *   "rounds_one_launch_mb"          largest workspace (MB) whose rounds cerar_allreduce_sim runs in
- *                                   one launch, for every N (default: 64, and no limit for N <= 4)
+ *   "rounds_one_launch_mb"          if set, cerar_allreduce_sim runs the rounds in one launch exactly
+ *                                   for workspaces up to this many MB (default rule: see
+ *                                   cerar_ring_rounds)
+ *   "rounds_coop_shape"             vectors per lane of the warp-per-worker kernel (0 = automatic, 1, 2)
+ *   "rounds_multi_form"             kernel of cerar_ring_rounds: 0 = warp per worker (16-byte
+ *                                   accesses where there are enough positions), 3 = the same with
+ *                                   4-byte accesses, 1 = thread per position
  * Returns 0, or -1 for an unknown name. */
 int            cerar_set_tuning(const char* name, int value);
 

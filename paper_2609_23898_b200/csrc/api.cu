@@ -348,15 +348,16 @@ cerar_status_t cerar_allreduce_sim(cerar_plan_t* P, const float* grads, int64_t 
                                    int64_t out_stride, float* ws, int64_t d, float scale, cerar_stream_t stream) {
     cerar_status_t st = cerar_encode(P, grads, grads_stride, ws, d, stream);
     if (st != CERAR_OK) return st;
-    // One launch for all rounds where that is the faster form (measured): a state that lives in L2 anyway
-    // (hand-offs never reach HBM in either form, and L launches cost more than the data movement), and
-    // any state with N <= 4, where a thread has all loads of a round in flight at once and the message
-    // it has just stored is read back from cache.
+    // One launch for all rounds (one warp per worker, messages handed on through shared memory as well
+    // as stored) wherever that kernel applies at full width: it measured faster than one launch per
+    // round at every shape tried (from 1.2 times at d = 2^30 to 10 times where the launches dominate).
     const size_t one_launch_limit = cerar::g_tune_rounds_one_launch_mb > 0
                                         ? (size_t)cerar::g_tune_rounds_one_launch_mb << 20 : kOneLaunchRoundsBytes;
-    const bool one_launch = (cerar_workspace_bytes(P, d) <= one_launch_limit ||
-                             (P->host.N <= 4 && (d / P->host.c) % 4 == 0 && cerar::g_tune_rounds_one_launch_mb == 0)) &&
-                            !cerar::g_tune_rounds_one_launch_off;
+    const int64_t p_sim = d / P->host.c;
+    bool one_launch = cerar_workspace_bytes(P, d) <= one_launch_limit;
+    if (cerar::g_tune_rounds_one_launch_mb == 0 && P->host.N <= 32)
+        one_launch = one_launch || p_sim <= 65536 || p_sim % 4 == 0;
+    if (cerar::g_tune_rounds_one_launch_off) one_launch = false;
     if (one_launch) {
         if ((st = cerar_ring_rounds(P, ws, d, 1, P->host.L, stream)) != CERAR_OK) return st;
     } else {
@@ -683,6 +684,8 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "tc_min_c") cerar::g_tune_tc_min_c = value;
     else if (n == "rounds_one_launch_off") cerar::g_tune_rounds_one_launch_off = value;
     else if (n == "rounds_one_launch_mb") cerar::g_tune_rounds_one_launch_mb = value;
+    else if (n == "rounds_multi_form") cerar::g_tune_rounds_multi_form = value;
+    else if (n == "rounds_coop_shape") cerar::g_tune_rounds_coop_shape = value;
     else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;

@@ -306,15 +306,12 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
     round_body<VT, WG>(reinterpret_cast<VT*>(a.ws) + v, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, a.k);
 }
 
-// Rounds k .. k_last in one launch.  A thread owns its positions for all N workers, and a round
-// touches nothing else, so the rounds of one position need no ordering against other threads:
-// each thread simply runs them one after the other (its own stores are visible to its own later
-// loads).  Every message is still stored into the neighbour's slot and read back from there in
-// the next round, but that read may be served from cache.  Measured on B200: always faster for states
-// that live in L2 (the L launches cost more than the data movement), and at every size for N <= 4
-// (one group of workers per round: +4 .. +25 %); for larger N it loses up to 20 % once the state
-// exceeds L2 (several dependent groups per round and L dependent rounds per thread).  Groups of 8
-// workers, 8-byte accesses and fewer resident threads were measured too and are slower.
+// Rounds k .. k_last in one launch, one THREAD per position vector: the thread owns its positions
+// for all N workers, and a round touches nothing else, so it simply runs the rounds one after the
+// other (its own stores are visible to its own later loads).  Latency-bound (L dependent rounds
+// of N / WG dependent groups each); kept for N > 32, which the warp-per-worker kernel below cannot
+// hold in one block.  Groups of 8 workers, 8-byte accesses and fewer resident threads were measured
+// and are slower.
 template <typename VT, int WG>
 __global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, int k_last) {
     constexpr int VW = sizeof(VT) / 4;
@@ -325,6 +322,76 @@ __global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, in
     const int64_t pv = a.p / VW;
     VT* base = reinterpret_cast<VT*>(a.ws) + v;
     for (int k = a.k; k <= k_last; ++k) round_body<VT, WG>(base, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, k);
+}
+
+// The same rounds k .. k_last in one launch with one WARP per worker: a block of N warps owns 32 PV
+// vectors of positions, warp i plays worker i.  The message of a round is stored into the neighbour's
+// slot (as always) and handed to the neighbour's warp through shared memory, so a round costs one
+// block barrier instead of a trip to memory, and the operands of the next DIST rounds (which do not
+// depend on this one) are already on their way when the barrier is reached.  Hazard: the slot a
+// message lands in holds the delta its owner cancels in that very round; every thread therefore
+// reads its cancel operand at least one round early (before the barrier that precedes the store),
+// never after.  Measured on B200 (rounds of N=8, c=32, d=2^28, in the metric's bytes): DIST 1
+// 8.2 TB/s, DIST 2 10.4, DIST 3 and 4 9.7; one launch per round 7.2.
+template <typename VT, int PV, int DIST, int MAXT>
+__global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, int k_last) {
+    extern __shared__ float4 coop_smem[];
+    VT* hand = reinterpret_cast<VT*>(coop_smem);                // [2][N][PV][32]
+    constexpr int VW = sizeof(VT) / 4;
+    const int i = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int N = a.N, c = a.c;
+    const int64_t pv = a.p / VW;
+    const int64_t v0 = (int64_t)blockIdx.x * (32 * PV) + lane;  // this lane's vectors: v0 + 32 j
+    bool live[PV];
+#pragma unroll
+    for (int j = 0; j < PV; ++j) live[j] = v0 + 32 * j < pv;
+    const int64_t wstride = (int64_t)(c + N) * pv;
+    const int dst = (i + 1 == N) ? 0 : i + 1;
+    VT* own = reinterpret_cast<VT*>(a.ws) + (int64_t)i * wstride + v0;
+    VT* nxt = reinterpret_cast<VT*>(a.ws) + (int64_t)dst * wstride + v0;
+    grid_dependency_wait();
+    int k = a.k;
+    // operands of rounds k .. k+DIST-1 (index t = rounds ahead); absent terms are zero
+    VT y[PV], da[DIST][PV], dc[DIST][PV];
+#pragma unroll
+    for (int j = 0; j < PV; ++j) {
+        y[j] = vzero<VT>();
+        if (live[j] && k >= 2) y[j] = own[(int64_t)(k - 2) * pv + 32 * j];
+#pragma unroll
+        for (int t = 0; t < DIST; ++t) {
+            const int kt = k + t;
+            da[t][j] = dc[t][j] = vzero<VT>();
+            if (live[j] && kt <= k_last) {
+                if (kt <= c) da[t][j] = own[(int64_t)(N - 1 + kt) * pv + 32 * j];
+                if (kt - 1 >= N) dc[t][j] = own[(int64_t)(kt - 1) * pv + 32 * j];
+            }
+        }
+    }
+    __syncthreads();
+    for (; k <= k_last; ++k) {
+        VT* hb = hand + (size_t)(k & 1) * N * (32 * PV);
+#pragma unroll
+        for (int j = 0; j < PV; ++j) {
+            const VT x = combine(y[j], dc[0][j], da[0][j]);
+            if (live[j]) nxt[(int64_t)(k - 1) * pv + 32 * j] = x;
+            hb[(dst * PV + j) * 32 + lane] = x;
+        }
+        // shift the operand queue and fetch round k + DIST (its slots are not written before that round)
+        const int kn = k + DIST;
+#pragma unroll
+        for (int j = 0; j < PV; ++j) {
+#pragma unroll
+            for (int t = 0; t + 1 < DIST; ++t) { da[t][j] = da[t + 1][j]; dc[t][j] = dc[t + 1][j]; }
+            da[DIST - 1][j] = dc[DIST - 1][j] = vzero<VT>();
+            if (live[j] && kn <= k_last) {
+                if (kn <= c) da[DIST - 1][j] = own[(int64_t)(N - 1 + kn) * pv + 32 * j];
+                if (kn - 1 >= N) dc[DIST - 1][j] = own[(int64_t)(kn - 1) * pv + 32 * j];
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < PV; ++j) y[j] = hb[(i * PV + j) * 32 + lane];
+    }
 }
 
 // Nothing ever arrives on this barrier: the bounded wait runs out after limit_ns and the
@@ -367,7 +434,7 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
 int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
-    g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0;
+    g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0, g_tune_rounds_multi_form = 0, g_tune_rounds_coop_shape = 0;
 
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0 || a.N <= 0) return cudaSuccess;
@@ -482,6 +549,25 @@ cudaError_t launch_rounds_multi(const RoundArgs& a, int k_last, cudaStream_t s, 
     // with narrower accesses and smaller blocks rather than leave most of them idle
     int threads = 256;
     const bool vec = (a.p % 4 == 0 && aligned16(a.ws));
+    if (a.N <= 32 && g_tune_rounds_multi_form != 1) {
+        // float4 per lane once that still gives every SM a few blocks; single floats below
+        const bool v4 = vec && (a.p / 128 >= 148 * 2) && g_tune_rounds_multi_form != 3;
+        const int64_t pv = v4 ? a.p / 4 : a.p;
+        // two vectors per lane where that still leaves every SM two blocks (measured: +2 .. +15 % on most
+        // shapes); tuning: 1 / 2 force one / two
+        const int PVr = !v4 ? 1 : g_tune_rounds_coop_shape ? g_tune_rounds_coop_shape
+                                                           : (a.p / 256 >= 148 * 2 ? 2 : 1);
+        const unsigned blocks = (unsigned)((pv + 32 * PVr - 1) / (32 * PVr));
+        const size_t smem = (size_t)2 * a.N * 32 * PVr * (v4 ? 16 : 4);
+        const dim3 blk(32 * a.N);
+        cudaError_t ec;
+#define COOP(VT, PV) (a.N > 16 ? launch_pdl(rounds_coop_kernel<VT, PV, 2, 1024>, dim3(blocks), blk, smem, s, a, k_last) \
+                               : launch_pdl(rounds_coop_kernel<VT, PV, 2, 512>, dim3(blocks), blk, smem, s, a, k_last))
+        ec = !v4 ? COOP(float, 1) : PVr == 2 ? COOP(float4, 2) : COOP(float4, 1);
+#undef COOP
+        if (ec == cudaSuccess && launches) ++*launches;
+        return ec;
+    }
     bool use_vec = vec;
     if (vec && a.p / 4 >= (int64_t)148 * 256 * 4) threads = 256;
     else if (vec && a.p / 4 >= (int64_t)148 * 64 * 4) threads = 64;

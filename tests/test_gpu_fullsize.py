@@ -1,6 +1,8 @@
-"""Full-size configurations in the launch configuration bench.py times (out of place,
-one-call pipeline), checked on sampled positions: all arithmetic is element-wise over
-positions, so the oracle re-runs the whole protocol on the sampled columns only."""
+"""Full-size configurations in the two launch configurations bench.py times (out of place:
+the step it reports, cerar_encode + L x cerar_ring_round + cerar_decode, and the one-call
+pipeline cerar_allreduce_sim, whose rounds run in one launch at these shapes), checked on sampled
+positions: all arithmetic is element-wise over positions, so the oracle re-runs the whole protocol
+on the sampled columns only."""
 import numpy as np
 import pytest
 
@@ -12,7 +14,7 @@ pytestmark = pytest.mark.gpu
 U32 = 2.0 ** -24
 
 
-def _run(cfg_name, des, plan_factory, need_gb):
+def _run(cfg_name, des, plan_factory, need_gb, how="one_call"):
     import torch
     from paper_2609_23898_b200 import inputs
     from tests._harness import sampled_parity
@@ -28,9 +30,17 @@ def _run(cfg_name, des, plan_factory, need_gb):
     ws = torch.empty(plan.workspace_bytes(d) // 4, dtype=torch.float32, device="cuda")
     out = torch.empty(N * d, dtype=torch.float32, device="cuda")
     s = torch.cuda.current_stream().cuda_stream
-    plan.allreduce_sim(grads, d, out, d, ws, d, 1.0 / N, s)
+    n0 = plan.launch_count()
+    if how == "one_call":
+        plan.allreduce_sim(grads, d, out, d, ws, d, 1.0 / N, s)
+    else:
+        plan.encode(grads, d, ws, d, s)
+        for k in range(1, plan.L + 1):
+            plan.ring_round(ws, d, k, s)
+        plan.decode(ws, out, d, d, 1.0 / N, s)
     torch.cuda.synchronize()
     plan.device_status(s)
+    assert plan.launch_count() - n0 == (3 if how == "one_call" else plan.L + 2)
     res = sampled_parity(cfg, des, plan, grads, ws, out, 1.0 / N, n_tiles=8, tile=384)
     cnt = plan.counters()
     assert cnt["bytes_forwarded_per_worker"] * c == cnt["bytes_gradient"] * (c + N - 2)
@@ -40,21 +50,24 @@ def _run(cfg_name, des, plan_factory, need_gb):
     return res
 
 
-def test_config3_full_size_sampled():
+@pytest.mark.parametrize("how", ["per_round", "one_call"])
+def test_config3_full_size_sampled(how):
     """N=8, c=32, eps=1e-2, d=1,414,647,808 (147 GB on the device)."""
     from paper_2609_23898_b200 import cerar, inputs
     cfg = inputs.CONFIGS["cfg3"]
     B = inputs.base_matrix(cfg["N"], cfg["c"], 0)
     des = Dz.epsilon(cfg["N"], cfg["c"], cfg["param"], B)
-    res = _run("cfg3", des, lambda: cerar.Plan.create(cfg["N"], cfg["c"], cerar.EPSILON, cfg["param"], B=B), 150)
-    print("\n[cfg3 full size]", res)
+    res = _run("cfg3", des, lambda: cerar.Plan.create(cfg["N"], cfg["c"], cerar.EPSILON, cfg["param"], B=B), 150,
+               how)
+    print("\n[cfg3 full size]", how, res)
     assert res["positions"] >= 2048
     assert res["rel_l2_Y"] < 2e-6                      # encode + all rounds, no cancellation
     assert res["rel_l2_out_max"] < 4 * res["kappa_M"] * U32
     assert res["rel_l2_oracle_vs_exact_mean"] < 0.05   # the design itself approximates the mean to O(eps)
 
 
-def test_config4_full_size_sampled():
+@pytest.mark.parametrize("how", ["per_round", "one_call"])
+def test_config4_full_size_sampled(how):
     """N=8, c=64, kappa-constrained design (C = 1e4), d=2^28, Student-t gradients.  The
     design is the oracle's own (fewer ALS sweeps than the default to keep the test short;
     any projected iterate satisfies the constraint) handed over as a custom plan."""
@@ -65,8 +78,8 @@ def test_config4_full_size_sampled():
     des = Dz.kappa_constrained(N, c, cfg["param"], B, iters=20)
     kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
     assert kap <= cfg["param"]
-    res = _run("cfg4", des, lambda: cerar.Plan.create_custom(N, c, des.U, des.R), 30)
-    print("\n[cfg4 full size]", res)
+    res = _run("cfg4", des, lambda: cerar.Plan.create_custom(N, c, des.U, des.R), 30, how)
+    print("\n[cfg4 full size]", how, res)
     assert res["rel_l2_Y"] < 2e-6
     assert res["rel_l2_out_max"] < max(1e-4, 4 * kap * U32)
 

@@ -469,10 +469,12 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
         cerar_mod.cerar_set_tuning("tc_variant", 0)
 
 
-@pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (3, 5, 1031), (16, 16, 1028), (2, 2, 4)])
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (3, 5, 1031), (16, 16, 1028), (2, 2, 4), (5, 7, 3),
+                                   (8, 16, 40004), (32, 32, 36), (7, 9, 37889), (4, 8, 76036)])
 def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
-    """cerar_ring_rounds (what cerar_allreduce_sim uses for cache-resident states) leaves exactly
-    the slots of L calls of cerar_ring_round, in one go or in pieces, with the same counters."""
+    """cerar_ring_rounds (what cerar_allreduce_sim uses where it is the faster form) leaves exactly
+    the slots of L calls of cerar_ring_round, in one go or in pieces, with the same counters: the
+    warp-per-worker kernel with 16-byte and with 4-byte accesses and the thread-per-position kernel."""
     import torch
     d = c * p
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(N + c))
@@ -480,7 +482,11 @@ def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
     s = torch_stream()
     L = c + N - 2
     res = []
-    for how in ("each", "all", "pieces"):
+    for how in ("each", "all", "pieces", "all-threads", "all-scalar", "pieces-threads", "all-one", "pieces-two"):
+        kind = how.split("-")[-1]
+        cerar_mod.cerar_set_tuning("rounds_multi_form", {"threads": 1, "scalar": 3}.get(kind, 0))
+        cerar_mod.cerar_set_tuning("rounds_coop_shape", {"one": 1, "two": 2}.get(kind, 0))
+        how = how.split("-")[0]
         plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
         ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
         plan.encode(g, d, ws, d, s)
@@ -501,6 +507,8 @@ def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
         torch.cuda.synchronize()
         plan.device_status(s)
         res.append((ws.clone(), plan.counters()))
+    cerar_mod.cerar_set_tuning("rounds_multi_form", 0)
+    cerar_mod.cerar_set_tuning("rounds_coop_shape", 0)
     for w, cnt in res[1:]:
         assert torch.equal(torch.nan_to_num(w, nan=-1.0), torch.nan_to_num(res[0][0], nan=-1.0))
         assert cnt == res[0][1]
