@@ -5,9 +5,12 @@
 Points: d per worker in {2^18, 2^20, ..., 2^30} fp32, N in {4, 8, 16}, c in {N, 2N, 4N, 8N},
 epsilon-construction with eps = 1e-3, i.i.d. N(0,1) gradients.  Every point runs in place
 (the gradients are generated directly in the D rows of the workspace and the result
-overwrites them), so the largest point (N=16, d=2^30, c=16) needs 137 GB.  Per point:
-3 warm-up and 5 timed aggregations (CUDA events around cerar_allreduce_sim, median), the
-gradients are regenerated before every aggregation (outside the timed region).
+overwrites them), so the largest point (N=16, d=2^30, c=16) needs 137 GB.  Per point and
+launch form: 3 warm-up and 5 timed aggregations (CUDA events around cerar_allreduce_sim,
+median), the gradients are regenerated before every aggregation (outside the timed region).
+Two launch forms: "round by round" (one launch per round, every hand-off through HBM: the
+step bench.py reports) and "one call" (cerar_allreduce_sim as it stands: all rounds in one
+launch, messages also handed on chip, so fewer bytes than the metric counts reach DRAM).
 
 Reported: seconds per aggregation, algorithmic GB/s (N (8c+3N-8) p 4 bytes per
 aggregation) and its fraction of the measured HBM copy bandwidth.  Points whose whole
@@ -52,8 +55,8 @@ def main():
         return fused_table(args, exps, peak, free, stream)
     if args.ring:
         return ring_table(args, exps, peak, free, stream)
-    print("| N | c | d | state MB | ms / aggregation | GB/s | frac of measured HBM | note |")
-    print("|---|---|---|---|---|---|---|---|")
+    print("| N | c | d | state MB | round by round: ms | GB/s | frac | launches | one call: ms | GB/s | frac | launches | note |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|---|")
     for N in (4, 8, 16):
         for mult in (1, 2, 4, 8):
             c = N * mult
@@ -77,37 +80,42 @@ def main():
                 p = d // c
                 ws_bytes = plan.workspace_bytes(d)
                 if ws_bytes > free - (2 << 30):
-                    print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | - | - | - | skipped: needs {ws_bytes / 1e9:.1f} GB |")
+                    print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | - | - | - | - | - | - | - | - | "
+                          f"skipped: needs {ws_bytes / 1e9:.1f} GB |")
                     continue
                 ws = torch.empty(ws_bytes // 4, dtype=torch.float32, device="cuda")
                 wstride = (c + N) * p
                 dptr = ws.data_ptr() + 4 * N * p
-                times = []
-                for rep in range(8):
-                    for i in range(N):
-                        ws[i * wstride + N * p:(i + 1) * wstride].normal_()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    plan.allreduce_sim(dptr, wstride, dptr, wstride, ws, d, 1.0 / N, stream)
-                    e1.record()
-                    torch.cuda.synchronize()
-                    if rep >= 3:
-                        times.append(e0.elapsed_time(e1))
-                plan.device_status(stream)
-                n0 = plan.launch_count()
-                plan.allreduce_sim(dptr, wstride, dptr, wstride, ws, d, 1.0 / N, stream)
-                torch.cuda.synchronize()
-                launches = plan.launch_count() - n0
-                ms = float(np.median(times))
+                res = {}
+                for form in ("round by round", "one call"):
+                    # "round by round": one launch per round, every hand-off through HBM (the step bench.py
+                    # reports); "one call": cerar_allreduce_sim as it stands (rounds in one launch)
+                    cerar.cerar_set_tuning("rounds_one_launch_off", 1 if form == "round by round" else 0)
+                    times = []
+                    for rep in range(8):
+                        for i in range(N):
+                            ws[i * wstride + N * p:(i + 1) * wstride].normal_()
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        n0 = plan.launch_count()
+                        e0.record()
+                        plan.allreduce_sim(dptr, wstride, dptr, wstride, ws, d, 1.0 / N, stream)
+                        e1.record()
+                        torch.cuda.synchronize()
+                        if rep >= 3:
+                            times.append(e0.elapsed_time(e1))
+                    plan.device_status(stream)
+                    res[form] = (float(np.median(times)), plan.launch_count() - n0)
+                cerar.cerar_set_tuning("rounds_one_launch_off", 0)
                 ab = 4 * N * p * (8 * c + 3 * N - 8)
-                gbs = ab / ms / 1e6
+                (ms_r, l_r), (ms, launches) = res["round by round"], res["one call"]
+                gbs_r, gbs = ab / ms_r / 1e6, ab / ms / 1e6
                 l2 = "L2-resident" if ws_bytes < 100e6 else ""
-                one = "rounds in one launch" if launches == 3 else ""
                 row = dict(N=N, c=c, d=d, state_mb=ws_bytes / 1e6, ms=ms, gbps=gbs, frac=gbs / peak, launches=launches,
-                           note=", ".join(x for x in (note, l2, one) if x))
+                           ms_round_by_round=ms_r, gbps_round_by_round=gbs_r, frac_round_by_round=gbs_r / peak,
+                           launches_round_by_round=l_r, note=", ".join(x for x in (note, l2) if x))
                 rows.append(row)
-                print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | {ms:.3f} | {gbs:.0f} | {gbs / peak:.2f} | {row['note']} |",
-                      flush=True)
+                print(f"| {N} | {c} | 2^{e} | {ws_bytes / 1e6:.0f} | {ms_r:.3f} | {gbs_r:.0f} | {gbs_r / peak:.2f} | {l_r} | "
+                      f"{ms:.3f} | {gbs:.0f} | {gbs / peak:.2f} | {launches} | {row['note']} |", flush=True)
                 del ws
                 torch.cuda.empty_cache()
             plan.destroy()
