@@ -198,7 +198,8 @@ cerar_status_t cerar_ring_round(cerar_plan_t* plan, float* ws, int64_t d, int k,
  * hand-off that cerar_ring_round performs (per steady round 2 reads + 1 write reach memory
  * instead of 3 + 1).  (N > 32: one thread per position runs its N workers in turn.)
  * cerar_allreduce_sim uses it on its own (it measured faster than L launches at every shape
- * tried), except for N <= 32 with d/c > 65536 not a multiple of 4 and a workspace above 64 MB. */
+ * tried); only a workspace above 64 MB with N > 32, or with d/c > 65536 not a multiple of 4,
+ * goes round by round. */
 cerar_status_t cerar_ring_rounds(cerar_plan_t* plan, float* ws, int64_t d, int k_first, int k_last,
                                  cerar_stream_t stream);
 cerar_status_t cerar_decode(cerar_plan_t* plan, const float* ws, float* out, int64_t out_stride,
