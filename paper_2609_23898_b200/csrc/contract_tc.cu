@@ -182,15 +182,19 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         afull_ph ^= 1u << bit;
                         tc_fence_after();
                         const uint32_t a_hi = tmem_base + a_col0 + ab * (2u * KC), a_lo = a_hi + KC;
-                        int ksteps = KC / 8;
                         const int rows_left = tp.K_rows - kc * KC;               // rows with data in this chunk
-                        if (rows_left < KC) ksteps = (rows_left + 7) / 8;
-                        for (int ks = 0; ks < ksteps; ++ks) {
-                            // descriptor start address advances by 8 rows x 128 B (in 16-byte units)
-                            const uint64_t boff = (uint64_t)(((kc * KC + ks * 8) * 128) >> 4);
-                            tc_mma_tf32_ts(d_tmem, a_lo + ks * 8u, bhi0 + boff, idesc, (kc | ks) != 0);
-                            tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, blo0 + boff, idesc, 1u);
-                            tc_mma_tf32_ts(d_tmem, a_hi + ks * 8u, bhi0 + boff, idesc, 1u);
+                        // descriptor start address: 8 rows x 128 B = 64 units of 16 bytes per k-step
+                        const uint64_t bh = bhi0 + (uint64_t)(kc * KC * 8), bl = blo0 + (uint64_t)(kc * KC * 8);
+                        if (rows_left >= KC) {
+#pragma unroll
+                            for (int ks = 0; ks < KC / 8; ++ks)
+                                tc_mma_tf32_ts_x3(d_tmem, a_hi + ks * 8u, a_lo + ks * 8u, bh + (uint64_t)(ks * 64),
+                                                  bl + (uint64_t)(ks * 64), idesc, ks ? 1u : (uint32_t)(kc != 0));
+                        } else {
+                            const int ksteps = (rows_left + 7) / 8;
+                            for (int ks = 0; ks < ksteps; ++ks)
+                                tc_mma_tf32_ts_x3(d_tmem, a_hi + ks * 8u, a_lo + ks * 8u, bh + (uint64_t)(ks * 64),
+                                                  bl + (uint64_t)(ks * 64), idesc, (uint32_t)((kc | ks) != 0));
                         }
                         tc_commit(a_empty + 8u * ab);      // the A buffer is free once these MMAs have read it
                     }
@@ -400,10 +404,12 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     const int tile_w = halves * HALF_M;
     tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
     if (tp.NAh > 4) tp.NAh = 4;
-    // Measured on B200 at c = 32: a second issuer per half pays once a tile has more than 4 k-steps
-    // (decode +8 .. +25 %), and costs 2 % below that (encode).  With one half per tile two issuers
-    // (even / odd tiles) are the minimum that keeps one issuing while the other drains.
-    tp.four_issuers = ((tp.K_rows + 7) / 8 > 4 || halves == 1) ? 1 : 0;
+    // Issuers per half, measured on B200 with the k-steps issued in bursts of three products: a second one
+    // (even / odd tiles) pays for 32 output columns once a chunk has more than 4 k-steps (c = 32 decode
+    // 5.3 -> 6.0 TB/s; it costs 2 % below that), and costs 10-15 % for 64 columns (c = 48, 56, 64: the
+    // products are twice as long, two issuers already keep the pipe fed).  With one half per tile two
+    // issuers (even / odd tiles) are the minimum that keeps one issuing while the other drains.
+    tp.four_issuers = (halves == 1 || (tp.Npad <= 32 && (tp.K_rows + 7) / 8 > 4)) ? 1 : 0;
     if (g_tune_tc_variant == 2) tp.four_issuers = 0;
     if (g_tune_tc_variant == 3) tp.four_issuers = 1;
     tp.tmem_cols = 32;

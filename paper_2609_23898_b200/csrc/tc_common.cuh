@@ -36,13 +36,19 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem descriptor]
-__device__ __forceinline__ void tc_mma_tf32_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc,
-                                               uint32_t accumulate) {
+// One k-step (8 rows) of the 3 x TF32 product, A in tensor memory, B through a shared-memory descriptor:
+// D (+)= A_lo B_hi, D += A_hi B_lo, D += A_hi B_hi, issued back to
+// back from one asm statement.  An issuing thread cannot start a tcgen05.mma more often than every ~54 clk
+// (measured; the pipe takes 16 clk for M128 N32 K8), and whatever integer work sits between two of them adds
+// to that, so the operands are prepared before the burst.
+__device__ __forceinline__ void tc_mma_tf32_ts_x3(uint32_t tmem_d, uint32_t tmem_a_hi, uint32_t tmem_a_lo, uint64_t bhi,
+                                                  uint64_t blo, uint32_t idesc, uint32_t accumulate_first) {
     asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}\n"
-        ::"r"(tmem_d), "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+        "{\n .reg .pred p, q;\n setp.ne.b32 p, %6, 0;\n setp.eq.b32 q, 0, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%2], %3, %5, p;\n"
+        " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %4, %5, q;\n"
+        " tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %3, %5, q;\n}\n"
+        ::"r"(tmem_d), "r"(tmem_a_hi), "r"(tmem_a_lo), "l"(bhi), "l"(blo), "r"(idesc), "r"(accumulate_first) : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
     uint32_t r[32];
