@@ -271,6 +271,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         uint32_t hi[KG], lo[KG];
 #pragma unroll
                         for (int k = 0; k < KG; ++k) {
+                            hi[k] = lo[k] = 0u;
                             if ((k & ~3) < kuse) {
                                 const float x = col[k * TILE_W + h * HALF_M];
                                 hi[k] = tf32_bits(x);
@@ -285,12 +286,9 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         if (!warp_wait(a_empty + 8u * ab, pa ^ 1u)) { failed = true; break; }
                         tc_fence_after();
                         const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC) + (uint32_t)r0;
-#pragma unroll
-                        for (int k4 = 0; k4 < KG / 4; ++k4) {
-                            if (4 * k4 < kuse) {               // uniform over the warp
-                                tc_st4(ta + 4u * k4, hi + 4 * k4);
-                                tc_st4(ta + KC + 4u * k4, lo + 4 * k4);
-                            }
+                        if (kuse > 0) {                        // uniform over the warp; rows beyond the data are zeros
+                            tc_st_cols<KG>(ta, hi);
+                            tc_st_cols<KG>(ta + KC, lo);
                         }
                         tc_wait_st();
                         tc_fence_before();

@@ -105,6 +105,19 @@ __device__ __forceinline__ void tc_st4(uint32_t taddr, const uint32_t* v) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1,%2,%3,%4};"
                  ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
 }
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+                   "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+                 : "memory");
+}
+// N consecutive columns (N a multiple of 4) with as few instructions as possible
+template <int N>
+__device__ __forceinline__ void tc_st_cols(uint32_t taddr, const uint32_t* v) {
+    if constexpr (N >= 16) { tc_st16(taddr, v); tc_st_cols<N - 16>(taddr + 16u, v + 16); }
+    else if constexpr (N >= 8) { tc_st8(taddr, v); tc_st_cols<N - 8>(taddr + 8u, v + 8); }
+    else if constexpr (N >= 4) { tc_st4(taddr, v); tc_st_cols<N - 4>(taddr + 4u, v + 4); }
+}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_alloc(uint32_t slot_smem, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
