@@ -521,3 +521,33 @@ def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
     assert plan.launch_count() - n0 == 3
     ora = run_oracle(des.U, des.R, g.view(N, d).cpu().numpy(), 1.0)
     assert max(rel_l2(out.view(N, d)[i].cpu().numpy(), ora["out"][i]) for i in range(N)) < 5e-6
+
+
+def test_rounds_in_one_launch_randomised_shapes(cerar_mod):
+    """Seeded random (N, c, p, first round): cerar_ring_rounds leaves the slots of round-by-round stepping, bit for bit."""
+    import torch
+    rng = np.random.default_rng(77)
+    s = torch_stream()
+    for trial in range(24):
+        N = int(rng.integers(2, 33))
+        c = N + int(rng.integers(0, 41))
+        p = int(rng.choice([1, 3, 4, 33, 128, 516, 1031, 4100, 9001, 38000]))
+        L = c + N - 2
+        cut = int(rng.integers(0, L))                       # rounds 1..cut one by one, the rest in one launch
+        d = c * p
+        des = Dz.custom_orthogonal(N, c, np.random.default_rng(trial))
+        g = torch.randn(N * d, device="cuda")
+        res = []
+        for how in ("each", "multi"):
+            plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+            ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
+            plan.encode(g, d, ws, d, s)
+            for k in range(1, (L if how == "each" else cut) + 1):
+                plan.ring_round(ws, d, k, s)
+            if how == "multi":
+                plan.ring_rounds(ws, d, cut + 1, L, s)
+            torch.cuda.synchronize()
+            plan.device_status(s)
+            res.append(ws)
+        assert torch.equal(torch.nan_to_num(res[0], nan=-1.0), torch.nan_to_num(res[1], nan=-1.0)), (N, c, p, cut)
+
