@@ -332,7 +332,9 @@ __global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, in
 // message lands in holds the delta its owner cancels in that very round; every thread therefore
 // reads its cancel operand at least one round early (before the barrier that precedes the store),
 // never after.  Measured on B200 (rounds of N=8, c=32, d=2^28, in the metric's bytes): DIST 1
-// 8.2 TB/s, DIST 2 10.4, DIST 3 and 4 9.7; one launch per round 7.2.
+// 8.2 TB/s, DIST 2 10.4, DIST 3 and 4 9.7; one launch per round 7.2.  Keeping the deltas that are
+// cancelled N rounds later in a register ring (N <= 8, loop unrolled by N) instead of reading them
+// again: 6.8-7.0 TB/s (100-200 registers per thread), rejected.
 template <typename VT, int PV, int DIST, int MAXT>
 __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, int k_last) {
     extern __shared__ float4 coop_smem[];
