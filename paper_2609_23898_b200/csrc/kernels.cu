@@ -557,8 +557,8 @@ cudaError_t launch_rounds_multi(const RoundArgs& a, int k_last, cudaStream_t s, 
         const int64_t pv = v4 ? a.p / 4 : a.p;
         // two vectors per lane where that still leaves every SM two blocks (measured: +2 .. +15 % on most
         // shapes); tuning: 1 / 2 force one / two
-        const int PVr = !v4 ? 1 : g_tune_rounds_coop_shape ? g_tune_rounds_coop_shape
-                                                           : (a.p / 256 >= 148 * 2 ? 2 : 1);
+        int PVr = !v4 ? 1 : g_tune_rounds_coop_shape ? g_tune_rounds_coop_shape : (a.p / 256 >= 148 * 2 ? 2 : 1);
+        if ((size_t)2 * a.N * 32 * PVr * 16 > 48 * 1024) PVr = 1;   // the hand-off tiles stay within the default 48 KB
         const unsigned blocks = (unsigned)((pv + 32 * PVr - 1) / (32 * PVr));
         const size_t smem = (size_t)2 * a.N * 32 * PVr * (v4 ? 16 : 4);
         const dim3 blk(32 * a.N);

@@ -470,7 +470,7 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
 
 
 @pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (3, 5, 1031), (16, 16, 1028), (2, 2, 4), (5, 7, 3),
-                                   (8, 16, 40004), (32, 32, 36), (7, 9, 37889), (4, 8, 76036), (33, 33, 20)])
+                                   (8, 16, 40004), (32, 32, 36), (7, 9, 37889), (4, 8, 76036), (33, 33, 20), (32, 32, 76036), (20, 24, 76032)])
 def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
     """cerar_ring_rounds (what cerar_allreduce_sim uses where it is the faster form) leaves exactly
     the slots of L calls of cerar_ring_round, in one go or in pieces, with the same counters: the
