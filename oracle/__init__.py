@@ -14,6 +14,8 @@ protocol : chunking, encoding, the ring rounds exactly as Algorithm 1 states
 designs  : the coefficient constructions (multiplicative perturbation
            construction, Vandermonde, epsilon-construction, the
            condition-number-constrained alternating least squares heuristic).
+mixed    : the ring rounds with bfloat16 messages (binary32 worker arithmetic,
+           every transmitted vector rounded to nearest-even by its sender).
 
 Pins (what each function is checked against, see tests/test_oracle_*.py):
   rounds / whole pipeline : brute-force composition Y_i = G^(i) M_i(U) for
@@ -21,7 +23,12 @@ Pins (what each function is checked against, see tests/test_oracle_*.py):
   MPC / Vandermonde / epsilon designs : Prop. 1, Prop. 2, Theorem 1's closed
       form, Eq. (error_scaling), Theorem 2 / Corollary 1 scaling laws, the
       finite-difference identity (Lemma 2) and the printed F_3.
-  kappa-constrained design : invariants only (spectral interval, kappa bound,
-      monotone least-squares steps).  The fitted U, R values themselves have no
-      published counterpart: PARITY UNPINNED for `designs.kappa_constrained`.
+  kappa-constrained design : every step against its defining property (U- and
+      R-step are stationary minimisers of the brute-force Phi, the projection is
+      the nearest matrix with singular values in the interval), the invariants of
+      the iteration, and the known optimum Phi = 0 at c = N.  The fitted U, R at
+      c > N have no published counterpart: PARITY UNPINNED for that end point.
+  bfloat16 messages : the rounding against worked values, IEEE properties and
+      torch's conversion; the rounds against Algorithm 1 where nothing rounds and
+      against the error the message precision implies.
 """

@@ -1,0 +1,71 @@
+"""Ring rounds of CERAR with low-precision messages (bfloat16 transport).
+
+Test infrastructure only (see the package docstring).  The paper leaves the combination
+with gradient quantisation open (Sec. I, Related Work: compression acts "along a direction
+orthogonal" to the coding and may be applied in conjunction).  This module states one such
+combination so that the device path has something to be compared with: Algorithm 1 (Sec. II)
+unchanged, except that every transmitted message x_{i,k} is rounded to bfloat16 by its sender;
+the receiver stores and uses the rounded vector.
+
+A rounding is a decision, and both sides must take it in the same precision (the device's):
+the workers' arithmetic here is IEEE binary32 in the order Algorithm 1 prescribes
+(C <- C + D_k ; send ; C <- received ; C <- C - D_j), on binary32 encoded vectors that are
+an INPUT (the device's own Delta, or any other).  Given the same Delta the observations Y are
+therefore fixed bit for bit.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+from . import protocol
+
+
+def round_bf16(x) -> np.ndarray:
+    """binary32 -> bfloat16 (8 significant bits), round to nearest, ties to even, returned
+    as binary32.  Written on the bit pattern: keep the upper 16 bits, round on the lower 16."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    bits = x.view(np.uint32).astype(np.uint64)
+    lower = bits & 0xFFFF
+    upper = bits >> 16
+    up = (lower > 0x8000) | ((lower == 0x8000) & ((upper & 1) == 1))
+    out = ((upper + up.astype(np.uint64)) << 16).astype(np.uint32)
+    res = out.view(np.float32).copy()
+    nan = np.isnan(x)
+    res[nan] = np.float32(np.nan)
+    return res.reshape(x.shape)
+
+
+def run_rounds_bf16(Delta32):
+    """Algorithm 1 for all N workers with binary32 worker arithmetic and bfloat16 messages.
+
+    Delta32 : list of N arrays (p x c), binary32; column j-1 is delta_{i,j}.
+    Returns Y: list of N arrays (p x (L+1)), binary32: [B_1 .. B_{N-1} | D_1 .. D_c] after
+    round L, where every B and every overwritten D holds a received (rounded) message.
+    """
+    N = len(Delta32)
+    p, c = Delta32[0].shape
+    L = protocol.num_rounds(N, c)
+    f32 = np.float32
+    D = [[np.array(Delta32[i][:, j], dtype=f32) for j in range(c)] for i in range(N)]
+    B = [[None] * (N - 1) for _ in range(N)]
+    C = [np.zeros(p, dtype=f32) for _ in range(N)]
+    for k in range(1, L + 1):
+        x = []
+        for i in range(N):
+            if k <= c:
+                C[i] = (C[i] + D[i][k - 1]).astype(f32)
+            x.append(round_bf16(C[i]))                     # what leaves worker i
+        for i in range(N):
+            C[i] = x[(i - 1) % N].copy()
+            if k <= N - 1:
+                B[i][k - 1] = C[i].copy()
+            else:
+                j = k - N + 1
+                C[i] = (C[i] - D[i][j - 1]).astype(f32)
+                D[i][j - 1] = x[(i - 1) % N].copy()
+    return [np.stack(B[i] + D[i], axis=1).astype(f32) for i in range(N)]
+
+
+def message_bytes(N: int, c: int, p: int) -> int:
+    """Bytes one worker forwards over the L rounds with 2-byte messages."""
+    return 2 * p * protocol.num_rounds(N, c)
