@@ -274,6 +274,18 @@ cerar_status_t cerar_rank_round(cerar_plan_t* plan, int rank, const float* ws, f
  * the receiver takes it straight into slot k-1 of its workspace (a contiguous row). */
 cerar_status_t cerar_rank_round_msg(cerar_plan_t* plan, int rank, const float* ws, float* msg, int64_t d, int k,
                                     cerar_stream_t stream);
+/* Low-precision transport (the paper notes that quantisation is complementary to the coding, Sec. I,
+ * Related Work; the combination is this library's): cerar_rank_round_msg_bf16 forms the same message in
+ * binary32 and leaves it in `msg` (d/c values of 2 bytes, device memory, 2-byte aligned; 8-byte aligned
+ * for the vector path) rounded to bfloat16, nearest with ties to even; cerar_rank_recv_bf16 expands a
+ * message that has arrived into slot k-1 of the receiver's workspace.  The worker's own arithmetic
+ * and its slots stay binary32; half the bytes cross the transport.  The decoded sum then carries the
+ * messages' relative rounding error of 2^-8 amplified by the decoder (kappa_2(M_i)), so this is for
+ * well-conditioned designs only. */
+cerar_status_t cerar_rank_round_msg_bf16(cerar_plan_t* plan, int rank, const float* ws, uint16_t* msg, int64_t d,
+                                         int k, cerar_stream_t stream);
+cerar_status_t cerar_rank_recv_bf16(cerar_plan_t* plan, int rank, float* ws, const uint16_t* msg, int64_t d, int k,
+                                    cerar_stream_t stream);
 cerar_status_t cerar_rank_decode(cerar_plan_t* plan, int rank, const float* ws, float* out, int64_t d,
                                  float scale, cerar_stream_t stream);
 

@@ -43,7 +43,8 @@ struct RankRoundArgs {
     int64_t p;
     int N, c, k;            // round k in 1..L
     int slot_prev, slot_cancel, slot_add, slot_land;   // filled in by the launcher (-1 = term absent)
-    int to_message;         // 1: peer_ws is a plain p-float message buffer (row 0), not a workspace
+    int to_message;         // 1: peer_ws is a plain p-float message buffer (row 0), not a workspace;
+                            // 2: a buffer of p bfloat16 values (the message rounded to nearest-even)
 };
 
 // All L rounds of up to RING_MAX_WORKERS workers in one launch (blockIdx.y = index into the arrays).
@@ -83,6 +84,8 @@ cudaError_t launch_rounds_multi(const RoundArgs& a, int k_last, cudaStream_t s, 
 // in the neighbour's workspace; the one definition that launcher and callers share.
 void rank_round_slots(int N, int c, int k, int* slot_prev, int* slot_cancel, int* slot_add, int* slot_land);
 cudaError_t launch_rank_round(RankRoundArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_rank_recv_bf16(float* slot, const unsigned short* msg, int64_t p, int num_sms, cudaStream_t s,
+                                  uint64_t* launches);
 // cooperative = true when the launch serves workers that wait on one another (all on this GPU).
 cudaError_t launch_ring_rounds(const RingFusedArgs& a, int nworkers, bool cooperative, int num_sms, cudaStream_t s,
                                uint64_t* launches);

@@ -257,6 +257,60 @@ def test_round_into_a_message_buffer_equals_the_peer_store(mods, N, c, p):
         plan.rank_round_msg(N, b.ws[0], raw[0, :p], d, 1, s)
 
 
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192 + 260), (3, 5, 1031), (2, 2, 4), (8, 32, 4100), (5, 7, 3), (4, 4, 4096)])
+def test_bf16_messages_equal_the_oracle_bit_for_bit(mods, N, c, p):
+    """Messages rounded to bfloat16 by the sender (cerar_rank_round_msg_bf16) and expanded by the receiver
+    (cerar_rank_recv_bf16).  The rounding is a decision, so the oracle takes it in the device's precision
+    on the device's own encoded vectors: the observations Y must then agree bit for bit; the decode is
+    compared within the usual tolerance, and the distance to the exact protocol is what 8-bit messages cost."""
+    import torch
+    from oracle import mixed as Mx
+    from oracle import protocol as P
+    cerar, inputs, ring = mods
+    d = c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(5 * N + c))
+    g = inputs.gradients_numpy(N, d, "normal", seed=12)
+    plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+    s = torch.cuda.current_stream().cuda_stream
+    r = ring.LocalRing(plan, d)
+    for w in r.ws:
+        w.fill_(float("nan"))
+    grads = [torch.from_numpy(g[i]).cuda() for i in range(N)]
+    r.encode(grads, s)
+    rows = c + N + 1
+    delta32 = [r.ws[i].view(rows, p)[N + 1:N + 1 + c].cpu().numpy().T.copy() for i in range(N)]      # p x c
+    raw = torch.zeros((N, p + 5), dtype=torch.bfloat16, device="cuda")
+    for k in range(1, plan.L + 1):
+        off = 1 if k % 3 == 0 else 0                      # every third round: a buffer that is only 2-byte aligned
+        for i in range(N):
+            plan.rank_round_msg_bf16(i, r.ws[i], raw[i, off:off + p], d, k, s)
+        for i in range(N):                                # "transport": worker i+1 receives worker i's buffer
+            plan.rank_recv_bf16((i + 1) % N, r.ws[(i + 1) % N], raw[i, off:off + p], d, k, s)
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    ys = ring.y_slots(plan)
+    Y_dev = [r.ws[i].view(rows, p)[ys].cpu().numpy().T for i in range(N)]                             # p x (L+1)
+    Y_ora = Mx.run_rounds_bf16(delta32)
+    for i in range(N):
+        assert np.array_equal(Y_dev[i].view(np.uint32), Y_ora[i].view(np.uint32)), i
+    outs = [torch.empty(d, device="cuda") for _ in range(N)]
+    r.decode(outs, 1.0 / N, s)
+    torch.cuda.synchronize()
+    exact = run_oracle(des.U, des.R, g, 1.0 / N)
+    worst_dec, worst_exact = 0.0, 0.0
+    for i in range(N):
+        want = P.unchunk(P.decode(Y_ora[i].astype(np.float64), des.R[i], 1.0 / N))
+        worst_dec = max(worst_dec, rel_l2(outs[i].cpu().numpy(), want))
+        worst_exact = max(worst_exact, rel_l2(outs[i].cpu().numpy(), exact["out"][i]))
+    assert worst_dec < 5e-6
+    if p >= 1000:
+        assert 1e-4 < worst_exact < 2.0 ** -8 * (c + N)   # the price of 8-bit messages with kappa ~ 1
+    with pytest.raises(cerar.CerarError):
+        plan.rank_round_msg_bf16(0, r.ws[0], raw[0, :p], d, plan.L + 1, s)
+    with pytest.raises(cerar.CerarError):
+        plan.rank_recv_bf16(N, r.ws[0], raw[0, :p], d, 1, s)
+
+
 def test_rank_level_kernels_on_symmetric_memory_allocations(mods):
     """DistributedRing keeps workspaces and counters in torch's symmetric memory.  With one GPU
     the peer mapping cannot be exercised, but the allocations can: a one-rank NCCL group,

@@ -105,6 +105,19 @@ class _CpuPlan:
         msg.copy_(x)
         self.calls.append(("round_msg", rank, k))
 
+    def rank_round_msg_bf16(self, rank, ws, msg, d, k, stream=0):
+        import torch
+        p = d // self.c
+        _land, x = self._message(self._rows(ws, d), k, 0, p)
+        msg.copy_(x.to(torch.bfloat16))                   # torch rounds to nearest, ties to even
+        self.calls.append(("round_msg_bf16", rank, k))
+
+    def rank_recv_bf16(self, rank, ws, msg, d, k, stream=0):
+        import torch
+        land = self.real.rank_round_slots(k)[3]
+        self._rows(ws, d)[land] = msg.to(torch.float32)
+        self.calls.append(("recv_bf16", rank, k))
+
     def rank_rounds_fused(self, rank, ws, peer_ws, landed_local, freed_local, landed_next, freed_prev, d, epoch,
                           stream=0):
         p = d // self.c
@@ -210,7 +223,7 @@ def test_distributed_ring_driver_with_two_gloo_ranks(fused):
             assert calls == (["encode"] + ["round"] * L + ["decode"]) * 2
 
 
-def _worker_sendrecv(rank, world, port, c, p, q):
+def _worker_sendrecv(rank, world, port, c, p, q, bf16=False):
     sys.path.insert(0, ROOT)
     import torch
     import torch.distributed as dist
@@ -223,7 +236,7 @@ def _worker_sendrecv(rank, world, port, c, p, q):
     N, d = world, c * p
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(6))
     plan = _CpuPlan(cerar.Plan.create_custom(N, c, des.U, des.R, host_only=True))
-    r = ring.SendRecvRing(plan, d, device=torch.device("cpu"))
+    r = ring.SendRecvRing(plan, d, device=torch.device("cpu"), bf16_messages=bf16)
     errs = []
     for rep in range(2):
         rng = np.random.default_rng(300 + rep)
@@ -256,3 +269,27 @@ def test_send_receive_ring_driver_with_gloo_ranks(N, c):
     for rank, errs, calls in res:
         assert max(errs) < 5e-6, errs
         assert calls == (["encode"] + ["round_msg"] * L + ["decode"]) * 2
+
+
+def test_send_receive_ring_driver_with_bf16_messages():
+    """The driver's bfloat16 transport: round on the sender, move 2-byte buffers, expand on the receiver
+    (stand-ins for the two calls use torch's own bfloat16 conversion).  With orthogonal encoders the
+    result is the exact mean up to the messages' 2^-8 rounding."""
+    import torch.multiprocessing as mp
+    sys.path.insert(0, ROOT)
+    N, c, p = 3, 4, 37
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker_sendrecv, args=(r, N, port, c, p, q, True)) for r in range(N)]
+    for pr in procs:
+        pr.start()
+    res = sorted(q.get(timeout=240) for _ in procs)
+    for pr in procs:
+        pr.join(timeout=60)
+        assert pr.exitcode == 0
+    L = c + N - 2
+    for rank, errs, calls in res:
+        assert 1e-5 < max(errs) < 2.0 ** -8 * (c + N), errs
+        assert calls == (["encode"] + ["round_msg_bf16", "recv_bf16"] * L + ["decode"]) * 2
+
