@@ -400,6 +400,27 @@ def main():
                                  "+ 1 write reach memory instead of the 3 + 1 that the algorithmic bytes count"
                                  if n_one == 3 else "")}
 
+    if n_one == 3:
+        # the same three launches with an event between them (a few aggregations, outside the figure above)
+        ph = []
+        for _ in range(min(K, 5)):
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            e[0].record()
+            plan.encode(grads, d, ws, d, stream)
+            e[1].record()
+            plan.ring_rounds(ws, d, 1, L, stream)
+            e[2].record()
+            plan.decode(ws, out, d, d, scale, stream)
+            e[3].record()
+            torch.cuda.synchronize()
+            ph.append([e[i].elapsed_time(e[i + 1]) for i in range(3)])
+        ph = np.median(np.array(ph), axis=0)
+        line["one_call"]["per_launch"] = {
+            "encode": {"ms": float(ph[0]), "GBps": ab["encode"] / ph[0] / 1e6},
+            "rounds_one_launch": {"ms": float(ph[1]), "GBps_in_metric_bytes": ab["rounds"] / ph[1] / 1e6},
+            "decode": {"ms": float(ph[2]), "GBps": ab["decode"] / ph[2] / 1e6}}
+        plan.device_status(stream)
+
     des = None
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
