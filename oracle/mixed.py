@@ -10,8 +10,8 @@ the receiver stores and uses the rounded vector.
 A rounding is a decision, and both sides must take it in the same precision (the device's):
 the workers' arithmetic here is IEEE binary32 in the order Algorithm 1 prescribes
 (C <- C + D_k ; send ; C <- received ; C <- C - D_j), on binary32 encoded vectors that are
-an INPUT (the device's own Delta, or any other).  Given the same Delta the observations Y are
-therefore fixed bit for bit.
+an INPUT (seeded synthetic ones, or an fp64 encode cast to binary32).  Given the same Delta the
+observations Y are therefore fixed bit for bit.
 """
 from __future__ import annotations
 
