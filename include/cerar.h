@@ -140,6 +140,15 @@ cerar_status_t cerar_plan_info(cerar_plan_t* plan, cerar_plan_info_t* out);
  * (equally spaced in [-1, 1]). */
 cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, const double* h,
                                   double* gamma_out);
+/* A deterministic choice of H from B (the paper's appendix on the numerical experiments mentions
+ * that H may be "chosen in a deterministic manner using the constructed B" and gives no rule; this
+ * is the library's reading): coordinate ascent on gamma(B, H).  Start: h as passed (use_start != 0)
+ * or equally spaced in [-1, 1]; scaled to max|h| = 1; coordinates are visited in order, each moves
+ * to the first of `grid` equally spaced values of [-1, 1] with the largest gamma if that beats the
+ * current gamma and leaves max|h| = 1; at most `sweeps` passes.  h (c doubles, host) receives the
+ * result, which goes into cerar_options_t.h; gamma_out / moves_out may be NULL.  Host only. */
+cerar_status_t cerar_design_optimize_h(int N, int c, const double* B, uint64_t seed, double* h, int use_start,
+                                       int sweeps, int grid, double* gamma_out, int* moves_out);
 
 /* Smallest d' >= d that is a multiple of 4c.  The protocol needs c | d (the caller pads the
  * gradient with zeros, Sec. II); the fast kernels additionally need rows of p = d/c values to

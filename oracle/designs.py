@@ -225,6 +225,42 @@ def gamma(B, h, N: int, c: int) -> float:
     return min(float(np.linalg.svd(k_limit(B, h, N, c, l), compute_uv=False)[-1]) for l in range(N))
 
 
+def optimize_h(B, N: int, c: int, h0=None, sweeps: int = 2, grid: int = 17):
+    """A deterministic choice of the diagonal H from B.  The paper only says that H may be "chosen in a
+    deterministic manner using the constructed B" (appendix on the numerical experiments) and that the
+    analysis needs gamma(B, H) > 0 (Sec. II-C); the reading taken here is coordinate ascent on gamma:
+    start from h0 (default: equally spaced in [-1, 1]); visit the coordinates j = 0..c-1 in order; for
+    each, try the `grid` equally spaced values of [-1, 1] in increasing order and move h_j to the first
+    value that gives the largest gamma, if that is larger than the current one (by more than 1e-12
+    relative) and leaves max|h| = 1 (so that ||H||_2 = 1 stays comparable between choices); stop after
+    `sweeps` passes or a pass without a move.  Returns (h, gamma(B, h), moves)."""
+    B = np.asarray(B, dtype=np.float64)
+    h = np.array(default_h(c) if h0 is None else h0, dtype=np.float64)
+    h = h / np.abs(h).max()
+    cand = [-1.0 + 2.0 * t / (grid - 1) for t in range(grid)]
+    best = gamma(B, h, N, c)
+    moves = 0
+    for _ in range(sweeps):
+        moved = False
+        for j in range(c):
+            keep, best_j, val_j = h[j], None, best
+            for g in cand:
+                if g == keep:
+                    continue
+                h[j] = g
+                if np.abs(h).max() < 1.0:
+                    continue
+                v = gamma(B, h, N, c)
+                if v > val_j * (1 + 1e-12):
+                    val_j, best_j = v, g
+            h[j] = keep if best_j is None else best_j
+            if best_j is not None:
+                best, moved, moves = val_j, True, moves + 1
+        if not moved:
+            break
+    return h, best, moves
+
+
 # ---------------------------------------------------------- kappa-constrained design
 
 def _ls_R(U, N, c):

@@ -70,6 +70,8 @@ lib.cerar_plan_get_R.argtypes = [_vp, C.c_int, C.POINTER(C.c_double)]
 lib.cerar_plan_info.argtypes = [_vp, C.POINTER(PlanInfo)]
 lib.cerar_design_gamma.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double), C.c_uint64, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double)]
+lib.cerar_design_optimize_h.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_uint64, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                        C.POINTER(C.c_double), C.POINTER(C.c_int)]
 lib.cerar_padded_length.argtypes = [_vp, _i64]
 lib.cerar_padded_length.restype = _i64
 lib.cerar_workspace_bytes.argtypes = [_vp, _i64]
@@ -136,6 +138,17 @@ def design_gamma(N: int, c: int, B=None, h=None, seed: int = 0) -> float:
     _check(lib.cerar_design_gamma(N, c, Ba.ctypes.data_as(dp) if Ba is not None else None, seed,
                                   ha.ctypes.data_as(dp) if ha is not None else None, C.byref(out)))
     return out.value
+
+
+def optimize_h(N: int, c: int, B=None, h0=None, sweeps: int = 2, grid: int = 17, seed: int = 0):
+    """cerar_design_optimize_h: coordinate ascent on gamma(B, H).  Returns (h, gamma, moves)."""
+    import numpy as np
+    Ba = None if B is None else np.ascontiguousarray(B, dtype=np.float64)
+    h = np.zeros(c, dtype=np.float64) if h0 is None else np.array(h0, dtype=np.float64)
+    g, m = C.c_double(0.0), C.c_int(0)
+    _check(lib.cerar_design_optimize_h(N, c, None if Ba is None else Ba.ctypes.data, seed, h.ctypes.data,
+                                       0 if h0 is None else 1, sweeps, grid, C.byref(g), C.byref(m)))
+    return h, g.value, m.value
 
 
 def select_h(N: int, c: int, B, candidates):

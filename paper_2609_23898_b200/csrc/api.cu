@@ -259,6 +259,28 @@ cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, 
     return CERAR_OK;
 }
 
+cerar_status_t cerar_design_optimize_h(int N, int c, const double* B, uint64_t seed, double* h, int use_start,
+                                       int sweeps, int grid, double* gamma_out, int* moves_out) {
+    if (!h || N < 2 || c < N) return fail(CERAR_ERR_INVALID_ARG, "need 2 <= N <= c and a buffer for h");
+    if (sweeps < 1 || grid < 3 || grid > 1025) return fail(CERAR_ERR_INVALID_ARG, "need sweeps >= 1 and 3 <= grid <= 1025");
+    std::vector<double> Bdef;
+    if (!B) { Bdef = cerar::default_base_matrix(N, c, seed); B = Bdef.data(); }
+    for (int i = 0; i < N * c; ++i) if (!std::isfinite(B[i])) return fail(CERAR_ERR_INVALID_ARG, "B is not finite");
+    if (!use_start) {
+        const std::vector<double> h0 = cerar::default_nodes(c);
+        for (int j = 0; j < c; ++j) h[j] = h0[j];
+    }
+    bool any = false;
+    for (int j = 0; j < c; ++j) {
+        if (!std::isfinite(h[j])) return fail(CERAR_ERR_INVALID_ARG, "h is not finite");
+        any = any || h[j] != 0.0;
+    }
+    if (!any) return fail(CERAR_ERR_INVALID_ARG, "the start h is zero");
+    const double g = cerar::optimize_h(N, c, B, h, sweeps, grid, moves_out);
+    if (gamma_out) *gamma_out = g;
+    return CERAR_OK;
+}
+
 int64_t cerar_padded_length(const cerar_plan_t* P, int64_t d) {
     if (!P || d <= 0) return 0;
     const int64_t q = 4 * (int64_t)P->host.c;

@@ -303,6 +303,38 @@ double k_limit_gamma(int N, int c, const double* B, const double* h) {
     return gamma;
 }
 
+double optimize_h(int N, int c, const double* B, double* h, int sweeps, int grid, int* moves_out) {
+    double hmax = 0;
+    for (int j = 0; j < c; ++j) hmax = std::max(hmax, std::fabs(h[j]));
+    if (hmax > 0) for (int j = 0; j < c; ++j) h[j] /= hmax;
+    std::vector<double> cand(grid);
+    for (int t = 0; t < grid; ++t) cand[t] = -1.0 + 2.0 * t / (grid - 1);
+    double best = k_limit_gamma(N, c, B, h);
+    int moves = 0;
+    for (int sweep = 0; sweep < sweeps; ++sweep) {
+        bool moved = false;
+        for (int j = 0; j < c; ++j) {
+            const double keep = h[j];
+            double val_j = best, best_j = keep;
+            bool found = false;
+            for (int t = 0; t < grid; ++t) {
+                if (cand[t] == keep) continue;
+                h[j] = cand[t];
+                double m = 0;
+                for (int q = 0; q < c; ++q) m = std::max(m, std::fabs(h[q]));
+                if (m < 1.0) continue;                         // ||H||_2 = 1 stays: choices remain comparable
+                const double v = k_limit_gamma(N, c, B, h);
+                if (v > val_j * (1 + 1e-12)) { val_j = v; best_j = cand[t]; found = true; }
+            }
+            h[j] = best_j;
+            if (found) { best = val_j; moved = true; ++moves; }
+        }
+        if (!moved) break;
+    }
+    if (moves_out) *moves_out = moves;
+    return best;
+}
+
 double phi_direct(const HostPlan& P) { return phi_blocks<ld>(P); }
 
 double kappa_U_max(const HostPlan& P) {

@@ -37,6 +37,9 @@ int build_kappa(int N, int c, double kappa_max, const double* B, const double* h
 // epsilon-construction assumes positive (Sec. II-C): K^(l) stacks B, BH, .., BH^(beta-1) and, when
 // c = beta N + s with s > 0, the rows {l, .., l+s-1} mod N of BH^beta.  H = diag(h).
 double k_limit_gamma(int N, int c, const double* B, const double* h);
+// Coordinate ascent on gamma over `grid` equally spaced values of [-1, 1] per coordinate; h is the start and the
+// result (scaled to max|h| = 1 first); returns gamma of the result.
+double optimize_h(int N, int c, const double* B, double* h, int sweeps, int grid, int* moves_out);
 
 // Phi(U,R) from the block form sum_{i,s} ||U_{i-1-s} W_s(R_i) - I||_F^2.
 double phi_direct(const HostPlan& P);

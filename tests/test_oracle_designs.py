@@ -319,6 +319,37 @@ def test_gamma_special_case_and_lower_bound_on_sigma_min():
             assert smin <= 1e3 * eps ** r_star            # and not a different power of eps
 
 
+@pytest.mark.parametrize("N,c", [(3, 5), (4, 8), (2, 6)])
+def test_optimize_h_is_a_coordinatewise_maximum_of_gamma(N, c):
+    """The deterministic H: gamma never decreases, ||H|| stays 1, the result cannot be improved by moving
+    any single coordinate to any grid value (brute force), and it is reproducible."""
+    B = _rng_B(N, c, 21)
+    grid = 9
+    h0 = Dz.default_h(c)
+    g0 = Dz.gamma(B, np.asarray(h0, float), N, c)
+    h, g, moves = Dz.optimize_h(B, N, c, sweeps=6, grid=grid)
+    assert g >= g0 and moves >= 1 and g > g0 * 1.01                 # it does find something better than the start
+    assert g == pytest.approx(Dz.gamma(B, h, N, c), rel=1e-12)
+    assert np.abs(h).max() == 1.0
+    cand = [-1.0 + 2.0 * t / (grid - 1) for t in range(grid)]
+    assert all(min(abs(x - g_) for g_ in cand) < 1e-15 or x in np.asarray(h0, float) / np.abs(h0).max() for x in h)
+    for j in range(c):                                              # no single move helps any more
+        for v in cand:
+            t = h.copy()
+            t[j] = v
+            if np.abs(t).max() < 1.0:
+                continue
+            assert Dz.gamma(B, t, N, c) <= g * (1 + 1e-9), (j, v)
+    h2, g2, _ = Dz.optimize_h(B, N, c, sweeps=6, grid=grid)
+    assert np.array_equal(h, h2) and g == g2
+    # and the design built with it is a valid epsilon-construction with a smaller kappa at the same Phi order
+    des0 = Dz.epsilon(N, c, 1e-2, B)
+    des1 = Dz.epsilon(N, c, 1e-2, B, h=h)
+    k0 = max(P.kappa2(P.m_matrix(des0.U, i)) for i in range(N))
+    k1 = max(P.kappa2(P.m_matrix(des1.U, i)) for i in range(N))
+    assert P.phi(des1.U, des1.R) < 10 * P.phi(des0.U, des0.R) and k1 < 10 * k0
+
+
 # ------------------------------------------------------------------ kappa-constrained
 
 def test_kappa_constrained_invariants():

@@ -212,3 +212,34 @@ def test_padded_length():
     assert plan.padded_length(1_414_647_808) == 1_414_647_840 and 1_414_647_840 % 48 == 0
     assert plan.padded_length(48) == 48 and plan.padded_length(49) == 96 and plan.padded_length(1) == 48
     assert plan.padded_length(0) == 0
+
+
+@pytest.mark.parametrize("N,c", [(3, 5), (4, 8), (2, 6), (4, 12)])
+def test_optimize_h_matches_the_oracle_and_feeds_a_plan(N, c):
+    """cerar_design_optimize_h against oracle.designs.optimize_h (same start, same grid, same B): the same
+    diagonal, the same gamma; and the diagonal goes into a plan whose diagnostics are the oracle's."""
+    from oracle import designs as Dz
+    from oracle import protocol as P
+    from paper_2609_23898_b200 import cerar
+    B = np.random.default_rng(30 + N + c).standard_normal((N, c))
+    h_o, g_o, m_o = Dz.optimize_h(B, N, c, sweeps=3, grid=9)
+    h_l, g_l, m_l = cerar.optimize_h(N, c, B, sweeps=3, grid=9)
+    assert m_l == m_o and np.allclose(h_l, h_o, atol=1e-15)
+    assert g_l == pytest.approx(g_o, rel=1e-9)
+    assert g_l >= cerar.design_gamma(N, c, B) * (1 - 1e-12)
+    # a start of the caller's, here the reversed default
+    h0 = np.linspace(1.0, -1.0, c)
+    h_o2, g_o2, _ = Dz.optimize_h(B, N, c, h0=h0, sweeps=2, grid=9)
+    h_l2, g_l2, _ = cerar.optimize_h(N, c, B, h0=h0, sweeps=2, grid=9)
+    assert np.allclose(h_l2, h_o2, atol=1e-15) and g_l2 == pytest.approx(g_o2, rel=1e-9)
+    plan = cerar.Plan.create(N, c, cerar.EPSILON, 1e-2, B=B, h=h_l, host_only=True)
+    des = Dz.epsilon(N, c, 1e-2, B, h=h_o)
+    info = plan.info()
+    assert info["phi"] == pytest.approx(P.phi(des.U, des.R), rel=1e-6)
+    for i in range(N):
+        assert np.allclose(plan.get_U(i), des.U[i], rtol=1e-8, atol=1e-8 * np.abs(des.U[i]).max())
+    with pytest.raises(cerar.CerarError):
+        cerar.optimize_h(N, c, B, h0=np.zeros(c))
+    with pytest.raises(cerar.CerarError):
+        cerar.optimize_h(N, c, B, grid=2)
+
