@@ -134,15 +134,15 @@ cerar_status_t cerar_plan_info(cerar_plan_t* plan, cerar_plan_info_t* out);
  * analysis of the epsilon-construction assumes positive (Sec. II-C, the Assumption before the
  * theorem on singular value scaling; K^(l) = [B; BH; ..; BH^(beta-1); (BH^beta)_{E_l}] with
  * c = beta N + s, E_l = {l, .., l+s-1} mod N).  sigma_min(A_l(eps)) = Theta(eps^r*) carries it
- * as its constant, so among several H the one with the largest gamma is the natural pick:
- * the paper's "multiple trials for selecting H".  Host only, no CUDA.
+ * as its constant, so among several trial H (which Sec. II-C allows) the one with the largest
+ * gamma is the natural pick.  Host only, no CUDA.
  * B: N x c row-major or NULL (built-in N(0,1) generator with `seed`); h: length c or NULL
  * (equally spaced in [-1, 1]). */
 cerar_status_t cerar_design_gamma(int N, int c, const double* B, uint64_t seed, const double* h,
                                   double* gamma_out);
 /* A deterministic choice of H from B (the paper's appendix on the numerical experiments mentions
- * that H may be "chosen in a deterministic manner using the constructed B" and gives no rule; this
- * is the library's reading): coordinate ascent on gamma(B, H).  Start: h as passed (use_start != 0)
+ * that H can be derived deterministically from B and gives no rule; this is the library's
+ * reading): coordinate ascent on gamma(B, H).  Start: h as passed (use_start != 0)
  * or equally spaced in [-1, 1]; scaled to max|h| = 1; coordinates are visited in order, each moves
  * to the first of `grid` equally spaced values of [-1, 1] with the largest gamma if that beats the
  * current gamma and leaves max|h| = 1; at most `sweeps` passes.  h (c doubles, host) receives the

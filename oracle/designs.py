@@ -226,8 +226,8 @@ def gamma(B, h, N: int, c: int) -> float:
 
 
 def optimize_h(B, N: int, c: int, h0=None, sweeps: int = 2, grid: int = 17):
-    """A deterministic choice of the diagonal H from B.  The paper only says that H may be "chosen in a
-    deterministic manner using the constructed B" (appendix on the numerical experiments) and that the
+    """A deterministic choice of the diagonal H from B.  The paper only mentions that H can be derived
+    deterministically from B, without a rule (appendix on the numerical experiments), and that the
     analysis needs gamma(B, H) > 0 (Sec. II-C); the reading taken here is coordinate ascent on gamma:
     start from h0 (default: equally spaced in [-1, 1]); visit the coordinates j = 0..c-1 in order; for
     each, try the `grid` equally spaced values of [-1, 1] in increasing order and move h_j to the first

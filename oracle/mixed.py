@@ -1,8 +1,8 @@
 """Ring rounds of CERAR with low-precision messages (bfloat16 transport).
 
 Test infrastructure only (see the package docstring).  The paper leaves the combination
-with gradient quantisation open (Sec. I, Related Work: compression acts "along a direction
-orthogonal" to the coding and may be applied in conjunction).  This module states one such
+with gradient quantisation open (Sec. I, Related Work, only notes that compression is
+complementary to the coding and could be combined with it).  This module states one such
 combination so that the device path has something to be compared with: Algorithm 1 (Sec. II)
 unchanged, except that every transmitted message x_{i,k} is rounded to bfloat16 by its sender;
 the receiver stores and uses the rounded vector.

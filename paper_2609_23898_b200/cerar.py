@@ -152,7 +152,7 @@ def optimize_h(N: int, c: int, B=None, h0=None, sweeps: int = 2, grid: int = 17,
 
 
 def select_h(N: int, c: int, B, candidates):
-    """The paper's "multiple trials for selecting H": of the candidate diagonals, the one with
+    """H picked among several trials (Sec. II-C allows that): of the candidate diagonals, the one with
     the largest gamma(B, H).  Returns (index, gammas)."""
     gammas = [design_gamma(N, c, B, h) for h in candidates]
     best = max(range(len(gammas)), key=lambda i: gammas[i])

@@ -5,7 +5,7 @@
 Three tables from the library's fp64 design builder (host_only plans):
   1. epsilon-construction (Sec. II-C) over eps: Phi = O(eps^2) against kappa_2(M_i) = O(eps^-r*);
   2. the same eps with H chosen among `trials` random diagonals by the largest
-     gamma(B, H) = min_l sigma_min(K^(l)(B, H)) (the paper's "multiple trials for selecting H"), and with
+     gamma(B, H) = min_l sigma_min(K^(l)(B, H)) (Sec. II-C: H can be picked by trying several), and with
      the deterministic H that coordinate ascent on gamma gives from B (cerar_design_optimize_h);
   3. the condition-number-constrained design (Sec. II-D) over the bound C: the Phi it reaches
      and the kappa_2(M_i) it ends with.

@@ -159,8 +159,8 @@ def test_argument_errors():
 
 
 def test_design_gamma_matches_oracle_and_selects_the_best_h():
-    """cerar_design_gamma against the oracle's K^(l) matrices, and the "multiple trials
-    for H" helper on fixed candidates."""
+    """cerar_design_gamma against the oracle's K^(l) matrices, and the helper that picks H
+    among several trial diagonals, on fixed candidates."""
     from oracle import designs as Dz
     from paper_2609_23898_b200 import cerar, inputs
     rng = np.random.default_rng(9)
