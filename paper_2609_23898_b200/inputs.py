@@ -95,3 +95,20 @@ def fill_gradients_torch(dst, workload: str = "normal", seed: int = 0, std: floa
         else:
             raise ValueError(workload)
     return dst
+
+
+def structured_base(N: int, c: int, seed: int = 0):
+    """(B, h) for a block-structured design: row r of the N x c base matrix is non-zero on its own c/N
+    columns only (i.i.d. N(0,1) there), and the diagonal h repeats c/N equally spaced values of [-1, 1] in
+    every block.  Needs N | c.  Seeded input data only: what the design does with them is the library's
+    (and, separately, the oracle's) business."""
+    if c % N:
+        raise ValueError("a block-structured base matrix needs N | c")
+    beta = c // N
+    rng = np.random.default_rng(77000 + seed)
+    B = np.zeros((N, c))
+    for r in range(N):
+        B[r, r * beta:(r + 1) * beta] = rng.standard_normal(beta)
+    hb = np.linspace(-1.0, 1.0, beta) if beta > 1 else np.ones(1)
+    return B, np.tile(hb, N)
+

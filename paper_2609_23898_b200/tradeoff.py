@@ -2,12 +2,14 @@
 
   python -m paper_2609_23898_b200.tradeoff [--N 4] [--c 12] [--trials 16] [--seed 0]
 
-Three tables from the library's fp64 design builder (host_only plans):
+Four tables from the library's fp64 design builder (host_only plans):
   1. epsilon-construction (Sec. II-C) over eps: Phi = O(eps^2) against kappa_2(M_i) = O(eps^-r*);
   2. the same eps with H chosen among `trials` random diagonals by the largest
      gamma(B, H) = min_l sigma_min(K^(l)(B, H)) (Sec. II-C: H can be picked by trying several), and with
      the deterministic H that coordinate ascent on gamma gives from B (cerar_design_optimize_h);
-  3. the condition-number-constrained design (Sec. II-D) over the bound C: the Phi it reaches
+  3. the same eps with a block-structured base matrix (row r of B non-zero on its own c/N columns only),
+     for which U_k and R_i are block sparse;
+  4. the condition-number-constrained design (Sec. II-D) over the bound C: the Phi it reaches
      and the kappa_2(M_i) it ends with.
 Phi is the squared least-squares error of Eq. (F); the relative error of the decoded sum is
 about sqrt(Phi / (N c)) for i.i.d. gradients.
@@ -63,6 +65,20 @@ def main():
                 out.append((float("nan"),) * 4)
         print(f"| {eps:g} | {out[0][0]:.3e} / {out[1][0]:.3e} / {out[2][0]:.3e} | {out[0][1]:.3e} | {out[1][1]:.3e} | "
               f"{out[2][1]:.3e} | {out[0][3]:.2e} | {out[1][3]:.2e} | {out[2][3]:.2e} |", flush=True)
+    if c % N == 0 and c > N:
+        # block-structured base matrix (row r on its own c/N columns): U_k, R_i come out block sparse
+        Bs, hs = inputs.structured_base(N, c, args.seed)
+        print(f"\nblock-structured B (c/N = {c // N} non-zeros per column of U_k instead of {c}): gamma {cerar.design_gamma(N, c, Bs, hs):.3e}")
+        print("\n| eps | Phi | kappa_M | max abs U |")
+        print("|---|---|---|---|")
+        for eps in (1e-1, 3e-2, 1e-2, 3e-3, 1e-3):
+            try:
+                p = cerar.Plan.create(N, c, cerar.EPSILON, eps, B=Bs, h=hs, host_only=True)
+                r = row(p)
+                p.destroy()
+                print(f"| {eps:g} | {r[0]:.3e} | {r[1]:.3e} | {r[3]:.2e} |", flush=True)
+            except cerar.CerarError as e:
+                print(f"| {eps:g} | - | - | {e} |", flush=True)
     print("\n| C (bound on kappa_M) | Phi reached | kappa_M reached | ALS iterations |")
     print("|---|---|---|---|")
     for C in (1e2, 1e3, 1e4, 1e5, 1e6):

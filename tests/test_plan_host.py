@@ -243,3 +243,34 @@ def test_optimize_h_matches_the_oracle_and_feeds_a_plan(N, c):
     with pytest.raises(cerar.CerarError):
         cerar.optimize_h(N, c, B, grid=2)
 
+
+@pytest.mark.parametrize("N,c", [(4, 8), (4, 16), (8, 32)])
+def test_block_structured_base_matrix_gives_block_sparse_designs(N, c):
+    """A base matrix whose rows have disjoint supports (row r on its own c/N columns) makes every window A_l
+    block diagonal up to a permutation, hence U_k and the decoder rows block sparse: c/N non-zeros per column
+    of U_k instead of c.  Prop. 1 and Prop. 2 hold for any B with invertible windows, so the design is as valid
+    as a dense one; the library and the oracle agree on it, zeros included."""
+    from oracle import designs as Dz
+    from oracle import protocol as P
+    from paper_2609_23898_b200 import cerar, inputs
+    B, h = inputs.structured_base(N, c, 1)
+    beta = c // N
+    eps = 1e-2
+    plan = cerar.Plan.create(N, c, cerar.EPSILON, eps, B=B, h=h, host_only=True)
+    des = Dz.epsilon(N, c, eps, B, h=h)
+    D = 1.0 + eps * h
+    assert P.phi(des.U, des.R) == pytest.approx(N * (N - 1) / 2 * np.sum((1.0 / D - 1.0) ** 2), rel=1e-6)   # Prop. 2 (phi from fp64 U, R with kappa up to 1e9)
+    for i in range(N):
+        U, R = plan.get_U(i), plan.get_R(i)
+        assert np.array_equal(U != 0, des.U[i] != 0) and np.array_equal(R != 0, des.R[i] != 0)
+        assert np.all((U != 0).sum(axis=0) == beta) and np.all((U != 0).sum(axis=1) == beta)
+        assert np.all((R != 0).sum(axis=1) == beta)                      # a decoder row is one a_l: one block
+        assert np.allclose(U, des.U[i], rtol=1e-9, atol=1e-9 * np.abs(des.U[i]).max())
+        assert np.allclose(R, des.R[i], rtol=1e-9, atol=1e-12)
+    # the decoded sum is exact up to the O(eps) of every MPC design (worker 0 exactly)
+    rng = np.random.default_rng(2)
+    g = [rng.standard_normal(c * 3) for _ in range(N)]
+    res = P.allreduce(g, des.U, des.R, 1.0)
+    assert P.rel_l2(res["out"][0], P.exact_sum(g)) < 1e-6 * max(1.0, P.kappa2(P.m_matrix(des.U, 0)) * 1e-10)
+    assert max(P.rel_l2(res["out"][i], P.exact_sum(g)) for i in range(N)) < 0.2
+
