@@ -355,7 +355,8 @@ def test_full_size_config2(cerar_mod):
 
 
 @pytest.mark.parametrize("N,c,p", [(2, 2, 1), (2, 3, 5), (2, 16, 4), (3, 3, 4), (7, 7, 12), (4, 130, 8), (2, 512, 4),
-                                   (16, 16, 4), (8, 32, 4), (8, 32, 124), (4, 64, 132), (12, 36, 260)])
+                                   (16, 16, 4), (8, 32, 4), (8, 32, 124), (4, 64, 132), (12, 36, 260), (4, 160, 516), (8, 512, 36),
+                                   (32, 48, 260)])
 def test_degenerate_and_extreme_shapes(cerar_mod, N, c, p):
     """Smallest ring (N = 2, where L = c), c = N (the classic case), a single position,
     fewer positions than one tile or one vector, the largest c the library accepts
