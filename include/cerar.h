@@ -401,6 +401,7 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *                                   for workspaces up to this many MB (default rule: see
  *                                   cerar_ring_rounds)
  *   "rounds_coop_shape"             vectors per lane of the warp-per-worker kernel (0 = automatic, 1, 2)
+ *   "rounds_hints"                  L2 residency hints of that kernel (0 = automatic: from N = 8, 1 = off, 2 = on)
  *   "rounds_multi_form"             kernel of cerar_ring_rounds: 0 = warp per worker (16-byte
  *                                   accesses where there are enough positions), 3 = the same with
  *                                   4-byte accesses, 1 = thread per position

@@ -742,6 +742,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "rounds_one_launch_mb") cerar::g_tune_rounds_one_launch_mb = value;
     else if (n == "rounds_multi_form") cerar::g_tune_rounds_multi_form = value;
     else if (n == "rounds_coop_shape") cerar::g_tune_rounds_coop_shape = value;
+    else if (n == "rounds_hints") cerar::g_tune_rounds_hints = value;
     else if (n == "ring_tile") cerar::g_tune_ring_tile = (value / 4) * 4;
     else return -1;
     return 0;

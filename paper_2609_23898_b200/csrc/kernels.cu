@@ -335,6 +335,30 @@ __global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, in
 // 8.2 TB/s, DIST 2 10.4, DIST 3 and 4 9.7; one launch per round 7.2.  Keeping the deltas that are
 // cancelled N rounds later in a register ring (N <= 8, loop unrolled by N) instead of reading them
 // again: 6.8-7.0 TB/s (100-200 registers per thread), rejected.
+// L2 residency hints for the one-launch rounds: a delta is read twice, N rounds apart (added, then
+// cancelled): the first read asks L2 to keep the line, the second lets it go; a stored message is not
+// read again before the decode.
+__device__ __forceinline__ uint64_t policy_keep() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 ld_keep(const float4* p, uint64_t pol) {
+    float4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.f32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ float ld_keep(const float* p, uint64_t pol) {
+    float v;
+    asm volatile("ld.global.L2::cache_hint.f32 %0, [%1], %2;" : "=f"(v) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ float4 ld_last_use(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ float ld_last_use(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(float* p, float v) { __stcs(p, v); }
+
 template <typename VT, int PV, int DIST, int MAXT>
 __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, int k_last) {
     extern __shared__ float4 coop_smem[];
@@ -353,6 +377,8 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
     VT* nxt = reinterpret_cast<VT*>(a.ws) + (int64_t)dst * wstride + v0;
     grid_dependency_wait();
     int k = a.k;
+    const bool hints = a.reverse != 0;                          // set by the launcher
+    const uint64_t pol = policy_keep();
     // operands of rounds k .. k+DIST-1 (index t = rounds ahead); absent terms are zero
     VT y[PV], da[DIST][PV], dc[DIST][PV];
 #pragma unroll
@@ -364,8 +390,8 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
             const int kt = k + t;
             da[t][j] = dc[t][j] = vzero<VT>();
             if (live[j] && kt <= k_last) {
-                if (kt <= c) da[t][j] = own[(int64_t)(N - 1 + kt) * pv + 32 * j];
-                if (kt - 1 >= N) dc[t][j] = own[(int64_t)(kt - 1) * pv + 32 * j];
+                if (kt <= c) da[t][j] = hints ? ld_keep(own + (int64_t)(N - 1 + kt) * pv + 32 * j, pol) : own[(int64_t)(N - 1 + kt) * pv + 32 * j];
+                if (kt - 1 >= N) dc[t][j] = hints ? ld_last_use(own + (int64_t)(kt - 1) * pv + 32 * j) : own[(int64_t)(kt - 1) * pv + 32 * j];
             }
         }
     }
@@ -375,7 +401,7 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
 #pragma unroll
         for (int j = 0; j < PV; ++j) {
             const VT x = combine(y[j], dc[0][j], da[0][j]);
-            if (live[j]) nxt[(int64_t)(k - 1) * pv + 32 * j] = x;
+            if (live[j]) { if (hints) st_stream(nxt + (int64_t)(k - 1) * pv + 32 * j, x); else nxt[(int64_t)(k - 1) * pv + 32 * j] = x; }
             hb[(dst * PV + j) * 32 + lane] = x;
         }
         // shift the operand queue and fetch round k + DIST (its slots are not written before that round)
@@ -386,8 +412,8 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
             for (int t = 0; t + 1 < DIST; ++t) { da[t][j] = da[t + 1][j]; dc[t][j] = dc[t + 1][j]; }
             da[DIST - 1][j] = dc[DIST - 1][j] = vzero<VT>();
             if (live[j] && kn <= k_last) {
-                if (kn <= c) da[DIST - 1][j] = own[(int64_t)(N - 1 + kn) * pv + 32 * j];
-                if (kn - 1 >= N) dc[DIST - 1][j] = own[(int64_t)(kn - 1) * pv + 32 * j];
+                if (kn <= c) da[DIST - 1][j] = hints ? ld_keep(own + (int64_t)(N - 1 + kn) * pv + 32 * j, pol) : own[(int64_t)(N - 1 + kn) * pv + 32 * j];
+                if (kn - 1 >= N) dc[DIST - 1][j] = hints ? ld_last_use(own + (int64_t)(kn - 1) * pv + 32 * j) : own[(int64_t)(kn - 1) * pv + 32 * j];
             }
         }
         __syncthreads();
@@ -436,7 +462,7 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
 int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
-    g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0, g_tune_rounds_multi_form = 0, g_tune_rounds_coop_shape = 0;
+    g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0, g_tune_rounds_multi_form = 0, g_tune_rounds_coop_shape = 0, g_tune_rounds_hints = 0;
 
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0 || a.N <= 0) return cudaSuccess;
@@ -545,7 +571,11 @@ cudaError_t launch_round(const RoundArgs& a_in, cudaStream_t s, uint64_t* launch
     return e;
 }
 
-cudaError_t launch_rounds_multi(const RoundArgs& a, int k_last, cudaStream_t s, uint64_t* launches) {
+cudaError_t launch_rounds_multi(const RoundArgs& a_in, int k_last, cudaStream_t s, uint64_t* launches) {
+    RoundArgs a = a_in;
+    // L2 residency hints (measured: +6..+13 % at N = 8, +1..+4 % at N = 16, -1..-4 % at N = 4, where the
+    // delta to cancel is still in L2 anyway); tuning: 1 = off, 2 = on
+    a.reverse = g_tune_rounds_hints ? (g_tune_rounds_hints == 2) : (a.N >= 8);
     if (a.p <= 0 || k_last < a.k) return cudaSuccess;
     // this form is latency-bound (L dependent rounds per thread): spread a small job over all SMs
     // with narrower accesses and smaller blocks rather than leave most of them idle

@@ -487,6 +487,7 @@ def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
         kind = how.split("-")[-1]
         cerar_mod.cerar_set_tuning("rounds_multi_form", {"threads": 1, "scalar": 3}.get(kind, 0))
         cerar_mod.cerar_set_tuning("rounds_coop_shape", {"one": 1, "two": 2}.get(kind, 0))
+        cerar_mod.cerar_set_tuning("rounds_hints", {"one": 2, "two": 1}.get(kind, 0))     # hints forced on / off as well
         how = how.split("-")[0]
         plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
         ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
@@ -510,6 +511,7 @@ def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
         res.append((ws.clone(), plan.counters()))
     cerar_mod.cerar_set_tuning("rounds_multi_form", 0)
     cerar_mod.cerar_set_tuning("rounds_coop_shape", 0)
+    cerar_mod.cerar_set_tuning("rounds_hints", 0)
     for w, cnt in res[1:]:
         assert torch.equal(torch.nan_to_num(w, nan=-1.0), torch.nan_to_num(res[0][0], nan=-1.0))
         assert cnt == res[0][1]
