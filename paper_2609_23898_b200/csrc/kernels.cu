@@ -561,8 +561,9 @@ cudaError_t launch_round(const RoundArgs& a_in, cudaStream_t s, uint64_t* launch
     if (a.p % 4 == 0 && aligned16(a.ws)) {
         const int64_t nv = a.p / 4;
         const unsigned blocks = (unsigned)((nv + threads - 1) / threads);
-        // plain loads and stores, 4 workers in flight per thread: streaming cache hints, 512-thread
-        // blocks and 8 workers per group were all measured and are not faster at d = 1.4e9
+        // plain loads and stores, 4 workers in flight per thread: streaming cache hints (also with an L2
+        // evict_last policy on the message stores: -1..-4 %), 512-thread blocks and 8 workers per group were
+        // all measured and are not faster at d = 1.4e9
         e = launch_pdl(round_kernel<float4, 4>, dim3(blocks), dim3(threads), 0, s, a);
     } else {
         e = launch_pdl(round_kernel<float, 4>, dim3((unsigned)((a.p + threads - 1) / threads)), dim3(threads), 0, s, a);
