@@ -1,6 +1,6 @@
 """Throughput sweep of the CERAR pipeline on one GPU.
 
-  python -m paper_2609_23898_b200.sweep [--quick] [--out FILE]
+  python sweep.py [--quick] [--out FILE]
 
 Points: d per worker in {2^18, 2^20, ..., 2^30} fp32, N in {4, 8, 16}, c in {N, 2N, 4N, 8N},
 epsilon-construction with eps = 1e-3, i.i.d. N(0,1) gradients.  Every point runs in place
@@ -25,6 +25,10 @@ import sys
 
 import numpy as np
 
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
 
 def main():
     ap = argparse.ArgumentParser()
@@ -40,9 +44,9 @@ def main():
     args = ap.parse_args()
 
     import torch
-    from . import cerar, inputs
+    from paper_2609_23898_b200 import cerar, inputs
 
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    root = os.path.dirname(os.path.abspath(__file__))
     peak = 6650.0
     pk = os.path.join(root, "MEASURED_PEAKS.json")
     if os.path.exists(pk):
@@ -127,7 +131,7 @@ def main():
 def fused_table(args, exps, peak, free, stream):
     """Seconds per aggregation of the on-chip variant against the in-HBM pipeline (both out of place)."""
     import torch
-    from . import cerar, inputs
+    from paper_2609_23898_b200 import cerar, inputs
     print("| N | c | d | in-HBM pipeline ms | on-chip ms | speed-up | on-chip DRAM GB/s (8 N d bytes) |")
     print("|---|---|---|---|---|---|---|")
     rows = []
@@ -178,7 +182,7 @@ def fused_table(args, exps, peak, free, stream):
 def ring_table(args, exps, peak, free, stream):
     """The rank-level calls on one GPU: same algorithmic bytes, N launches per step instead of one."""
     import torch
-    from . import cerar, inputs, ring
+    from paper_2609_23898_b200 import cerar, inputs, ring
     print("| N | c | d | pipeline ms | rank-level ms (launches) | rank-level GB/s | frac | fused-rounds ms (launches) | "
           "fused GB/s | frac |")
     print("|---|---|---|---|---|---|---|---|---|---|")
