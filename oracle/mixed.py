@@ -8,8 +8,8 @@ unchanged, except that every transmitted message x_{i,k} is rounded to bfloat16 
 the receiver stores and uses the rounded vector.
 
 A rounding is a decision, and both sides must take it in the same precision (the device's):
-the workers' arithmetic here is IEEE binary32 in the order Algorithm 1 prescribes
-(C <- C + D_k ; send ; C <- received ; C <- C - D_j), on binary32 encoded vectors that are
+the workers' arithmetic here is IEEE binary32 (one rounding per sum or difference of the update
+equations, the message rounded once more by its sender), on binary32 encoded vectors that are
 an INPUT (seeded synthetic ones, or an fp64 encode cast to binary32).  Given the same Delta the
 observations Y are therefore fixed bit for bit.
 """
@@ -36,34 +36,37 @@ def round_bf16(x) -> np.ndarray:
 
 
 def run_rounds_bf16(Delta32):
-    """Algorithm 1 for all N workers with binary32 worker arithmetic and bfloat16 messages.
+    """The L rounds for all N workers with binary32 worker arithmetic and bfloat16 messages:
+    the update equations (Eq. update_eqns) with one rounding added where a vector leaves its sender,
+
+        x_{i,k}     = bf16( delta_{i,k} + sigma_{i,k-1} )   (k <= c),   bf16( sigma_{i,k-1} )   (k > c),
+        sigma_{i,k} = x_{i-1,k}   (k <= N-1),   x_{i-1,k} - delta_{i,k-N+1}   (k >= N),
+
+    every sum and difference rounded to binary32.  The receiver keeps the rounded vector as
+    its observation y_{i,k}; y_{i,L+1} = delta_{i,c} never travels and stays binary32.
 
     Delta32 : list of N arrays (p x c), binary32; column j-1 is delta_{i,j}.
-    Returns Y: list of N arrays (p x (L+1)), binary32: [B_1 .. B_{N-1} | D_1 .. D_c] after
-    round L, where every B and every overwritten D holds a received (rounded) message.
+    Returns Y: list of N arrays (p x (L+1)), binary32, columns y_{i,1} .. y_{i,L+1}.
     """
     N = len(Delta32)
     p, c = Delta32[0].shape
     L = protocol.num_rounds(N, c)
     f32 = np.float32
-    D = [[np.array(Delta32[i][:, j], dtype=f32) for j in range(c)] for i in range(N)]
-    B = [[None] * (N - 1) for _ in range(N)]
-    C = [np.zeros(p, dtype=f32) for _ in range(N)]
+
+    def delta(i, j):
+        return np.asarray(Delta32[i % N][:, j - 1], dtype=f32)
+
+    sigma = [np.zeros(p, dtype=f32) for _ in range(N)]
+    observed = [[] for _ in range(N)]
     for k in range(1, L + 1):
-        x = []
+        x = [round_bf16((delta(i, k) + sigma[i]).astype(f32) if k <= c else sigma[i]) for i in range(N)]
+        nxt = []
         for i in range(N):
-            if k <= c:
-                C[i] = (C[i] + D[i][k - 1]).astype(f32)
-            x.append(round_bf16(C[i]))                     # what leaves worker i
-        for i in range(N):
-            C[i] = x[(i - 1) % N].copy()
-            if k <= N - 1:
-                B[i][k - 1] = C[i].copy()
-            else:
-                j = k - N + 1
-                C[i] = (C[i] - D[i][j - 1]).astype(f32)
-                D[i][j - 1] = x[(i - 1) % N].copy()
-    return [np.stack(B[i] + D[i], axis=1).astype(f32) for i in range(N)]
+            y = x[(i - 1) % N]
+            observed[i].append(y.copy())
+            nxt.append(y.copy() if k <= N - 1 else (y - delta(i, k - N + 1)).astype(f32))
+        sigma = nxt
+    return [np.stack(observed[i] + [delta(i, c).copy()], axis=1).astype(f32) for i in range(N)]
 
 
 def message_bytes(N: int, c: int, p: int) -> int:

@@ -1,4 +1,4 @@
-"""CERAR data path in plain numpy fp64, step by step as the paper states it.
+"""CERAR data path in plain numpy fp64, written from the paper's definitions.
 
 Test infrastructure only (see the package docstring).  Notation follows the
 paper: N workers W_0..W_{N-1} on a clockwise ring, c chunks per gradient,
@@ -38,54 +38,94 @@ def encode(G: np.ndarray, U: np.ndarray) -> np.ndarray:
 
 
 def run_rounds(Delta, *, literal_store: bool = False, trace: bool = False):
-    """Algorithm 1, for all N workers concurrently.
+    """The L ring rounds for all N workers, evaluated from the update equations
+    (Eq. update_eqns):
+
+        x_{i,k}     = delta_{i,k} + sigma_{i,k-1}        for 1 <= k <= c,
+                    = sigma_{i,k-1}                      for c < k <= L,
+        sigma_{i,k} = x_{i-1,k}                          for 1 <= k <= N-1,
+                    = x_{i-1,k} - delta_{i,k-N+1}        for N <= k <= L,
+
+    with sigma_{i,0} = 0 and worker indices modulo N.  Worker i observes
+    y_{i,k} = x_{i-1,k} in round k (k = 1..L) and keeps y_{i,L+1} = delta_{i,c},
+    which no round overwrites; Y_i = [y_{i,1} .. y_{i,L+1}] is the order in which
+    Sec. II lists the stored observations (the N-1 dedicated buffers first, then
+    the c slots that held the encoded vectors).
 
     Delta : list of N arrays (p x c); column j-1 is delta_{i,j}.
-    literal_store : if True the received vector is stored exactly as the
-        algorithm prints it (C <- C - D_j ; D_j <- D_j + C); otherwise the
-        received vector is written to D_j directly.  The two agree up to
-        rounding.
+    literal_store : evaluate the same rounds on the storage slots D, B, C of
+        Sec. II instead (storage_rounds below), where a received vector reaches
+        its slot as "old content plus the new state".  Equal up to rounding.
     trace : also return the messages x[k][i] and the states sigma[k][i].
 
-    Returns (Y, sent, extra): Y[i] is the p x (L+1) observation matrix
-    [B_{i,1} .. B_{i,N-1} | D_{i,1} .. D_{i,c}], sent[i] the number of real
-    values worker i transmitted, extra a dict with the trace (or empty).
+    Returns (Y, sent, extra): Y[i] is the p x (L+1) observation matrix, sent[i]
+    the number of real values worker i transmitted, extra the trace (or empty).
     """
+    if literal_store:
+        return storage_rounds(Delta, trace=trace)
     N = len(Delta)
     p, c = Delta[0].shape
     L = num_rounds(N, c)
-    # buffers of worker i: D[i][j-1], B[i][k-1], C[i]
+
+    def delta(i, j):                       # delta_{i,j}, j = 1..c
+        return np.asarray(Delta[i % N][:, j - 1], dtype=np.float64)
+
+    sigma = [np.zeros(p, dtype=np.float64) for _ in range(N)]     # sigma_{i,0}
+    observed = [[] for _ in range(N)]
+    xs, sigmas = {}, {}
+    for k in range(1, L + 1):
+        x = [delta(i, k) + sigma[i] if k <= c else sigma[i].copy() for i in range(N)]
+        nxt = []
+        for i in range(N):
+            y = x[(i - 1) % N]
+            observed[i].append(y.copy())
+            nxt.append(y.copy() if k <= N - 1 else y - delta(i, k - N + 1))
+        sigma = nxt
+        if trace:
+            xs[k] = [v.copy() for v in x]
+            sigmas[k] = [v.copy() for v in sigma]
+    Y = [np.stack(observed[i] + [delta(i, c).copy()], axis=1) for i in range(N)]
+    sent = [L * p] * N                     # one length-p message per worker and round
+    extra = {"x": xs, "sigma": sigmas} if trace else {}
+    return Y, sent, extra
+
+
+def storage_rounds(Delta, *, trace: bool = False):
+    """The same rounds carried out on the storage of Sec. II: per worker the slots
+    D_1..D_c (initially the encoded vectors), the dedicated buffers B_1..B_{N-1}
+    and the rolling buffer C (initially zero).  What is sent in round k is the
+    content of C after D_k was added to it (k <= c); what arrives replaces C, is
+    copied to B_k while k <= N-1, and from round N on the returning delta in
+    D_{k-N+1} is taken out of C and the slot then receives "its old content plus
+    C", which is the arrived vector in exact arithmetic.  Kept as a check of
+    run_rounds (the two must agree to rounding) and of the storage count."""
+    N = len(Delta)
+    p, c = Delta[0].shape
+    L = num_rounds(N, c)
     D = [[np.array(Delta[i][:, j], dtype=np.float64) for j in range(c)] for i in range(N)]
     B = [[None] * (N - 1) for _ in range(N)]
-    C = [np.zeros(p, dtype=np.float64) for _ in range(N)]   # sigma_{i,0} = 0
+    C = [np.zeros(p, dtype=np.float64) for _ in range(N)]
     sent = [0] * N
     xs, sigmas = {}, {}
     for k in range(1, L + 1):
-        # Step 1: generate, accumulate, transmit
-        x = []
         for i in range(N):
             if k <= c:
                 C[i] = C[i] + D[i][k - 1]
-            x.append(C[i].copy())          # x_{i,k} leaves worker i
-            sent[i] += p
-        # Step 2: receive, store, update
+        outgoing = [C[i].copy() for i in range(N)]
         for i in range(N):
-            C[i] = x[(i - 1) % N].copy()   # receive x_{i-1,k} into C_i
+            sent[i] += p
+            C[i] = outgoing[(i - 1) % N].copy()
             if k <= N - 1:
                 B[i][k - 1] = C[i].copy()
             else:
-                j = k - N + 1
-                C[i] = C[i] - D[i][j - 1]              # cancel delta_{i,j}
-                if literal_store:
-                    D[i][j - 1] = D[i][j - 1] + C[i]   # = x_{i-1,k} in exact arithmetic
-                else:
-                    D[i][j - 1] = x[(i - 1) % N].copy()
+                slot = k - N            # 0-based index of D_{k-N+1}
+                C[i] = C[i] - D[i][slot]
+                D[i][slot] = D[i][slot] + C[i]
         if trace:
-            xs[k] = [v.copy() for v in x]
+            xs[k] = outgoing
             sigmas[k] = [v.copy() for v in C]
     Y = [np.stack(B[i] + D[i], axis=1) for i in range(N)]
-    extra = {"x": xs, "sigma": sigmas} if trace else {}
-    return Y, sent, extra
+    return Y, sent, ({"x": xs, "sigma": sigmas} if trace else {})
 
 
 def decode(Y: np.ndarray, R: np.ndarray, scale: float = 1.0) -> np.ndarray:
