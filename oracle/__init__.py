@@ -8,8 +8,8 @@ benchmark's CPU-baseline leg call into it.
 
 Contents
 --------
-protocol : chunking, encoding, the ring rounds exactly as Algorithm 1 states
-           them, the observation matrix Y_i, decoding, the matrices M_i(U),
+protocol : chunking, encoding, the ring rounds from the update equations (and,
+           as a cross-check, on the storage slots of Algorithm 1), the observation matrix Y_i, decoding, the matrices M_i(U),
            the least-squares objective Phi and the rate counters.
 designs  : the coefficient constructions (multiplicative perturbation
            construction, Vandermonde, epsilon-construction, the

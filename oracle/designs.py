@@ -10,9 +10,11 @@ The condition-number-constrained design is an fp64 iteration (numpy).
 kappa_constrained: every step of an iteration is pinned to the property that defines
 it (the U-step and the R-step are stationary minimisers of the brute-force Phi, the
 projection is the Frobenius-nearest matrix with singular values in the interval), the
-invariants of the whole iteration are tested, and for c = N, where the optimum Phi = 0 is
-known, it is checked to reach it.  PARITY UNPINNED for the end point at c > N only: the
-paper prints no U, R or Phi of this heuristic to compare with.
+loop is pinned to the order of its steps and to the pairs it reports (every history entry
+is Phi of the pair held then; the returned pair is a fixed point up to the stopping rule),
+and for c = N, where the optimum Phi = 0 is known, it is checked to reach it.  PARITY
+UNPINNED for the end point at c > N only: which local solution the heuristic reaches has no
+published counterpart (the paper prints no U, R or Phi for it).
 """
 from __future__ import annotations
 
@@ -289,8 +291,19 @@ def _project(U, a0, b0):
     return out
 
 
+def als_iteration(U, R, a0: float, b0: float, N: int, c: int):
+    """One iteration of the heuristic of Sec. II-D from the pair (U, R): minimise Phi over U with R
+    fixed, project the singular values of every U_k into [a0, b0], minimise Phi over R with the
+    projected U fixed.  Returns (U_ls, U_new, R_new): the unprojected minimiser, and the new pair."""
+    U_ls = _ls_U(R, N, c)
+    U_new = _project(U_ls, a0, b0)
+    R_new = _ls_R(U_new, N, c)
+    return U_ls, U_new, R_new
+
+
 def kappa_constrained(N: int, c: int, kappa_max: float, B, h=None, eps_init: float = 0.1,
-                      iters: int = 200, tol: float = 1e-6, dps: int = DEFAULT_DPS) -> Design:
+                      iters: int = 200, tol: float = 1e-6, dps: int = DEFAULT_DPS,
+                      keep_pairs: bool = False) -> Design:
     """Alternating least-squares heuristic for
         minimise Phi(U, R)  s.t.  kappa_2(M_i(U)) <= C        (Eq. F)
     as Sec. II-D describes it: start from the epsilon-construction; in one
@@ -299,7 +312,10 @@ def kappa_constrained(N: int, c: int, kappa_max: float, B, h=None, eps_init: flo
     with sqrt(N) b0 / a0 <= C.  Choices the paper leaves open (documented as
     readings): eps_init = 0.1, a0 = min_k sigma_min(U_k of the initial design),
     b0 = a0 C / sqrt(N), stop after `iters` iterations or when Phi changes by
-    less than tol (relative), and a last R-step after the last projection."""
+    less than tol (relative), and a last R-step after the last projection
+    (so the pair returned is always (projected U, its least-squares R)).
+    keep_pairs: also keep, in info["pairs"], every pair (U, R) the iteration held
+    and, in info["U_ls"], the unprojected U of every iteration (for the tests)."""
     init = epsilon(N, c, eps_init, B, h, dps)
     U = [u.copy() for u in init.U]
     a0 = min(np.linalg.svd(u, compute_uv=False)[-1] for u in U)
@@ -308,21 +324,28 @@ def kappa_constrained(N: int, c: int, kappa_max: float, B, h=None, eps_init: flo
     R = _ls_R(U, N, c)
     hist = [protocol.phi(U, R)]
     steps = []
+    pairs, unprojected = [(U, R)], []
     done = 0
+    stopped_on_tol = False
     for it in range(iters):
-        U_ls = _ls_U(R, N, c)
+        U_ls, U, R_next = als_iteration(U, R, a0, b0, N, c)
         phi_after_U = protocol.phi(U_ls, R)
-        U = _project(U_ls, a0, b0)
-        R = _ls_R(U, N, c)
+        R = R_next
         cur = protocol.phi(U, R)
         steps.append((hist[-1], phi_after_U, cur))
         hist.append(cur)
+        if keep_pairs:
+            pairs.append((U, R))
+            unprojected.append(U_ls)
         done = it + 1
         if abs(hist[-2] - cur) <= tol * max(cur, 1e-300):
+            stopped_on_tol = True
             break
     des = Design(N, c, U, R, "kappa")
     des.info.update(kappa_max=kappa_max, a0=a0, b0=b0, phi_history=hist, steps=steps,
-                    iters_done=done, eps_init=eps_init)
+                    iters_done=done, eps_init=eps_init, stopped_on_tol=stopped_on_tol)
+    if keep_pairs:
+        des.info.update(pairs=pairs, U_ls=unprojected)
     return des
 
 

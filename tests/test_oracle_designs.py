@@ -463,6 +463,92 @@ def test_als_projection_is_the_nearest_matrix_with_singular_values_in_the_interv
     assert np.allclose(Dz._project(once, a, b)[0], once[0], atol=1e-13)
 
 
+def _max_slope(U, R, which, rng, N, c, trials=6):
+    """Largest |d Phi / dt| over random unit directions in the U_k (which = "U") or the R_i (which = "R")."""
+    L = c + N - 2
+    worst = 0.0
+    for trial in range(trials):
+        idx = trial % N
+        E = rng.standard_normal((c, c) if which == "U" else (L + 1, c))
+        E /= np.linalg.norm(E)
+
+        def perturb(U_, R_, t, idx=idx, E=E):
+            if which == "U":
+                return [u + (t * E if k == idx else 0) for k, u in enumerate(U_)], R_
+            return U_, [r + (t * E if k == idx else 0) for k, r in enumerate(R_)]
+        slope, rise, _ = _phi_slope_and_rise(U, R, perturb)
+        assert rise > 0
+        worst = max(worst, abs(slope))
+    return worst
+
+
+def test_als_loop_holds_the_pairs_it_reports_and_takes_its_steps_in_order():
+    """The iteration of Sec. II-D as a whole (the single steps are pinned above): every entry of the
+    reported history is Phi of the pair held at that point, evaluated here from the M_i matrices; in
+    every iteration the unprojected U minimises Phi for the R of the iteration BEFORE (zero slope in U
+    there, and a clearly non-zero one for the new R, which rules out a swapped order), the new U is its
+    nearest point with singular values in [a0, b0] (Mirsky's bound attained), and the new R minimises
+    Phi for the projected U (zero slope in R; in particular the last R was refitted after the last
+    projection)."""
+    N, c, C = 3, 5, 1e2
+    des = Dz.kappa_constrained(N, c, C, _rng_B(N, c, 3), iters=6, tol=0.0, keep_pairs=True)
+    info = des.info
+    pairs, U_ls, hist = info["pairs"], info["U_ls"], info["phi_history"]
+    a0, b0 = info["a0"], info["b0"]
+    assert len(pairs) == len(hist) == info["iters_done"] + 1 == 7 and len(U_ls) == 6
+    for (U, R), ph in zip(pairs, hist):
+        assert P.phi(U, R) == pytest.approx(ph, rel=1e-12)
+    assert P.phi(des.U, des.R) == pytest.approx(hist[-1], rel=1e-12)
+    for a, b in zip(pairs[-1][0], des.U):
+        assert np.array_equal(a, b)
+    for a, b in zip(pairs[-1][1], des.R):
+        assert np.array_equal(a, b)
+    rng = np.random.default_rng(8)
+    for t in range(1, len(pairs)):
+        (U_prev, R_prev), (U_new, R_new), V = pairs[t - 1], pairs[t], U_ls[t - 1]
+        scale = max(1.0, hist[t - 1])
+        assert _max_slope(V, R_prev, "U", rng, N, c) < 1e-6 * scale          # U-step used the previous R
+        assert _max_slope(V, R_new, "U", rng, N, c) > 1e-4 * scale            # ... and not the new one
+        for k in range(N):                                                    # projection of exactly that V
+            sV = np.linalg.svd(V[k], compute_uv=False)
+            sU = np.linalg.svd(U_new[k], compute_uv=False)
+            assert sU[-1] >= a0 * (1 - 1e-10) and sU[0] <= b0 * (1 + 1e-10)
+            assert np.linalg.norm(V[k] - U_new[k]) == pytest.approx(np.linalg.norm(sV - np.clip(sV, a0, b0)),
+                                                                     rel=1e-8, abs=1e-12)
+        assert _max_slope(U_new, R_new, "R", rng, N, c) < 1e-6 * scale        # R-step after the projection
+        assert P.phi(V, R_prev) == pytest.approx(info["steps"][t - 1][1], rel=1e-12)
+    # the start: the projected epsilon-construction with its least-squares decoder
+    U0, R0 = pairs[0]
+    init = Dz.epsilon(N, c, info["eps_init"], _rng_B(N, c, 3))
+    assert a0 == pytest.approx(min(np.linalg.svd(u, compute_uv=False)[-1] for u in init.U), rel=1e-12)
+    for k in range(N):
+        sI = np.linalg.svd(init.U[k], compute_uv=False)
+        assert np.linalg.norm(init.U[k] - U0[k]) == pytest.approx(np.linalg.norm(sI - np.clip(sI, a0, b0)), rel=1e-8)
+    assert _max_slope(U0, R0, "R", rng, N, c) < 1e-6 * max(1.0, hist[0])
+
+
+def test_als_end_point_is_a_fixed_point_up_to_its_stopping_rule():
+    """When the run stops on its tolerance, one more iteration from the returned pair changes Phi by
+    about the tolerance and moves U and R by a step of the same small order (the heuristic converges
+    sublinearly: measured 3e-5 relative here), so what is returned is the loop's own fixed point and
+    not a pair from somewhere inside an iteration.  A run cut off by the iteration cap says so."""
+    N, c, C, tol = 3, 7, 1e2, 1e-6
+    B = _rng_B(N, c, 5)
+    des = Dz.kappa_constrained(N, c, C, B, iters=4000, tol=tol)
+    assert des.info["stopped_on_tol"] and des.info["iters_done"] < 4000
+    hist = des.info["phi_history"]
+    assert abs(hist[-2] - hist[-1]) <= tol * hist[-1]
+    assert all(abs(a - b) > tol * b for a, b in zip(hist[:-2], hist[1:-1]))       # it did not stop earlier
+    _, U2, R2 = Dz.als_iteration(des.U, des.R, des.info["a0"], des.info["b0"], N, c)
+    ph2 = P.phi(U2, R2)
+    assert abs(ph2 - hist[-1]) <= 2 * tol * hist[-1]
+    for k in range(N):
+        assert np.linalg.norm(U2[k] - des.U[k]) <= 2e-4 * np.linalg.norm(des.U[k])
+        assert np.linalg.norm(R2[k] - des.R[k]) <= 2e-4 * np.linalg.norm(des.R[k])
+    short = Dz.kappa_constrained(N, c, C, B, iters=5, tol=tol)
+    assert not short.info["stopped_on_tol"] and short.info["iters_done"] == 5
+
+
 def test_surrogate_is_well_conditioned():
     des = Dz.custom_orthogonal(4, 8, np.random.default_rng(0))
     for u in des.U:
