@@ -9,8 +9,9 @@ benchmark's CPU-baseline leg call into it.
 Contents
 --------
 protocol : chunking, encoding, the ring rounds from the update equations (and,
-           as a cross-check, on the storage slots of Algorithm 1), the observation matrix Y_i, decoding, the matrices M_i(U),
-           the least-squares objective Phi and the rate counters.
+           as a cross-check, on the storage slots of Algorithm 1), the
+           observation matrix Y_i, decoding, the matrices M_i(U), the
+           least-squares objective Phi and the rate counters.
 designs  : the coefficient constructions (multiplicative perturbation
            construction, Vandermonde, epsilon-construction, the
            condition-number-constrained alternating least squares heuristic).
@@ -25,9 +26,11 @@ Pins (what each function is checked against, see tests/test_oracle_*.py):
       finite-difference identity (Lemma 2) and the printed F_3.
   kappa-constrained design : every step against its defining property (U- and
       R-step are stationary minimisers of the brute-force Phi, the projection is
-      the nearest matrix with singular values in the interval), the invariants of
-      the iteration, and the known optimum Phi = 0 at c = N.  The fitted U, R at
-      c > N have no published counterpart: PARITY UNPINNED for that end point.
+      the nearest matrix with singular values in the interval), the order of the
+      steps in the loop, the reported history, the fixed-point property of what is
+      returned, and the known optimum Phi = 0 at c = N.  Which local solution is
+      reached at c > N has no published counterpart: PARITY UNPINNED for that
+      end point.
   bfloat16 messages : the rounding against worked values, IEEE properties and
       torch's conversion; the rounds against Algorithm 1 where nothing rounds and
       against the error the message precision implies.
