@@ -318,7 +318,13 @@ def kappa_constrained(N: int, c: int, kappa_max: float, B, h=None, eps_init: flo
     and, in info["U_ls"], the unprojected U of every iteration (for the tests)."""
     init = epsilon(N, c, eps_init, B, h, dps)
     U = [u.copy() for u in init.U]
-    a0 = min(np.linalg.svd(u, compute_uv=False)[-1] for u in U)
+    # sigma_min(U_k) = 1 / sigma_max(U_k^{-1}): the initial encoders have condition numbers up to
+    # 1e15 (Corollary 1), where an fp64 SVD of U_k itself gets its smallest singular value wrong in
+    # the fourth digit; the inverse (a window A_l, exact in the high-precision design) has it as its
+    # LARGEST singular value, which fp64 delivers to full accuracy
+    with mp.workdps(dps):
+        inv_norms = [np.linalg.svd(_to_np(mp.inverse(Um)), compute_uv=False)[0] for Um in init.U_mp]
+    a0 = float(min(1.0 / s for s in inv_norms))
     b0 = a0 * kappa_max / np.sqrt(N)
     U = _project(U, a0, b0)
     R = _ls_R(U, N, c)

@@ -430,11 +430,22 @@ int build_kappa(int N, int c, double kappa_max, const double* B, const double* h
     int st = build_epsilon(N, c, eps_init, B, h, P, err);
     if (st != BUILD_OK) return st;
     P.kind = 2; P.param = kappa_max; P.phi_closed = -1.0; P.inv_residual_max = -1.0;
+    // a0 = min_k sigma_min(U_k) of the initial design.  The initial encoders have condition numbers up
+    // to 1e15 (kappa = Theta(eps^-r*), Sec. II-C), where an SVD of U_k itself gets the smallest singular
+    // value wrong in the third digit; U_k^{-1} = A_{N-1-k} is at hand without any inversion (its rows are
+    // rows N-1-k .. N-1-k+c-1 of R_0, Eq. decoderconstruction) and has that value as the reciprocal of its
+    // LARGEST singular value, which the SVD delivers to full accuracy.
     double a0 = std::numeric_limits<double>::infinity();
-    for (int k = 0; k < N; ++k) {
+    const int L = P.L;
+    (void)L;
+    for (int l = 0; l < N; ++l) {
+        MatD A(c, c);
+        for (int t = 0; t < c; ++t)
+            for (int j = 0; j < c; ++j) A(t, j) = P.R[0][(size_t)(l + t) * c + j];
         MatD Uo, V; std::vector<double> s;
-        la::svd_jacobi(mat_of(P.U[k], c, c), Uo, s, V);
-        a0 = std::min(a0, s.back());
+        la::svd_jacobi(A, Uo, s, V);
+        if (!(s.front() > 0)) { a0 = 0; break; }
+        a0 = std::min(a0, 1.0 / s.front());
     }
     if (!(a0 > 0) || !std::isfinite(a0)) { err = "initial design is singular"; return BUILD_SINGULAR; }
     const double b0 = a0 * kappa_max / std::sqrt((double)N);

@@ -549,6 +549,22 @@ def test_als_end_point_is_a_fixed_point_up_to_its_stopping_rule():
     assert not short.info["stopped_on_tol"] and short.info["iters_done"] == 5
 
 
+def test_kappa_constrained_interval_comes_from_the_initial_design():
+    """[a0, b0] of Sec. II-D: a0 = the smallest singular value over the encoders of the initial
+    epsilon-construction, b0 = a0 C / sqrt(N).  Pinned to a 120-digit SVD of those encoders, which at
+    N = 4, c = 24 have condition numbers beyond 1e10, where an fp64 SVD of U_k would already lose digits."""
+    import mpmath as mp
+    N, c, C = 4, 24, 1e4
+    B = _rng_B(N, c, 2)
+    des = Dz.kappa_constrained(N, c, C, B, iters=1)
+    init = Dz.epsilon(N, c, des.info["eps_init"], B)
+    with mp.workdps(120):
+        smallest = min(min(mp.svd_r(Um, compute_uv=False)) for Um in init.U_mp)
+    assert des.info["a0"] == pytest.approx(float(smallest), rel=1e-12)
+    assert des.info["b0"] == pytest.approx(float(smallest) * C / np.sqrt(N), rel=1e-12)
+    assert max(P.kappa2(u) for u in init.U) > 1e10
+
+
 def test_surrogate_is_well_conditioned():
     des = Dz.custom_orthogonal(4, 8, np.random.default_rng(0))
     for u in des.U:

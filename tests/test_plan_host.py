@@ -105,6 +105,35 @@ def test_kappa_plan_matches_oracle_and_invariants():
     assert info["kappa_U_max"] == pytest.approx(max(P.kappa2(u) for u in U), rel=1e-6)
 
 
+def test_kappa_plan_at_the_fourth_configuration_shape():
+    """N = 8, c = 64, C = 1e4 (the fourth configuration).  The initial encoders have kappa ~ 1e15 there,
+    so two fp64 implementations of the first projection differ in the small singular directions by about
+    1e-4 of ||U_k||, and the least-squares decoder amplifies a change of U by kappa_2(M_i) ~ 4e3: the
+    library's and the oracle's U agree to 1e-3, their R only to first order, their Phi to 1e-3.  What
+    must hold exactly is checked on the library's own matrices: the projection interval (smallest singular
+    value of the initial design, taken from its well-conditioned inverse), the constraint, and that R_i
+    is the least-squares decoder of M_i(U) (zero slope of Phi in every R_i)."""
+    N, c, C, iters = 8, 64, 1e4, 3
+    B = inputs.base_matrix(N, c, 0)
+    pl = cerar.Plan.create(N, c, cerar.KAPPA, C, B=B, als_iters=iters, als_tol=1e-300, host_only=True)
+    des = Dz.kappa_constrained(N, c, C, B, iters=iters, tol=0.0)
+    U, R = _plan_mats(pl)
+    info = pl.info()
+    assert info["als_iters_done"] == iters
+    assert info["phi"] == pytest.approx(P.phi(U, R), rel=1e-8)
+    assert info["phi"] == pytest.approx(des.info["phi_history"][-1], rel=1e-3)
+    a0, b0 = des.info["a0"], des.info["b0"]
+    for i in range(N):
+        assert _normwise(U[i], des.U[i]) < 1e-3
+        sv = np.linalg.svd(U[i], compute_uv=False)
+        assert sv[-1] >= a0 * (1 - 1e-6) and sv[0] <= b0 * (1 + 1e-6)      # the library's interval is the oracle's
+        assert sv[0] == pytest.approx(b0, rel=1e-6)                         # and it binds at the top
+        M = P.m_matrix(U, i)
+        assert P.kappa2(M) <= C
+        grad = M.T @ (M @ R[i] - P.target(N, c))
+        assert np.abs(grad).max() < 1e-7 * np.abs(M).max() ** 2
+
+
 def test_custom_plan_roundtrip_and_info():
     rng = np.random.default_rng(0)
     N, c = 3, 5
