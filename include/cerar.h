@@ -348,8 +348,13 @@ cerar_status_t cerar_ring_rounds_fused_local(cerar_plan_t* plan, float* const* w
  * grads / out: device buffers as in cerar_allreduce_sim; they must not alias each
  * other or the workspace (the in-place forms are not available here).  The
  * device the plan was created on must be current.
- * First call on a device: looks up the array's device address (once per device);
- * make that first call before any stream capture begins.
+ * First call on a device: after checking that the plan has device copies and that
+ * its device is current, looks up the array's device address (once per device).
+ * The CUDA runtime may load this part of the library's device image only then, so
+ * that first call is where the 64 MiB are actually reserved on the device: it can
+ * fail (CERAR_ERR_NOMEM / CERAR_ERR_CUDA) if the device has no room left.  A caller
+ * whose framework is about to claim all free memory makes one call before that
+ * happens.  Make the first call before any stream capture begins.
  * All calls share the one array, which keeps whatever the previous call left in
  * it.  Nothing needs clearing between calls (every slot is written before it is
  * read), but two calls whose kernels overlap on the GPU (different streams, or

@@ -140,6 +140,8 @@ const char* cerar_last_error(void) { return g_err.c_str(); }
 
 // for the library's other translation units
 void cerar_internal_set_error(const char* msg) { g_err = msg ? msg : ""; }
+// device ordinal the plan's fp32 copies live on, or -1 for a plan without device copies
+int cerar_internal_plan_device(const cerar_plan_t* P) { return (P && P->on_device) ? P->device : -1; }
 
 cerar_status_t cerar_plan_create_ex(int N, int c, cerar_construction_t kind, double param,
                                     const cerar_options_t* opt, cerar_plan_t** out) {

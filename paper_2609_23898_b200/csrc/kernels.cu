@@ -377,7 +377,7 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
     VT* nxt = reinterpret_cast<VT*>(a.ws) + (int64_t)dst * wstride + v0;
     grid_dependency_wait();
     int k = a.k;
-    const bool hints = a.reverse != 0;                          // set by the launcher
+    const bool hints = a.hints != 0;                            // set by the launcher
     const uint64_t pol = policy_keep();
     // operands of rounds k .. k+DIST-1 (index t = rounds ahead); absent terms are zero
     VT y[PV], da[DIST][PV], dc[DIST][PV];
@@ -576,7 +576,7 @@ cudaError_t launch_rounds_multi(const RoundArgs& a_in, int k_last, cudaStream_t 
     RoundArgs a = a_in;
     // L2 residency hints (measured: +6..+13 % at N = 8, +1..+4 % at N = 16, -1..-4 % at N = 4, where the
     // delta to cancel is still in L2 anyway); tuning: 1 = off, 2 = on
-    a.reverse = g_tune_rounds_hints ? (g_tune_rounds_hints == 2) : (a.N >= 8);
+    a.hints = g_tune_rounds_hints ? (g_tune_rounds_hints == 2) : (a.N >= 8);
     if (a.p <= 0 || k_last < a.k) return cudaSuccess;
     // this form is latency-bound (L dependent rounds per thread): spread a small job over all SMs
     // with narrower accesses and smaller blocks rather than leave most of them idle

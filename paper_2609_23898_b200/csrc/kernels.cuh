@@ -33,7 +33,8 @@ struct RoundArgs {
     float* ws;              // workspace, worker i at ws + i*(c+N)*p
     int64_t p;
     int N, c, k;            // round k in 1..L
-    int reverse;            // 1: blocks walk the positions downwards (set by the launcher)
+    int reverse;            // round_kernel: 1 = blocks walk the positions downwards (set by the launcher)
+    int hints;              // rounds_coop_kernel: 1 = L2 residency hints on the delta rows (set by the launcher)
 };
 
 // One worker's ring round in the one-worker-per-GPU layout ((c+N+1) x p per worker).

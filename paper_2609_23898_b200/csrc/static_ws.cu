@@ -5,6 +5,7 @@
 
 #include <cstdio>
 #include <mutex>
+#include <string>
 
 #include "../../include/cerar.h"
 
@@ -18,6 +19,7 @@
 static __device__ __align__(256) float g_cerar_static_ws[CERAR_STATIC_WS_FLOATS];
 
 extern "C" void cerar_internal_set_error(const char* msg);    // api.cu: text behind cerar_last_error()
+extern "C" int cerar_internal_plan_device(const cerar_plan_t* plan);   // api.cu: -1 without device copies
 
 namespace {
 constexpr int kMaxDevices = 64;
@@ -42,22 +44,39 @@ extern "C" cerar_status_t cerar_allreduce_sim_static(cerar_plan_t* plan, const f
         cerar_internal_set_error(msg);
         return CERAR_ERR_TOO_LARGE;
     }
+    // The plan must have device copies and its device must be the current one BEFORE the array is looked
+    // up: the lookup below is what makes the CUDA runtime load this file's device image (and with it
+    // reserve the array) on the current device, and that must not happen on a device the call cannot use.
+    const int plan_dev = cerar_internal_plan_device(plan);
+    if (plan_dev < 0) {
+        cerar_internal_set_error("plan has no device copies (no CUDA device, or host_only)");
+        return CERAR_ERR_CUDA;
+    }
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
         cerar_internal_set_error(e != cudaSuccess ? cudaGetErrorString(e) : "device ordinal out of range");
         return CERAR_ERR_CUDA;
     }
+    if (dev != plan_dev) {
+        cerar_internal_set_error("the device the plan was created on must be current");
+        return CERAR_ERR_CUDA;
+    }
     float* ws = nullptr;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
         if (!g_device_ptr[dev]) {
-            // one-time set-up for this device (it is the current one)
+            // one-time set-up for this device (it is the current one).  With lazy module loading this
+            // is also the moment the 64 MiB are reserved on the device: it can fail for lack of memory
             void* p = nullptr;
             e = cudaGetSymbolAddress(&p, g_cerar_static_ws);
             if (e != cudaSuccess || !p) {
-                cerar_internal_set_error(e != cudaSuccess ? cudaGetErrorString(e) : "symbol address is NULL");
-                return CERAR_ERR_CUDA;
+                cerar_internal_set_error(e != cudaSuccess
+                                             ? (std::string("built-in workspace could not be set up on this device: ") +
+                                                cudaGetErrorString(e)).c_str()
+                                             : "symbol address is NULL");
+                cudaGetLastError();
+                return e == cudaErrorMemoryAllocation ? CERAR_ERR_NOMEM : CERAR_ERR_CUDA;
             }
             g_device_ptr[dev] = static_cast<float*>(p);
         }

@@ -132,7 +132,8 @@ def sampled_parity(cfg, des, plan, grads, ws, out, scale, n_tiles=6, tile=512):
     Y_ora = np.stack([ora["Y"][i].T for i in range(N)])
     out_dev = out.view(N, c, p)[:, :, idx_t].reshape(N, -1).cpu().numpy()
     kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
-    return {"positions": int(idx.size), "rel_l2_Y": P.rel_l2(Y_dev, Y_ora),
+    yard = rounding_yardsticks(des.U, des.R, g_sub, scale, Y_dev=Y_dev, out_dev=out_dev)
+    return {"positions": int(idx.size), "rel_l2_Y": P.rel_l2(Y_dev, Y_ora), "yardsticks": yard,
             "rel_l2_out_max": max(P.rel_l2(out_dev[i], ora["out"][i]) for i in range(N)),
             "kappa_M": kap, "kappa_times_2^-24": kap * 2.0 ** -24,
             "rel_l2_oracle_vs_exact_mean": max(P.rel_l2(ora["out"][i], P.exact_sum(list(g_sub)) * scale)

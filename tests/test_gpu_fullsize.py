@@ -63,14 +63,48 @@ def test_config3_full_size_sampled(how):
     assert res["positions"] >= 2048
     assert res["rel_l2_Y"] < 2e-6                      # encode + all rounds, no cancellation
     assert res["rel_l2_out_max"] < 4 * res["kappa_M"] * U32
+    # decode and the whole path within the a-priori fp32 rounding bounds (finite whatever kappa is)
+    assert res["yardsticks"]["decode_ratio"] <= 1.0 and res["yardsticks"]["end_to_end_ratio"] <= 1.0
     assert res["rel_l2_oracle_vs_exact_mean"] < 0.05   # the design itself approximates the mean to O(eps)
 
 
 @pytest.mark.parametrize("how", ["per_round", "one_call"])
 def test_config4_full_size_sampled(how):
-    """N=8, c=64, kappa-constrained design (C = 1e4), d=2^28, Student-t gradients.  The
-    design is the oracle's own (fewer ALS sweeps than the default to keep the test short;
-    any projected iterate satisfies the constraint) handed over as a custom plan."""
+    """N=8, c=64, kappa-constrained design (C = 1e4), d=2^28, Student-t gradients, with the plan the
+    benchmark times: the library's own design with its default 200 iterations.  At this shape the
+    library's and the oracle's iterates agree only to about 1e-3 (the first projection acts on
+    encoders with kappa ~ 1e15; see tests/test_plan_host.py), so the coefficient matrices are taken
+    from the plan here: they are inputs of the data path under test, like the gradients, and the
+    design itself is checked separately against the oracle's.  Its invariants are checked on the way."""
+    from types import SimpleNamespace
+    from paper_2609_23898_b200 import cerar, inputs
+    cfg = inputs.CONFIGS["cfg4"]
+    N, c = cfg["N"], cfg["c"]
+    B = inputs.base_matrix(N, c, 0)
+    plan_holder = {}
+
+    def factory():
+        plan_holder["plan"] = cerar.Plan.create(N, c, cerar.KAPPA, cfg["param"], B=B)
+        return plan_holder["plan"]
+    plan = factory()
+    des = SimpleNamespace(U=[plan.get_U(i) for i in range(N)], R=[plan.get_R(i) for i in range(N)])
+    kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+    assert kap <= cfg["param"]
+    assert plan.info()["kappa_M_max"] == pytest.approx(kap, rel=1e-6)
+    for i in range(N):                                   # R_i is the least-squares decoder of M_i(U)
+        M = P.m_matrix(des.U, i)
+        assert np.abs(M.T @ (M @ des.R[i] - P.target(N, c))).max() < 1e-7 * np.abs(M).max() ** 2
+    res = _run("cfg4", des, lambda: plan, 30, how)
+    print("\n[cfg4 full size, the library's own plan]", how, res)
+    assert res["rel_l2_Y"] < 2e-6
+    assert res["rel_l2_out_max"] < max(1e-4, 4 * kap * U32)
+    assert res["yardsticks"]["decode_ratio"] <= 1.0 and res["yardsticks"]["end_to_end_ratio"] <= 1.0
+
+
+def test_config4_full_size_sampled_with_the_oracle_design():
+    """The same shape with the oracle's own design (fewer sweeps, to keep the test short; any
+    projected iterate satisfies the constraint) handed over as a custom plan: no oracle input from
+    the library at all."""
     from paper_2609_23898_b200 import cerar, inputs
     cfg = inputs.CONFIGS["cfg4"]
     N, c = cfg["N"], cfg["c"]
@@ -78,10 +112,11 @@ def test_config4_full_size_sampled(how):
     des = Dz.kappa_constrained(N, c, cfg["param"], B, iters=20)
     kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
     assert kap <= cfg["param"]
-    res = _run("cfg4", des, lambda: cerar.Plan.create_custom(N, c, des.U, des.R), 30, how)
-    print("\n[cfg4 full size]", how, res)
+    res = _run("cfg4", des, lambda: cerar.Plan.create_custom(N, c, des.U, des.R), 30, "per_round")
+    print("\n[cfg4 full size, oracle design]", res)
     assert res["rel_l2_Y"] < 2e-6
     assert res["rel_l2_out_max"] < max(1e-4, 4 * kap * U32)
+    assert res["yardsticks"]["decode_ratio"] <= 1.0 and res["yardsticks"]["end_to_end_ratio"] <= 1.0
 
 
 def test_config3_full_size_one_worker_per_rank_fused_rounds():
@@ -130,5 +165,8 @@ def test_config3_full_size_one_worker_per_rank_fused_rounds():
                                                             "rel_l2_out_max": err_out, "kappa_M": kap})
     assert err_y < 2e-6
     assert err_out < 4 * kap * U32
+    from tests._harness import rounding_yardsticks
+    yard = rounding_yardsticks(des.U, des.R, g_sub, 1.0 / N, Y_dev=Y_dev, out_dev=out_dev)
+    assert yard["decode_ratio"] <= 1.0 and yard["end_to_end_ratio"] <= 1.0, yard
     del r, grads
     torch.cuda.empty_cache()

@@ -19,7 +19,8 @@ import pytest
 
 from oracle import designs as Dz
 from oracle import protocol as P
-from tests._harness import rel_l2, run_library, run_oracle, torch_stream
+from tests._harness import (assert_within_rounding_bounds, rel_l2, rounding_yardsticks, run_library, run_oracle,
+                            torch_stream)
 
 pytestmark = pytest.mark.gpu
 
@@ -219,6 +220,15 @@ def test_paper_designs_stagewise_and_reported_output(cerar_mod, N, c, kind, para
     res_c = run_library(plan_c, g, 1.0)
     assert rel_l2(res_c["Delta"], ora["Delta_rows"]) < STAGE_TOL
     assert rel_l2(res_c["Y"], ora["Y_rows"]) < STAGE_TOL
+    # ... and every stage of it, the decode with coefficients of magnitude up to 1e11 included, stays
+    # within the a-priori fp32 rounding bound of what it computes from the binary32 copies of these
+    # matrices (a bound that does not grow with kappa; a wrong element is ~1e5 times beyond it)
+    y = rounding_yardsticks(des.U, des.R, g, 1.0, Delta_dev=res_c["Delta"], Y_dev=res_c["Y"], out_dev=res_c["out"])
+    print(f"    residual / a-priori bound: {y}")
+    assert_within_rounding_bounds(y, K=1.0)
+    # the library-built plan holds the same binary32 coefficients up to an ulp in a few entries
+    y_lib = rounding_yardsticks(des.U, des.R, g, 1.0, Y_dev=res["Y"], out_dev=res["out"])
+    assert y_lib["decode_ratio"] <= 1.0 and y_lib["end_to_end_ratio"] <= 1.0, y_lib
 
 
 def test_state_machine_and_counters(cerar_mod):
@@ -350,6 +360,15 @@ def test_full_size_config2(cerar_mod):
     worst = max(rel_l2(res["out"][i], ora["out"][i]) for i in range(N))
     print(f"\n[cfg2] kappa_M={kap:.3e} kappa*2^-24={kap * U32:.3e} rel_l2(gpu, oracle)={worst:.3e}")
     assert worst < 4 * kap * U32
+    # the finite yardstick: a-priori rounding bounds per stage on a slice of positions (the bound needs
+    # a few dense fp64 products per worker)
+    sl = slice(0, 65536)
+    p = d // c
+    pick = lambda a: a.reshape(N, -1, p)[:, :, sl]
+    y = rounding_yardsticks(des.U, des.R, pick(g).reshape(N, -1), 1.0 / N, Delta_dev=pick(res["Delta"]),
+                            Y_dev=pick(res["Y"]), out_dev=pick(res["out"]).reshape(N, -1))
+    print(f"    residual / a-priori bound: {y}")
+    assert_within_rounding_bounds(y, K=1.0)
     res1 = run_library(plan, g, 1.0 / N, stepwise=False)
     np.testing.assert_array_equal(res1["out"], res["out"])       # same kernels, same order: bit-identical
 
