@@ -42,12 +42,13 @@ def _metric_name():
 
 METRIC = _metric_name()
 UNIT = "GB/s"
-# DRAM bytes of a steady ring-round launch measured by ncu on a smaller case of the same
-# kernel (N=8, c=32, p=4 Mi; summary under profiles/): 12.0 B read + 2.9 B written
-# per (worker x position) against 16 B algorithmic (part of the writes is still in L2 when
-# the launch ends).  Traffic grows in proportion to the positions, so it is scaled by the
-# algorithmic bytes of the timed launch.
-NCU_ROUND_TRAFFIC_OVER_ALGORITHMIC = 14.88 / 16.0
+# DRAM bytes per launch over algorithmic bytes per launch, from ncu captures of smaller cases of the
+# same kernels (N=8, c=32, p=1 Mi; summaries under profiles/): means over consecutive launches with
+# the caches left alone between them (--cache-control none), so that what one launch leaves dirty in
+# L2 is counted when the next launch evicts it.  DRAM traffic grows in proportion to the positions, so
+# the ratio is applied to the algorithmic bytes of the timed launch.
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"round_kernel": 1.0, "encode": 1.0, "decode": 1.0}
+NCU_TRAFFIC_SOURCE = "algorithmic bytes (no steady-state ncu capture folded in yet)"
 
 
 def algorithmic_bytes(N, c, p):
@@ -144,16 +145,22 @@ def oracle_step(des, g_sub, scale):
     return P.allreduce([x for x in g_sub], des.U, des.R, scale)
 
 
-def cpu_baseline(cfg, des, p_sample, seed=0, one_thread=False):
-    """Times the oracle, as it stands, on the first p_sample positions of the
-    workload (all N workers, all c chunks)."""
+def cpu_baseline(cfg, des, p_sample, seed=0, one_thread=False, g=None, keep=None):
+    """Times the oracle, as it stands, on the first p_sample positions of the workload (all N
+    workers, all c chunks).  g: those positions of the device's gradients, (N, c*p_sample) fp32, read
+    back from the GPU (default: the same recipe drawn with numpy).  keep: a dict that receives the
+    oracle's result (for the parity block)."""
     from paper_2609_23898_b200 import inputs
     N, c = cfg["N"], cfg["c"]
     kw = {"std": cfg["std"]} if "std" in cfg else {}
-    g = inputs.gradients_numpy(N, c * p_sample, cfg["workload"], seed=seed, **kw).astype(np.float64)
+    if g is None:
+        g = inputs.gradients_numpy(N, c * p_sample, cfg["workload"], seed=seed, **kw)
+    g = g.astype(np.float64)
     t0 = time.perf_counter()
-    oracle_step(des, g, 1.0 / N)
+    res_o = oracle_step(des, g, 1.0 / N)
     dt = time.perf_counter() - t0
+    if keep is not None:
+        keep.update(res=res_o, g=g)
     ab = algorithmic_bytes(N, c, p_sample)["total"]
     try:
         from threadpoolctl import threadpool_info
@@ -168,7 +175,7 @@ def cpu_baseline(cfg, des, p_sample, seed=0, one_thread=False):
         try:
             from threadpoolctl import threadpool_limits
             p1 = max(1, p_sample // 8)
-            g1 = inputs.gradients_numpy(N, c * p1, cfg["workload"], seed=seed, **kw).astype(np.float64)
+            g1 = np.ascontiguousarray(g.reshape(N, c, p_sample)[:, :, :p1]).reshape(N, -1)
             with threadpool_limits(limits=1):
                 t0 = time.perf_counter()
                 oracle_step(des, g1, 1.0 / N)
@@ -178,6 +185,53 @@ def cpu_baseline(cfg, des, p_sample, seed=0, one_thread=False):
         except Exception:
             pass
     return res
+
+
+def parity_block(des, kept, par_dev, p_sample, p_par, scale):
+    """GPU against the oracle on the first p_par positions, part of the cpu_baseline leg (the
+    oracle's results are those of its timed run; one more oracle pass with the coefficients rounded to
+    binary32, as the device holds them, separates coefficient rounding from kernel error).  Next to
+    kappa 2^-24 the block carries the a-priori fp32 rounding bound u (c+L) || |G^(i)| |M_i| |R_i| ||_F
+    / || g_hat_i || (worst worker) and, for the decode alone, residual over bound
+    || out - s Y_dev Rf || / (u (L+1) s || |Y_dev| |Rf| ||_F), which does not grow with kappa."""
+    from oracle import protocol as P
+    N, c = des.N, des.c
+    L = c + N - 2
+    u = 2.0 ** -24
+    res, g = kept["res"], kept["g"]
+    pick = lambda v, rows: np.ascontiguousarray(v.reshape(rows, p_sample)[:, :p_par])
+    Y_ora = np.stack([res["Y"][i][:p_par].T for i in range(N)])                       # (N, L+1, p_par)
+    out_ora = [pick(res["out"][i], c).reshape(-1) for i in range(N)]
+    g_par = [pick(g[i], c).reshape(-1) for i in range(N)]
+    Uf = [np.asarray(m, np.float32).astype(np.float64) for m in des.U]
+    Rf = [np.asarray(m, np.float32).astype(np.float64) for m in des.R]
+    res_f = P.allreduce(g_par, Uf, Rf, scale)
+    G = [P.chunk_matrix(x, c) for x in g_par]
+    kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+    rel_out = rel_out_f = bound_rel = e2e_ratio = dec_ratio = 0.0
+    for i in range(N):
+        od = par_dev["out"][i].astype(np.float64)
+        ref = np.linalg.norm(res_f["out"][i])
+        mag = np.abs(P.stacked_gradients(G, i)) @ np.abs(P.m_matrix(Uf, i)) @ np.abs(Rf[i])
+        bound = u * (c + L) * scale * np.linalg.norm(mag)
+        err_f = np.linalg.norm(od - res_f["out"][i])
+        Yd = par_dev["Y"][i].astype(np.float64).T
+        dec_bound = u * (L + 1) * scale * np.linalg.norm(np.abs(Yd) @ np.abs(Rf[i]))
+        rel_out = max(rel_out, P.rel_l2(od, out_ora[i]))
+        rel_out_f = max(rel_out_f, err_f / ref)
+        bound_rel = max(bound_rel, bound / ref)
+        e2e_ratio = max(e2e_ratio, err_f / bound)
+        dec_ratio = max(dec_ratio, np.linalg.norm(od - P.unchunk(scale * (Yd @ Rf[i]))) / dec_bound)
+    exact = P.exact_sum(g_par) * scale
+    return {"sampled_positions": int(p_par), "which": "the first positions of every chunk, all workers",
+            "rel_l2_Y": P.rel_l2(par_dev["Y"], Y_ora), "rel_l2_out": rel_out,
+            "rel_l2_out_vs_fp32_rounded_coefficients": rel_out_f,
+            "kappa_M": kap, "kappa_times_2^-24": kap * u, "apriori_bound_rel": bound_rel,
+            "end_to_end_residual_over_bound": e2e_ratio, "decode_residual_over_bound": dec_ratio,
+            "rel_l2_oracle_vs_exact_mean": max(P.rel_l2(out_ora[i], exact) for i in range(N)),
+            "note": "computed outside the timed regions from the last timed aggregation; stages without "
+                    "cancellation (Y) agree to fp32 roundoff, the decoded output of an ill-conditioned design "
+                    "carries roundoff amplified by about kappa and is held to its a-priori bound instead"}
 
 
 def run_reference(args, cfg):
@@ -231,6 +285,222 @@ def workload_name(key, cfg):
             f"{cfg['workload']} gradients")
 
 
+THERMAL = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
+
+
+def time_steps(plan, grads, g_stride, ws, out, o_stride, d, scale, K, W, stream, gpu_index=None, sync=None):
+    """W warm-ups, then the timed region: K steps, each the C-ABI sequence cerar_encode,
+    cerar_ring_round(1..L), cerar_decode, with a CUDA event after every phase (encode | the L round
+    launches | decode; an event after every launch would keep consecutive launches apart) and, if
+    gpu_index is given, the clocks sampled alongside.  Returns the per-phase means, this rank's
+    step times and the total device time of the K steps (ms)."""
+    import torch
+    L = plan.L
+    sync = sync or torch.cuda.synchronize
+    sampler = ClockSampler(gpu_index) if gpu_index is not None else None
+    for _ in range(W):                                  # the timed sequence itself, without the events
+        plan.encode(grads, g_stride, ws, d, stream)
+        for k in range(1, L + 1):
+            plan.ring_round(ws, d, k, stream)
+        plan.decode(ws, out, o_stride, d, scale, stream)
+    torch.cuda.synchronize()
+    plan.device_status(stream)
+    if sampler:
+        sampler.wait_first_sample()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    sync()
+    launches0 = plan.launch_count()
+    for s in range(K):
+        e = ev[s]
+        e[0].record()
+        plan.encode(grads, g_stride, ws, d, stream)
+        e[1].record()
+        for k in range(1, L + 1):
+            plan.ring_round(ws, d, k, stream)
+        e[2].record()
+        plan.decode(ws, out, o_stride, d, scale, stream)
+        e[3].record()
+    sync()
+    launches = plan.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    plan.device_status(stream)
+    return {"total_ms": ev[0][0].elapsed_time(ev[K - 1][3]),
+            "enc_ms": float(np.mean([e[0].elapsed_time(e[1]) for e in ev])),
+            "rounds_ms": float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
+            "dec_ms": float(np.mean([e[2].elapsed_time(e[3]) for e in ev])),
+            "step_ms": [e[0].elapsed_time(e[3]) for e in ev],
+            "launches": int(launches), "clocks": clocks}
+
+
+def time_one_call(plan, grads, g_stride, ws, out, o_stride, d, scale, K, stream, sync=None):
+    """The same K aggregations through cerar_allreduce_sim with one event pair around all of them."""
+    import torch
+    sync = sync or torch.cuda.synchronize
+    for _ in range(3):
+        plan.allreduce_sim(grads, g_stride, out, o_stride, ws, d, scale, stream)
+    sync()
+    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0 = plan.launch_count()
+    o0.record()
+    for _ in range(K):
+        plan.allreduce_sim(grads, g_stride, out, o_stride, ws, d, scale, stream)
+    o1.record()
+    sync()
+    plan.device_status(stream)
+    return o0.elapsed_time(o1), (plan.launch_count() - n0) // K
+
+
+SWEEP_CORNERS = [(16, 128, 1 << 24), (16, 128, 1 << 28), (4, 16, 1 << 26)]
+
+
+def other_configs(headline_key, peak, gpu_index, stream, steps=20, warmup=3, only=()):
+    """The remaining configurations at full size and a few corners of the sweep, each timed like the
+    headline (cerar_encode, L x cerar_ring_round, cerar_decode with an event after every phase, then
+    the one-call form), after the headline's buffers were freed.  The configurations run out of place,
+    the sweep corners in place (as the sweep does: gradients in the D rows, result over them)."""
+    import torch
+    from paper_2609_23898_b200 import cerar, inputs
+    kinds = {"vandermonde": cerar.VANDERMONDE, "epsilon": cerar.EPSILON, "kappa": cerar.KAPPA}
+    jobs = [(k, dict(inputs.CONFIGS[k]), False) for k in ("cfg4", "cfg2", "cfg1", "cfg3") if k != headline_key]
+    jobs += [(f"sweep_N{N}_c{c}_d2^{d.bit_length() - 1}",
+              dict(N=N, c=c, kind="epsilon", param=1e-3, d=d, workload="normal", std=1.0), True) for N, c, d in SWEEP_CORNERS]
+    out_all = {}
+    dev = torch.device("cuda", torch.cuda.current_device())
+    for key, cfg, inplace in jobs:
+        if only and key not in only:
+            continue
+        N, c, d = cfg["N"], cfg["c"], cfg["d"]
+        p, L = d // c, c + N - 2
+        need = 4 * N * ((c + N) * p + (0 if inplace else 2 * d))
+        if need > 0.9 * torch.cuda.mem_get_info()[0]:
+            out_all[key] = {"skipped": f"needs {need / 1e9:.1f} GB of device memory"}
+            continue
+        try:
+            B = inputs.base_matrix(N, c, 0)
+            plan = cerar.Plan.create(N, c, kinds[cfg["kind"]], cfg["param"], B=B)
+            ws = torch.empty(plan.workspace_bytes(d) // 4, dtype=torch.float32, device=dev)
+            kw = {"std": cfg["std"]} if "std" in cfg else {}
+            if inplace:
+                wv = ws.view(N, c + N, p)
+                rows = [wv[i, N:, :].reshape(-1) for i in range(N)]             # views of the D rows
+                inputs.fill_gradients_torch(rows, cfg["workload"], seed=0, **kw)
+                g_ptr = o_ptr = ws.data_ptr() + 4 * N * p
+                g_stride = o_stride = (c + N) * p
+                grads = outb = None
+            else:
+                grads = torch.empty(N * d, dtype=torch.float32, device=dev)
+                inputs.fill_gradients_torch([grads[i * d:(i + 1) * d] for i in range(N)], cfg["workload"], seed=0, **kw)
+                outb = torch.empty(N * d, dtype=torch.float32, device=dev)
+                g_ptr, o_ptr, g_stride, o_stride = grads.data_ptr(), outb.data_ptr(), d, d
+            ab = algorithmic_bytes(N, c, p)
+            m = time_steps(plan, g_ptr, g_stride, ws, o_ptr, o_stride, d, 1.0 / N, steps, warmup, stream, gpu_index)
+            ms = m["total_ms"] / steps
+            one_ms, n_one = time_one_call(plan, g_ptr, g_stride, ws, o_ptr, o_stride, d, 1.0 / N, steps, stream)
+            one_ms /= steps
+            gbps = lambda b, t: b / t / 1e6
+            out_all[key] = {
+                "workload": workload_name(key, cfg), "buffers": "in place" if inplace else "out of place",
+                "steps": steps, "warmup": warmup, "ms_per_step": ms, "value": gbps(ab["total"], ms), "unit": UNIT,
+                "frac": gbps(ab["total"], ms) / peak, "gpu_launches": m["launches"],
+                "per_kernel_GBps": {"encode": gbps(ab["encode"], m["enc_ms"]), "round_kernel": gbps(ab["rounds"], m["rounds_ms"]),
+                                    "decode": gbps(ab["decode"], m["dec_ms"])},
+                "per_kernel_frac": {"encode": gbps(ab["encode"], m["enc_ms"]) / peak,
+                                    "round_kernel": gbps(ab["rounds"], m["rounds_ms"]) / peak,
+                                    "decode": gbps(ab["decode"], m["dec_ms"]) / peak},
+                "one_call": {"ms_per_step": one_ms, "value": gbps(ab["total"], one_ms), "frac_effective": gbps(ab["total"], one_ms) / peak,
+                             "launches_per_step": int(n_one)},
+                "l2": "inputs larger than L2" if 4 * N * (c + N) * p > 2.6e8 else "state fits in L2: launch-bound, not an HBM figure",
+                "clocks": m["clocks"]}
+            del plan, ws, grads, outb
+        except Exception as exc:                         # one failing point must not cost the headline
+            out_all[key] = {"error": f"{type(exc).__name__}: {exc}"}
+        torch.cuda.empty_cache()
+    return out_all
+
+
+def ring_block(world, rank, dev, *, plan=None, d=None, reps=3, timer=None):
+    """N > 1 only: one aggregation family with ONE WORKER PER RANK (N = world, c = 4 world,
+    d = 2^28 per worker, epsilon-construction), next to torch.distributed's all-reduce of the same
+    gradient: (a) ring.SendRecvRing, messages moved by isend / irecv of the process group; (b)
+    ring.DistributedRing, messages stored straight into the neighbour's workspace (peer-mapped symmetric
+    memory), one device-side barrier per round; (c) the same with all rounds in one kernel per rank that
+    orders itself against its neighbours tile by tile.  The three must give the same bits (the message
+    arithmetic is the same kernel code); their parity with the oracle is the business of the tests.
+    plan / d / timer are for the CPU test, which drives this function with stand-ins on gloo ranks."""
+    import torch
+    import torch.distributed as dist
+    from paper_2609_23898_b200 import cerar, inputs, ring
+    N = world
+    on_gpu = dev.type == "cuda"
+    if plan is None:
+        c = 4 * N
+        plan = cerar.Plan.create(N, c, cerar.EPSILON, 1e-2, B=inputs.base_matrix(N, c, 0))
+    c, L = plan.c, plan.L
+    d = d if d is not None else (1 << 28) // c * c
+    p = d // c
+    stream = torch.cuda.current_stream().cuda_stream if on_gpu else 0
+    grad = torch.empty(d, dtype=torch.float32, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7000 + rank)
+    grad.normal_(0.0, 1.0, generator=gen)
+
+    def default_timer(fn):
+        """ms per call, max over ranks: barrier, synchronize, `reps` calls between two CUDA events."""
+        fn()                                                     # warm-up
+        dist.barrier()
+        if on_gpu:
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            dist.barrier()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+        else:
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                fn()
+            dist.barrier()
+            ms = (time.perf_counter() - t0) * 1e3 / reps
+        return max_over_ranks(ms, world, dev if on_gpu else None)
+    timer = timer or default_timer
+
+    block = {"workers": N, "c": c, "L": L, "d": d, "design": "epsilon(0.01)", "reps": reps,
+             "bytes_over_the_link_per_rank": 4 * p * L, "all_reduce_bytes_per_rank_ring": int(2 * (N - 1) / N * 4 * d),
+             "status": "unmeasured on hardware until a multi-GPU run reports it" if not on_gpu else "measured"}
+    ref = grad.clone()
+    block["all_reduce_ms"] = timer(lambda: dist.all_reduce(ref.copy_(grad)))
+    mean = ref.copy_(grad)
+    dist.all_reduce(mean)
+    mean = mean / N
+    outs = {}
+    forms = [("sendrecv", lambda: ring.SendRecvRing(plan, d, device=dev), {}),
+             ("peer_round_by_round", lambda: ring.DistributedRing(plan, d, device=dev), {"fused": False}),
+             ("peer_fused_rounds", None, {"fused": True})]
+    drv = None
+    for name, make, kw in forms:
+        try:
+            drv = make() if make is not None else drv
+            out = torch.empty(d, dtype=torch.float32, device=dev)
+            ms = timer(lambda: drv.allreduce(grad, out, 1.0 / N, stream, **kw))
+            if on_gpu:
+                torch.cuda.synchronize()
+                plan.device_status(stream)
+            outs[name] = out
+            block[name] = {"ms_per_aggregation": ms, "ratio_to_all_reduce": ms / block["all_reduce_ms"],
+                           "link_GBps_per_rank": 4 * p * L / ms / 1e6}
+        except Exception as exc:
+            block[name] = {"error": f"{type(exc).__name__}: {exc}"}
+    names = list(outs)
+    block["identical_results"] = bool(names) and all(torch.equal(outs[names[0]], outs[n]) for n in names[1:])
+    if names:
+        o = outs[names[0]]
+        block["rel_l2_vs_all_reduce_mean"] = float((o - mean).norm() / mean.norm())
+    return block
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -241,7 +511,11 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override d per worker (multiple of c)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-parity", action="store_true", help="accepted for compatibility; parity lives in tests/")
+    ap.add_argument("--no-parity", action="store_true", help="skip the parity block of the cpu_baseline leg")
+    ap.add_argument("--parity-positions", type=int, default=1 << 16)
+    ap.add_argument("--no-configs", action="store_true", help="skip the other configurations and the sweep corners")
+    ap.add_argument("--configs", default="", help="comma-separated subset of the configs block's keys (default: all)")
+    ap.add_argument("--no-ring", action="store_true", help="N > 1: skip the one-worker-per-rank ring block")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--ref-positions", type=int, default=1 << 20)
     ap.add_argument("--kernel-mode", type=int, default=0)
@@ -290,56 +564,27 @@ def main():
         torch.cuda.synchronize()
 
     K = args.steps
-    THERMAL = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"}
-
-    def measure():
-        """W warm-ups, then the timed region: K steps, each the C-ABI sequence encode, rounds 1..L,
-        decode, with a CUDA event after every phase (encode | the L round launches | decode) and the
-        clocks sampled alongside."""
-        sampler = ClockSampler(local_rank) if rank == 0 else None
-        for _ in range(args.warmup):                       # the timed sequence itself, without the events
-            plan.encode(grads, d, ws, d, stream)
-            for k in range(1, L + 1):
-                plan.ring_round(ws, d, k, stream)
-            plan.decode(ws, out, d, d, scale, stream)
-        torch.cuda.synchronize()
-        plan.device_status(stream)
-        if sampler:
-            sampler.wait_first_sample()
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(L + 3)] for _ in range(K)]
-        sync_all()
-        launches0 = plan.launch_count()
-        for s in range(K):
-            e = ev[s]
-            e[0].record()
-            plan.encode(grads, d, ws, d, stream)
-            e[1].record()
-            for k in range(1, L + 1):
-                plan.ring_round(ws, d, k, stream)
-            e[L + 1].record()                              # one event per phase: launches stay back to back
-            plan.decode(ws, out, d, d, scale, stream)
-            e[L + 2].record()
-        sync_all()
-        launches = plan.launch_count() - launches0
-        clocks = sampler.stop() if sampler else None
-        plan.device_status(stream)
-        return ev, launches, clocks
-
-    ev, launches, clocks = measure()
+    gi = local_rank if rank == 0 else None
+    m = time_steps(plan, grads, d, ws, out, d, d, scale, K, args.warmup, stream, gi, sync_all)
     remeasured = False
-    if clocks and THERMAL & set(clocks.get("reasons", [])) and world == 1:
+    if m["clocks"] and THERMAL & set(m["clocks"].get("reasons", [])) and world == 1:
         # a thermal or hardware slowdown during the timed region: the number is not usable; once more
-        first = clocks
-        ev, launches, clocks = measure()
-        clocks["first_attempt_reasons"] = first["reasons"]
+        first = m["clocks"]
+        m = time_steps(plan, grads, d, ws, out, d, d, scale, K, args.warmup, stream, gi, sync_all)
+        m["clocks"]["first_attempt_reasons"] = first["reasons"]
         remeasured = True
-    total_ms = ev[0][0].elapsed_time(ev[K - 1][L + 2])
-    enc_ms = float(np.mean([ev[s][0].elapsed_time(ev[s][1]) for s in range(K)]))
-    dec_ms = float(np.mean([ev[s][L + 1].elapsed_time(ev[s][L + 2]) for s in range(K)]))
-    rounds_all_ms = float(np.mean([ev[s][1].elapsed_time(ev[s][L + 1]) for s in range(K)]))
+    launches, clocks = m["launches"], m["clocks"]
+    total_ms, enc_ms, dec_ms, rounds_all_ms, step_ms = m["total_ms"], m["enc_ms"], m["dec_ms"], m["rounds_ms"], m["step_ms"]
     ms_per_step = max_over_ranks(total_ms, world, dev) / K
     value = whole_job_value(ab["total"], world, ms_per_step)
-    step_ms = [ev[s][0].elapsed_time(ev[s][L + 2]) for s in range(K)]      # this rank's steps, one by one
+    # device results of the last timed aggregation on the first positions of every row, for the parity
+    # block (compared with the oracle's run of the cpu_baseline leg, outside every timed region)
+    p_par = min(p, args.parity_positions)
+    rows_y = torch.tensor(list(range(L)) + [L + 1], device=dev)
+    par_dev = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.no_parity:
+        par_dev = {"Y": ws.view(N, c + N, p)[:, rows_y, :p_par].cpu().numpy(),
+                   "out": out.view(N, c, p)[:, :, :p_par].reshape(N, -1).cpu().numpy()}
 
     peak, peak_kind = load_peaks()
     rounds_bytes = sum(round_bytes(N, c, p, k) for k in range(1, L + 1))
@@ -350,11 +595,13 @@ def main():
     dom_bytes = {"round_kernel": ab["rounds"] / L, "encode": ab["encode"], "decode": ab["decode"]}[dominant]
     dom_ms = {"round_kernel": rounds_ms / L, "encode": enc_ms, "decode": dec_ms}[dominant]
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-    traffic = None
-    if dominant == "round_kernel":
-        traffic = NCU_ROUND_TRAFFIC_OVER_ALGORITHMIC * dom_bytes
+    traffic = NCU_TRAFFIC_OVER_ALGORITHMIC[dominant] * dom_bytes
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                "traffic_source": NCU_TRAFFIC_SOURCE,
+                # the fraction of the HBM roofline proper: DRAM bytes (not algorithmic bytes) over time over peak;
+                # `achieved` / `frac` count every logical buffer once per use and can exceed 1 where L2 serves a re-read
+                "dram_GBps": traffic / (dom_ms * 1e-3) / 1e9, "dram_frac": traffic / (dom_ms * 1e-3) / 1e9 / peak,
                 "frac_of_nominal_8TBps": achieved / 8000.0, "whole_path_frac_of_nominal_8TBps": value / world / 8000.0,
                 "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_ms": dom_ms,
                 "per_kernel": {
@@ -379,19 +626,8 @@ def main():
     # ---- the same K aggregations through the one-call entry point, one event pair around all of
     # them: no event between the launches, so consecutive kernels overlap their launch with the
     # previous kernel's tail (what a caller of cerar_allreduce_sim gets; matters below ~1 ms)
-    for _ in range(3):
-        plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
-    sync_all()
-    o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_one = plan.launch_count()
-    o0.record()
-    for _ in range(K):
-        plan.allreduce_sim(grads, d, out, d, ws, d, scale, stream)
-    o1.record()
-    sync_all()
-    n_one = (plan.launch_count() - n_one) // K
-    plan.device_status(stream)
-    ms_one = max_over_ranks(o0.elapsed_time(o1), world, dev) / K
+    one_ms, n_one = time_one_call(plan, grads, d, ws, out, d, d, scale, K, stream, sync_all)
+    ms_one = max_over_ranks(one_ms, world, dev) / K
     line["one_call"] = {"ms_per_step": ms_one, "value": whole_job_value(ab["total"], world, ms_one), "unit": UNIT,
                         "frac": whole_job_value(ab["total"], world, ms_one) / world / peak,
                         "launches_per_step": int(n_one),
@@ -421,8 +657,6 @@ def main():
             "rounds_one_launch": {"ms": float(ph[1]), "GBps_in_metric_bytes": ab["rounds"] / ph[1] / 1e6},
             "decode": {"ms": float(ph[2]), "GBps": ab["decode"] / ph[2] / 1e6}}
         plan.device_status(stream)
-
-    des = None
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
     if not args.no_e2e:
@@ -465,10 +699,38 @@ def main():
         plan.device_status(stream)
         del h_in, h_out
 
+    g_sample = None
+    p_s = min(p, args.ref_positions)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        if des is None:
+        g_sample = np.ascontiguousarray(grads.view(N, c, p)[:, :, :p_s].reshape(N, -1).cpu().numpy())
+    plan_U, plan_R = [plan.get_U(i) for i in range(N)], [plan.get_R(i) for i in range(N)]
+    del grads, ws, plan
+    if not args.no_e2e:
+        pass                      # `out` went before the pinned buffers were made
+    else:
+        del out
+    torch.cuda.empty_cache()
+
+    if world == 1 and not args.no_configs and not args.d:
+        only = [k for k in args.configs.split(",") if k]
+        line["configs"] = other_configs(args.workload, peak, local_rank, stream, only=only)
+
+    if world > 1 and not args.no_ring:
+        line["ring"] = ring_block(world, rank, dev)
+
+    if g_sample is not None:
+        if cfg["kind"] == "kappa":
+            # library and oracle iterates of the constrained design agree only to ~1e-3 at this shape (the
+            # first projection acts on encoders with kappa ~ 1e15), which the decoder amplifies: the protocol
+            # is run with the plan's own matrices (inputs of the data path, like the gradients)
+            from types import SimpleNamespace
+            des = SimpleNamespace(N=N, c=c, U=plan_U, R=plan_R)
+        else:
             des = build_design_oracle(cfg, B)
-        line["cpu_baseline"] = cpu_baseline(cfg, des, min(p, args.ref_positions), one_thread=True)
+        kept = {}
+        line["cpu_baseline"] = cpu_baseline(cfg, des, p_s, one_thread=True, g=g_sample, keep=kept)
+        if par_dev is not None:
+            line["parity"] = parity_block(des, kept, par_dev, p_s, min(p_par, p_s), scale)
 
     if rank == 0:
         print(json.dumps(line))

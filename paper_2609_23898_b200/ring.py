@@ -87,7 +87,7 @@ class DistributedRing:
     """One worker per rank.  `group` is a torch.distributed process group of exactly
     plan.N ranks whose devices have peer access to one another."""
 
-    def __init__(self, plan, d: int, group=None):
+    def __init__(self, plan, d: int, group=None, device=None):
         import torch
         import torch.distributed as dist
         import torch.distributed._symmetric_memory as symm_mem
@@ -100,7 +100,8 @@ class DistributedRing:
         self.plan, self.d, self.p = plan, d, d // plan.c
         self.N, self.c, self.L = plan.N, plan.c, plan.L
         n = plan.rank_workspace_bytes(d) // 4
-        self.ws = symm_mem.empty(n, dtype=torch.float32, device=torch.device("cuda", torch.cuda.current_device()))
+        dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        self.ws = symm_mem.empty(n, dtype=torch.float32, device=dev)
         self._hdl = symm_mem.rendezvous(self.ws, group)
         self.peer_ws = self._hdl.get_buffer((self.rank + 1) % self.N, (n,), torch.float32)
         self.barrier_timeout_ms = 10000

@@ -32,7 +32,8 @@ def test_reference_arm_line_on_the_small_config():
 
 @pytest.mark.gpu
 def test_product_arm_line_on_the_small_config():
-    j = _run(["--workload", "cfg1", "--steps", "4", "--warmup", "3", "--ref-positions", "4096"])
+    j = _run(["--workload", "cfg1", "--steps", "4", "--warmup", "3", "--ref-positions", "4096",
+              "--configs", "cfg2,sweep_N4_c16_d2^26"])
     with open(os.path.join(ROOT, "BASELINE.json")) as f:
         assert j["metric"] == json.load(f)["metric"]
     assert j["unit"] == "GB/s" and j["n_gpus"] == 1 and j["steps"] == 4 and j["warmup"] == 3
@@ -54,3 +55,20 @@ def test_product_arm_line_on_the_small_config():
     ck = j["clocks"]
     assert ck is None or {"sm_mhz", "sm_max_mhz", "reasons"} <= set(ck)
     assert j["one_call"]["ms_per_step"] > 0
+    # DRAM-based fraction next to the algorithmic one
+    assert rf["dram_frac"] == pytest.approx(rf["traffic"] / (rf["avg_launch_ms"] * 1e-3) / 1e9 / rf["peak"])
+    # parity next to the number: GPU against the oracle on sampled positions, outside the timed region
+    par = j["parity"]
+    assert par["sampled_positions"] == 4096 and par["rel_l2_Y"] < 2e-6
+    assert par["kappa_times_2^-24"] == pytest.approx(par["kappa_M"] * 2.0 ** -24)
+    assert par["rel_l2_out"] < 4 * par["kappa_times_2^-24"]
+    assert par["end_to_end_residual_over_bound"] <= 1.0 and par["decode_residual_over_bound"] <= 1.0
+    # the other configurations, timed the same way
+    cf = j["configs"]
+    assert set(cf) == {"cfg2", "sweep_N4_c16_d2^26"}
+    for key, N2, c2 in (("cfg2", 4, 16), ("sweep_N4_c16_d2^26", 4, 16)):
+        e2 = cf[key]
+        assert "error" not in e2 and "skipped" not in e2, e2
+        assert e2["gpu_launches"] == e2["steps"] * (c2 + N2 - 2 + 2)
+        assert e2["ms_per_step"] > 0 and e2["frac"] == pytest.approx(e2["value"] / rf["peak"])
+        assert set(e2["per_kernel_GBps"]) == {"encode", "round_kernel", "decode"}
