@@ -15,8 +15,9 @@ protocol : chunking, encoding, the ring rounds from the update equations (and,
 designs  : the coefficient constructions (multiplicative perturbation
            construction, Vandermonde, epsilon-construction, the
            condition-number-constrained alternating least squares heuristic).
-mixed    : the ring rounds with bfloat16 messages (binary32 worker arithmetic,
-           every transmitted vector rounded to nearest-even by its sender).
+mixed    : the ring rounds with bfloat16 or 8-bit (e4m3, power-of-two scale per
+           tile of positions) messages: binary32 worker arithmetic, every
+           transmitted vector rounded to nearest-even by its sender.
 
 Pins (what each function is checked against, see tests/test_oracle_*.py):
   rounds / whole pipeline : brute-force composition Y_i = G^(i) M_i(U) for
@@ -31,6 +32,9 @@ Pins (what each function is checked against, see tests/test_oracle_*.py):
       returned, and the known optimum Phi = 0 at c = N.  Which local solution is
       reached at c > N has no published counterpart: PARITY UNPINNED for that
       end point.
+  8-bit messages : the e4m3 rounding against hand-worked values (ties, subnormals,
+      clamping) and torch's float8_e4m3fn conversion bit for bit; the tile scales
+      against their defining inequality; the rounds as for bfloat16.
   bfloat16 messages : the rounding against worked values, IEEE properties and
       torch's conversion; the rounds against Algorithm 1 where nothing rounds and
       against the error the message precision implies.
