@@ -42,13 +42,19 @@ def _metric_name():
 
 METRIC = _metric_name()
 UNIT = "GB/s"
-# DRAM bytes per launch over algorithmic bytes per launch, from ncu captures of smaller cases of the
-# same kernels (N=8, c=32, p=1 Mi; summaries under profiles/): means over consecutive launches with
-# the caches left alone between them (--cache-control none), so that what one launch leaves dirty in
-# L2 is counted when the next launch evicts it.  DRAM traffic grows in proportion to the positions, so
-# the ratio is applied to the algorithmic bytes of the timed launch.
-NCU_TRAFFIC_OVER_ALGORITHMIC = {"round_kernel": 1.0, "encode": 1.0, "decode": 1.0}
-NCU_TRAFFIC_SOURCE = "algorithmic bytes (no steady-state ncu capture folded in yet)"
+# DRAM bytes per launch against algorithmic bytes per launch, from ncu captures of a smaller case of the
+# same kernels (N=8, c=32, p=1 Mi; profiles/dram_traffic_steady_state_N8_c32_p1M.md): means over
+# consecutive launches with the caches left alone between them (--cache-control none), so that what one
+# launch leaves dirty in L2 is counted when the next one evicts it.  The contractions' traffic grows in
+# proportion to the positions (encode 0.997, decode 1.019 of the algorithmic bytes: decode also fetches the
+# stale slot between y_L and y_{L+1}).  A ring round finds the newest part of the previous round's message
+# still in L2: 22.8 MB per launch at that size, a window of L2's size that does not grow with p, so it is
+# subtracted rather than scaled.
+NCU_TRAFFIC_OVER_ALGORITHMIC = {"round_kernel": 1.0, "encode": 0.997, "decode": 1.019}
+NCU_L2_WINDOW_BYTES = {"round_kernel": 22.8e6, "encode": 0.0, "decode": 0.0}
+NCU_TRAFFIC_SOURCE = ("ncu dram__bytes_read.sum + dram__bytes_write.sum, steady state over consecutive launches at "
+                      "N=8, c=32, p=2^20; contractions scaled by positions, rounds: algorithmic bytes minus the "
+                      "22.8 MB per launch that L2 served there")
 
 
 def algorithmic_bytes(N, c, p):
@@ -199,6 +205,9 @@ def parity_block(des, kept, par_dev, p_sample, p_par, scale):
     L = c + N - 2
     u = 2.0 ** -24
     res, g = kept["res"], kept["g"]
+    p_dev = par_dev["Y"].shape[2]                      # positions read back from the device (>= p_par)
+    par_dev = {"Y": np.ascontiguousarray(par_dev["Y"][:, :, :p_par]),
+               "out": np.ascontiguousarray(par_dev["out"].reshape(N, c, p_dev)[:, :, :p_par]).reshape(N, -1)}
     pick = lambda v, rows: np.ascontiguousarray(v.reshape(rows, p_sample)[:, :p_par])
     Y_ora = np.stack([res["Y"][i][:p_par].T for i in range(N)])                       # (N, L+1, p_par)
     out_ora = [pick(res["out"][i], c).reshape(-1) for i in range(N)]
@@ -595,7 +604,7 @@ def main():
     dom_bytes = {"round_kernel": ab["rounds"] / L, "encode": ab["encode"], "decode": ab["decode"]}[dominant]
     dom_ms = {"round_kernel": rounds_ms / L, "encode": enc_ms, "decode": dec_ms}[dominant]
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_OVER_ALGORITHMIC[dominant] * dom_bytes
+    traffic = NCU_TRAFFIC_OVER_ALGORITHMIC[dominant] * dom_bytes - min(NCU_L2_WINDOW_BYTES[dominant], 0.25 * dom_bytes)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                 "traffic_source": NCU_TRAFFIC_SOURCE,

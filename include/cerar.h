@@ -295,6 +295,24 @@ cerar_status_t cerar_rank_round_msg_bf16(cerar_plan_t* plan, int rank, const flo
                                          int k, cerar_stream_t stream);
 cerar_status_t cerar_rank_recv_bf16(cerar_plan_t* plan, int rank, float* ws, const uint16_t* msg, int64_t d, int k,
                                     cerar_stream_t stream);
+/* 8-bit transport (same remark on the paper as for bfloat16: Sec. I, Related Work only notes that
+ * quantisation is complementary; the combination is this library's).  cerar_rank_round_msg_fp8 forms the
+ * message of round k in binary32 and writes, per tile of CERAR_FP8_TILE consecutive positions, one
+ * power-of-two scale 2^e (binary32; e the smallest integer with max|x| 2^-e <= 448 over the tile, 0 for a
+ * tile of zeros, kept within [-100, 100]) and per position the 8-bit code of x 2^-e in the e4m3 format
+ * (4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest value 448), rounded to nearest
+ * with ties to even.  msg: device memory of cerar_fp8_message_bytes(plan, d) bytes, 16-byte aligned:
+ * d/c codes, padding to a multiple of 16 bytes, then the scales.  cerar_rank_recv_fp8 expands a message
+ * that has arrived into slot k-1 of the receiver's workspace (code value times scale, exact in binary32).
+ * A quarter of the bytes cross the transport; every message carries a relative error of up to 2^-4 of
+ * its tile's largest magnitude, which the decoder amplifies by about kappa_2(M_i): for designs with a
+ * condition number of order 1..100 only (c = N, or the constrained design with a small bound). */
+#define CERAR_FP8_TILE 1024
+size_t         cerar_fp8_message_bytes(const cerar_plan_t* plan, int64_t d);
+cerar_status_t cerar_rank_round_msg_fp8(cerar_plan_t* plan, int rank, const float* ws, void* msg, int64_t d, int k,
+                                        cerar_stream_t stream);
+cerar_status_t cerar_rank_recv_fp8(cerar_plan_t* plan, int rank, float* ws, const void* msg, int64_t d, int k,
+                                   cerar_stream_t stream);
 cerar_status_t cerar_rank_decode(cerar_plan_t* plan, int rank, const float* ws, float* out, int64_t d,
                                  float scale, cerar_stream_t stream);
 

@@ -9,7 +9,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libcerar.so")
-SOURCES = ["api.cu", "kernels.cu", "contract_tc.cu", "fused.cu", "ring.cu", "ring_fused.cu", "static_ws.cu", "plan.cpp"]
+SOURCES = ["api.cu", "kernels.cu", "contract_tc.cu", "fused.cu", "ring.cu", "ring_fused.cu", "ring_fp8.cu", "static_ws.cu", "plan.cpp"]
 HEADERS = ["kernels.cuh", "ptx.cuh", "tc_common.cuh", "plan.hpp", "linalg.hpp", os.path.join("..", "..", "include", "cerar.h")]
 
 

@@ -94,6 +94,10 @@ lib.cerar_rank_decode.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, C.c_float, _
 lib.cerar_rank_round_msg.argtypes = [_vp, C.c_int, _f32p, _f32p, _i64, C.c_int, _vp]
 lib.cerar_rank_round_msg_bf16.argtypes = [_vp, C.c_int, _f32p, _vp, _i64, C.c_int, _vp]
 lib.cerar_rank_recv_bf16.argtypes = [_vp, C.c_int, _f32p, _vp, _i64, C.c_int, _vp]
+lib.cerar_fp8_message_bytes.argtypes = [_vp, _i64]
+lib.cerar_fp8_message_bytes.restype = C.c_size_t
+lib.cerar_rank_round_msg_fp8.argtypes = [_vp, C.c_int, _f32p, _vp, _i64, C.c_int, _vp]
+lib.cerar_rank_recv_fp8.argtypes = [_vp, C.c_int, _f32p, _vp, _i64, C.c_int, _vp]
 lib.cerar_ring_tiles.argtypes = [_vp, _i64]
 lib.cerar_ring_tiles.restype = _i64
 lib.cerar_rank_rounds_fused.argtypes = [_vp, C.c_int, _f32p, _f32p, _vp, _vp, _vp, _vp, _i64, C.c_uint, _vp]
@@ -297,6 +301,15 @@ class Plan:
 
     def rank_recv_bf16(self, rank, ws, msg, d, k, stream=0):
         _check(lib.cerar_rank_recv_bf16(self._h, rank, _ptr(ws), _ptr(msg), d, k, stream))
+
+    def fp8_message_bytes(self, d: int) -> int:
+        return int(lib.cerar_fp8_message_bytes(self._h, d))
+
+    def rank_round_msg_fp8(self, rank, ws, msg, d, k, stream=0):
+        _check(lib.cerar_rank_round_msg_fp8(self._h, rank, _ptr(ws), _ptr(msg), d, k, stream))
+
+    def rank_recv_fp8(self, rank, ws, msg, d, k, stream=0):
+        _check(lib.cerar_rank_recv_fp8(self._h, rank, _ptr(ws), _ptr(msg), d, k, stream))
 
     def ring_tiles(self, d: int) -> int:
         return int(lib.cerar_ring_tiles(self._h, d))

@@ -552,6 +552,44 @@ cerar_status_t cerar_rank_recv_bf16(cerar_plan_t* P, int rank, float* ws, const 
     return CERAR_OK;
 }
 
+size_t cerar_fp8_message_bytes(const cerar_plan_t* P, int64_t d) {
+    if (!P || d <= 0 || d % P->host.c != 0) return 0;
+    return cerar::fp8_message_bytes(d / P->host.c);
+}
+
+cerar_status_t cerar_rank_round_msg_fp8(cerar_plan_t* P, int rank, const float* ws, void* msg, int64_t d, int k,
+                                        cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !msg) return fail(CERAR_ERR_INVALID_ARG, "ws or msg is NULL");
+    if (reinterpret_cast<uintptr_t>(msg) & 15u) return fail(CERAR_ERR_INVALID_ARG, "msg must be 16-byte aligned");
+    if (rank < 0 || rank >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    if (k < 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "round index outside 1..L");
+    cerar::RankRoundArgs a{};
+    a.ws = ws; a.peer_ws = nullptr; a.p = p; a.N = P->host.N; a.c = P->host.c; a.k = k; a.to_message = 3;
+    cudaError_t e = cerar::launch_rank_round_fp8(a, msg, P->num_sms, (cudaStream_t)stream, &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rank round (8-bit message) launch");
+    return CERAR_OK;
+}
+
+cerar_status_t cerar_rank_recv_fp8(cerar_plan_t* P, int rank, float* ws, const void* msg, int64_t d, int k,
+                                   cerar_stream_t stream) {
+    int64_t p;
+    cerar_status_t st = check_data_call(P, d, &p);
+    if (st != CERAR_OK) return st;
+    if (!ws || !msg) return fail(CERAR_ERR_INVALID_ARG, "ws or msg is NULL");
+    if (reinterpret_cast<uintptr_t>(msg) & 15u) return fail(CERAR_ERR_INVALID_ARG, "msg must be 16-byte aligned");
+    if (rank < 0 || rank >= P->host.N) return fail(CERAR_ERR_INVALID_ARG, "rank outside 0..N-1");
+    if (k < 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "round index outside 1..L");
+    int sp, sc, sa, sl;
+    cerar::rank_round_slots(P->host.N, P->host.c, k, &sp, &sc, &sa, &sl);
+    cudaError_t e = cerar::launch_rank_recv_fp8(ws + (int64_t)sl * p, msg, p, P->num_sms, (cudaStream_t)stream,
+                                                &P->launches);
+    if (e != cudaSuccess) return cuda_fail(e, "rank receive (8-bit message) launch");
+    return CERAR_OK;
+}
+
 cerar_status_t cerar_rank_decode(cerar_plan_t* P, int rank, const float* ws, float* out, int64_t d, float scale,
                                  cerar_stream_t stream) {
     int64_t p;

@@ -87,6 +87,10 @@ void rank_round_slots(int N, int c, int k, int* slot_prev, int* slot_cancel, int
 cudaError_t launch_rank_round(RankRoundArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 cudaError_t launch_rank_recv_bf16(float* slot, const unsigned short* msg, int64_t p, int num_sms, cudaStream_t s,
                                   uint64_t* launches);
+// 8-bit messages (e4m3 codes + one power-of-two scale per CERAR_FP8_TILE positions); msg is 16-byte aligned
+size_t fp8_message_bytes(int64_t p);
+cudaError_t launch_rank_round_fp8(RankRoundArgs a, void* msg, int num_sms, cudaStream_t s, uint64_t* launches);
+cudaError_t launch_rank_recv_fp8(float* slot, const void* msg, int64_t p, int num_sms, cudaStream_t s, uint64_t* launches);
 // cooperative = true when the launch serves workers that wait on one another (all on this GPU).
 cudaError_t launch_ring_rounds(const RingFusedArgs& a, int nworkers, bool cooperative, int num_sms, cudaStream_t s,
                                uint64_t* launches);
