@@ -144,10 +144,11 @@ class DistributedRing:
 class SendRecvRing:
     """One worker per rank, messages moved by torch.distributed send / receive.
     bf16_messages=True: the sender rounds every message to bfloat16 and the receiver expands it
-    (cerar_rank_round_msg_bf16 / cerar_rank_recv_bf16): half the bytes on the wire, for
-    well-conditioned designs."""
+    (cerar_rank_round_msg_bf16 / cerar_rank_recv_bf16): half the bytes on the wire; fp8_messages=True:
+    e4m3 codes with a power-of-two scale per 1024 positions (cerar_rank_round_msg_fp8 /
+    cerar_rank_recv_fp8): a quarter.  Both for well-conditioned designs only."""
 
-    def __init__(self, plan, d: int, group=None, device=None, bf16_messages=False):
+    def __init__(self, plan, d: int, group=None, device=None, bf16_messages=False, fp8_messages=False):
         import torch
         import torch.distributed as dist
         self.group = group if group is not None else dist.group.WORLD
@@ -161,8 +162,17 @@ class SendRecvRing:
         dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
         self.ws = torch.empty(plan.rank_workspace_bytes(d) // 4, dtype=torch.float32, device=dev)
         self.bf16 = bool(bf16_messages)
-        self.msg = torch.empty(self.p, dtype=torch.bfloat16 if self.bf16 else torch.float32, device=dev)
-        self.msg_in = torch.empty(self.p, dtype=torch.bfloat16, device=dev) if self.bf16 else None
+        self.fp8 = bool(fp8_messages)
+        if self.bf16 and self.fp8:
+            raise ValueError("one message format at a time")
+        if self.fp8:
+            # e4m3 codes plus one scale per tile (cerar_rank_round_msg_fp8 / cerar_rank_recv_fp8)
+            nb = (plan.fp8_message_bytes(d) + 15) // 16 * 16
+            self.msg = torch.empty(nb, dtype=torch.uint8, device=dev)
+            self.msg_in = torch.empty(nb, dtype=torch.uint8, device=dev)
+        else:
+            self.msg = torch.empty(self.p, dtype=torch.bfloat16 if self.bf16 else torch.float32, device=dev)
+            self.msg_in = torch.empty(self.p, dtype=torch.bfloat16, device=dev) if self.bf16 else None
         self.schedule = round_schedule(plan)
         self.nxt = dist.get_global_rank(self.group, (self.rank + 1) % self.N)
         self.prv = dist.get_global_rank(self.group, (self.rank - 1) % self.N)
@@ -174,14 +184,18 @@ class SendRecvRing:
         self.plan.rank_encode(self.rank, grad, self.ws, self.d, stream)
         rows = self.ws.view(self.c + self.N + 1, self.p)
         for k, _prev, _cancel, _add, land in self.schedule:
-            if self.bf16:
+            if self.fp8:
+                self.plan.rank_round_msg_fp8(self.rank, self.ws, self.msg, self.d, k, stream)
+            elif self.bf16:
                 self.plan.rank_round_msg_bf16(self.rank, self.ws, self.msg, self.d, k, stream)
             else:
                 self.plan.rank_round_msg(self.rank, self.ws, self.msg, self.d, k, stream)
             ops = [dist.P2POp(dist.isend, self.msg, self.nxt, self.group),
-                   dist.P2POp(dist.irecv, self.msg_in if self.bf16 else rows[land], self.prv, self.group)]
+                   dist.P2POp(dist.irecv, self.msg_in if (self.bf16 or self.fp8) else rows[land], self.prv, self.group)]
             for req in dist.batch_isend_irecv(ops):
                 req.wait()
-            if self.bf16:
+            if self.fp8:
+                self.plan.rank_recv_fp8(self.rank, self.ws, self.msg_in, self.d, k, stream)
+            elif self.bf16:
                 self.plan.rank_recv_bf16(self.rank, self.ws, self.msg_in, self.d, k, stream)
         self.plan.rank_decode(self.rank, self.ws, out, self.d, scale, stream)

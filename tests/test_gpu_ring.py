@@ -348,6 +348,124 @@ def test_bf16_messages_whole_pipeline_within_the_rounding_noise(mods, N, c, p):
     assert 1e-4 < worst_exact < 2.0 ** -8 * (c + N), worst_exact
 
 
+def _fp8_rounds_on_device(plan, r, d, N, s, torch, keep_round=None):
+    """All L rounds with 8-bit messages: every worker's message (codes + tile scales) into a byte buffer,
+    then the neighbour expands that buffer into its landing slot.  Returns the buffers of round keep_round."""
+    nbytes = plan.fp8_message_bytes(d)
+    raw = torch.full((N, (nbytes + 15) // 16 * 16), 0xAB, dtype=torch.uint8, device="cuda")
+    kept = None
+    for k in range(1, plan.L + 1):
+        for i in range(N):
+            plan.rank_round_msg_fp8(i, r.ws[i], raw[i], d, k, s)
+        if k == keep_round:
+            torch.cuda.synchronize()
+            kept = raw.cpu().numpy().copy()
+        for i in range(N):
+            plan.rank_recv_fp8((i + 1) % N, r.ws[(i + 1) % N], raw[i], d, k, s)
+    return kept
+
+
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192 + 260), (3, 5, 1031), (2, 2, 4), (8, 32, 4100), (5, 7, 3), (4, 4, 4096),
+                                   (4, 4, 1024), (3, 6, 2049)])
+def test_fp8_messages_equal_the_oracle_bit_for_bit(mods, N, c, p):
+    """8-bit messages (cerar_rank_round_msg_fp8 / cerar_rank_recv_fp8): a power-of-two scale per tile of 1024
+    positions and an e4m3 code per position.  As for bfloat16, both sides quantise the SAME binary32 encoded
+    vectors (seeded synthetic deltas of widely different magnitudes per row, a zero tile included), so
+    codes, scales and the observations Y must agree with the oracle bit for bit; ragged last tiles, p not a
+    multiple of 4 and p smaller than a tile are among the shapes."""
+    import torch
+    from oracle import mixed as Mx
+    from oracle import protocol as P
+    cerar, inputs, ring = mods
+    d = c * p
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(5 * N + c))
+    plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+    assert plan.fp8_message_bytes(d) == (p + 15) // 16 * 16 + 4 * ((p + 1023) // 1024)
+    s = torch.cuda.current_stream().cuda_stream
+    r = ring.LocalRing(plan, d)
+    rows = c + N + 1
+    delta = inputs.gradients_numpy(N, d, "normal", seed=14).reshape(N, c, p)
+    mags = 10.0 ** np.random.default_rng(3).uniform(-6, 6, (N, c, 1))
+    delta = (delta * mags).astype(np.float32)
+    delta[0, 0, :min(p, 1024)] = 0.0                                       # a tile of zeros in the first message
+    for i in range(N):
+        r.ws[i].fill_(float("nan"))
+        r.ws[i].view(rows, p)[N + 1:N + 1 + c].copy_(torch.from_numpy(delta[i]))
+    kept = _fp8_rounds_on_device(plan, r, d, N, s, torch, keep_round=1)
+    torch.cuda.synchronize()
+    plan.device_status(s)
+    # round 1: x_{i,1} = delta_{i,1}; what went on the wire, byte for byte
+    off = (p + 15) // 16 * 16
+    nt = (p + 1023) // 1024
+    for i in range(N):
+        codes, scales, _ = Mx.quantize_fp8_tiles(delta[i, 0])
+        assert np.array_equal(kept[i, :p], codes), i
+        assert np.array_equal(kept[i, off:off + 4 * nt].view(np.float32), scales), i
+    ys = ring.y_slots(plan)
+    Y_dev = [r.ws[i].view(rows, p)[ys].cpu().numpy().T for i in range(N)]
+    Y_ora = Mx.run_rounds_fp8([delta[i].T.copy() for i in range(N)])
+    for i in range(N):
+        assert np.array_equal(Y_dev[i].view(np.uint32), Y_ora[i].view(np.uint32)), i
+    outs = [torch.empty(d, device="cuda") for _ in range(N)]
+    r.decode(outs, 1.0 / N, s)
+    torch.cuda.synchronize()
+    for i in range(N):
+        want = P.unchunk(P.decode(Y_ora[i].astype(np.float64), des.R[i], 1.0 / N))
+        assert rel_l2(outs[i].cpu().numpy(), want) < 5e-6
+    raw = torch.zeros(plan.fp8_message_bytes(d) + 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(cerar.CerarError):
+        plan.rank_round_msg_fp8(0, r.ws[0], raw, d, plan.L + 1, s)
+    with pytest.raises(cerar.CerarError):
+        plan.rank_recv_fp8(N, r.ws[0], raw, d, 1, s)
+    with pytest.raises(cerar.CerarError):
+        plan.rank_round_msg_fp8(0, r.ws[0], raw.data_ptr() + 4, d, 1, s)          # not 16-byte aligned
+
+
+def test_message_precision_against_the_condition_number(mods):
+    """What low-precision messages cost, by design: decoded relative error (against the fp64 oracle with
+    exact messages) for binary32 / bfloat16 / 8-bit messages on a well-conditioned design (c = N) and on one
+    with kappa ~ 1e4.  The error follows kappa_2(M_i) times the message precision: usable at c = N, useless
+    where kappa times 2^-4 exceeds one."""
+    import torch
+    from oracle import protocol as P
+    cerar, inputs, ring = mods
+    p = 4096
+    table = []
+    for N, c, eps in ((4, 4, 1e-3), (8, 8, 1e-3), (4, 8, 1e-2)):
+        d = c * p
+        B = inputs.base_matrix(N, c, 0)
+        des = Dz.epsilon(N, c, eps, B)
+        kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+        plan = cerar.Plan.create_custom(N, c, des.U, des.R)
+        g = inputs.gradients_numpy(N, d, "normal", seed=15)
+        ora = run_oracle(des.U, des.R, g, 1.0 / N)
+        s = torch.cuda.current_stream().cuda_stream
+        errs = {}
+        for kind in ("f32", "bf16", "fp8"):
+            r = ring.LocalRing(plan, d)
+            r.encode([torch.from_numpy(g[i]).cuda() for i in range(N)], s)
+            if kind == "f32":
+                for k in range(1, plan.L + 1):
+                    r.round(k, s)
+            elif kind == "bf16":
+                _bf16_rounds_on_device(plan, ring, r, d, p, N, s, torch)
+            else:
+                _fp8_rounds_on_device(plan, r, d, N, s, torch)
+            outs = [torch.empty(d, device="cuda") for _ in range(N)]
+            r.decode(outs, 1.0 / N, s)
+            torch.cuda.synchronize()
+            plan.device_status(s)
+            errs[kind] = max(rel_l2(outs[i].cpu().numpy(), ora["out"][i]) for i in range(N))
+        table.append((N, c, kap, errs))
+        print(f"\n[N={N} c={c} kappa_M={kap:.2e}] rel. error of the decoded mean: f32 {errs['f32']:.2e}  "
+              f"bf16 {errs['bf16']:.2e}  fp8 {errs['fp8']:.2e}")
+        assert errs["f32"] < 4 * kap * 2.0 ** -24 + 1e-6
+        assert errs["f32"] < errs["bf16"] < errs["fp8"]
+        assert errs["bf16"] < kap * 2.0 ** -8 * 4 and errs["fp8"] < kap * 2.0 ** -4 * 4
+    assert table[0][3]["fp8"] < 0.5                                        # c = N: coarse but a mean
+    assert table[2][3]["fp8"] > 1.0                                        # kappa ~ 1e4: no correct digit left
+
+
 def test_rank_level_kernels_on_symmetric_memory_allocations(mods):
     """DistributedRing keeps workspaces and counters in torch's symmetric memory.  With one GPU
     the peer mapping cannot be exercised, but the allocations can: a one-rank NCCL group,
