@@ -13,6 +13,14 @@ Four tables from the library's fp64 design builder (host_only plans):
      and the kappa_2(M_i) it ends with.
 Phi is the squared least-squares error of Eq. (F); the relative error of the decoded sum is
 about sqrt(Phi / (N c)) for i.i.d. gradients.
+
+  python -m paper_2609_23898_b200.tradeoff --messages            (needs a GPU)
+
+A fifth table, measured on the device: the relative error of the decoded mean (against the exact
+mean of the gradients, max over workers) when the ring messages travel as binary32, bfloat16 or 8-bit
+e4m3 values, for designs of increasing kappa_2(M_i): c = N (r* = 0), the constrained design with a
+small bound, and an epsilon-construction with c = 2N.  One worker per workspace on this GPU
+(ring.LocalRing); a "transport" is the sender's message kernel followed by the receiver's.
 """
 from __future__ import annotations
 
@@ -30,8 +38,11 @@ def main():
     ap.add_argument("--als-iters", type=int, default=200)
     ap.add_argument("--sweeps", type=int, default=2)
     ap.add_argument("--grid", type=int, default=17)
+    ap.add_argument("--messages", action="store_true", help="message precision against kappa (GPU)")
     args = ap.parse_args()
     from . import cerar, inputs
+    if args.messages:
+        return message_precision_table(args.seed)
     N, c = args.N, args.c
     B = inputs.base_matrix(N, c, args.seed)
     r_star = -(-c // N) - 1
@@ -89,6 +100,53 @@ def main():
             p.destroy()
         except cerar.CerarError as e:
             print(f"| {C:g} | - | - | {e} |", flush=True)
+
+
+def message_precision_table(seed=0, p=1 << 16):
+    import torch
+    from . import cerar, inputs, ring
+    stream = torch.cuda.current_stream().cuda_stream
+    designs = [("epsilon 1e-3, c = N", 4, 4, cerar.EPSILON, 1e-3), ("epsilon 1e-3, c = N", 8, 8, cerar.EPSILON, 1e-3),
+               ("epsilon 1e-3, c = N", 16, 16, cerar.EPSILON, 1e-3), ("kappa <= 30", 4, 12, cerar.KAPPA, 30.0),
+               ("kappa <= 100", 4, 12, cerar.KAPPA, 100.0), ("kappa <= 100", 8, 32, cerar.KAPPA, 100.0),
+               ("epsilon 1e-2, c = 2N", 4, 8, cerar.EPSILON, 1e-2)]
+    print("| design | N | c | kappa_M | Phi | binary32 | bfloat16 | e4m3 + tile scale | bytes per message value |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for name, N, c, kind, param in designs:
+        d = c * p
+        plan = cerar.Plan.create(N, c, kind, param, B=inputs.base_matrix(N, c, seed))
+        info = plan.info()
+        g = torch.empty(N, d, device="cuda")
+        inputs.fill_gradients_torch([g[i] for i in range(N)], "normal", seed=seed)
+        mean = g.double().mean(dim=0)
+        errs = []
+        for fmt in ("f32", "bf16", "fp8"):
+            r = ring.LocalRing(plan, d)
+            r.encode([g[i] for i in range(N)], stream)
+            if fmt == "f32":
+                for k in range(1, plan.L + 1):
+                    r.round(k, stream)
+            else:
+                nb = p * 2 if fmt == "bf16" else (plan.fp8_message_bytes(d) + 15) // 16 * 16
+                raw = torch.empty(N, nb, dtype=torch.uint8, device="cuda")
+                send = plan.rank_round_msg_bf16 if fmt == "bf16" else plan.rank_round_msg_fp8
+                recv = plan.rank_recv_bf16 if fmt == "bf16" else plan.rank_recv_fp8
+                for k in range(1, plan.L + 1):
+                    for i in range(N):
+                        send(i, r.ws[i], raw[i], d, k, stream)
+                    for i in range(N):
+                        recv((i + 1) % N, r.ws[(i + 1) % N], raw[i], d, k, stream)
+            outs = [torch.empty(d, device="cuda") for _ in range(N)]
+            r.decode(outs, 1.0 / N, stream)
+            torch.cuda.synchronize()
+            plan.device_status(stream)
+            errs.append(max(float((o.double() - mean).norm() / mean.norm()) for o in outs))
+            del r, outs
+        print(f"| {name} | {N} | {c} | {info['kappa_M_max']:.2e} | {info['phi']:.2e} | {errs[0]:.2e} | {errs[1]:.2e} | "
+              f"{errs[2]:.2e} | 4 / 2 / {plan.fp8_message_bytes(d) / p:.3f} |", flush=True)
+        plan.destroy()
+        del g
+        torch.cuda.empty_cache()
 
 
 if __name__ == "__main__":

@@ -170,3 +170,59 @@ def test_config3_full_size_one_worker_per_rank_fused_rounds():
     assert yard["decode_ratio"] <= 1.0 and yard["end_to_end_ratio"] <= 1.0, yard
     del r, grads
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("N,c,lg_d", [(4, 4, 26), (8, 8, 28), (16, 16, 28), (16, 32, 26), (16, 128, 24)])
+def test_sweep_points_at_the_size_they_are_timed_at(N, c, lg_d):
+    """Points of the throughput sweep (epsilon-construction with eps = 1e-3, N(0,1) gradients, in place) at
+    the d they are timed at, checked on sampled positions.  c = N has kappa_2(M_i) below 1e3: the decoded mean
+    must be within 1e-4 of the oracle's.  The points with c > N are ill-conditioned: observations to
+    roundoff, decoded output within the a-priori rounding bounds."""
+    import torch
+    from paper_2609_23898_b200 import cerar, inputs
+    from tests._harness import rounding_yardsticks
+    d = (1 << lg_d) // (4 * c) * (4 * c)
+    p, L = d // c, c + N - 2
+    B = inputs.base_matrix(N, c, 0)
+    des = Dz.epsilon(N, c, 1e-3, B)
+    kap = max(P.kappa2(P.m_matrix(des.U, i)) for i in range(N))
+    plan = cerar.Plan.create(N, c, cerar.EPSILON, 1e-3, B=B)
+    ws = torch.empty(plan.workspace_bytes(d) // 4, dtype=torch.float32, device="cuda")
+    wv = ws.view(N, c + N, p)
+    s = torch.cuda.current_stream().cuda_stream
+    rng = np.random.default_rng(lg_d + c)
+    tile = 256
+    starts = sorted({0, p - tile} | {int(x) for x in rng.integers(0, p - tile, 6)})
+    idx = torch.from_numpy(np.concatenate([np.arange(a, a + tile) for a in starts])).cuda()
+    rows_y = torch.tensor(list(range(L)) + [L + 1], device="cuda")
+    gp, stride = ws.data_ptr() + 4 * N * p, (c + N) * p
+    outs = {}
+    for how in ("per_round", "one_call"):
+        inputs.fill_gradients_torch([wv[i, N:, :].reshape(-1) for i in range(N)], "normal", seed=3)
+        g_sub = wv[:, N:, :][:, :, idx].reshape(N, -1).cpu().numpy()
+        if how == "per_round":
+            plan.encode(gp, stride, ws, d, s)
+            for k in range(1, L + 1):
+                plan.ring_round(ws, d, k, s)
+            Y_dev = wv[:, rows_y[:, None], idx[None, :]].cpu().numpy()
+            plan.decode(ws, gp, stride, d, 1.0 / N, s)
+        else:
+            plan.allreduce_sim(gp, stride, gp, stride, ws, d, 1.0 / N, s)
+        torch.cuda.synchronize()
+        plan.device_status(s)
+        outs[how] = wv[:, N:, :][:, :, idx].reshape(N, -1).cpu().numpy()
+    ora = P.allreduce([x.astype(np.float64) for x in g_sub], des.U, des.R, 1.0 / N)
+    Y_ora = np.stack([ora["Y"][i].T for i in range(N)])
+    err_y = P.rel_l2(Y_dev, Y_ora)
+    yard = rounding_yardsticks(des.U, des.R, g_sub, 1.0 / N, Y_dev=Y_dev, out_dev=outs["per_round"])
+    err_out = max(P.rel_l2(outs["per_round"][i], ora["out"][i]) for i in range(N))
+    print(f"\n[sweep N={N} c={c} d=2^{lg_d}] kappa_M {kap:.2e} rel_l2_Y {err_y:.2e} rel_l2_out {err_out:.2e} {yard}")
+    assert err_y < 2e-6
+    assert np.array_equal(outs["per_round"], outs["one_call"])          # the two launch forms agree bit for bit
+    assert yard["decode_ratio"] <= 1.0 and yard["end_to_end_ratio"] <= 1.0
+    if kap <= 1e3:
+        assert err_out <= 1e-4
+    else:
+        assert err_out < 4 * kap * U32 or not np.isfinite(kap)
+    del ws
+    torch.cuda.empty_cache()
