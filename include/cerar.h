@@ -413,6 +413,9 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "tc_variant"                    1 = always tiles of 128 positions (default: tiles of 256
  *                                   positions for c <= 64); 2 / 3 = tiles of 256 with one /
  *                                   two MMA issuers per half
+ *   "tc_epi"                        epilogue of the tensor-core kernels: 1 = a group of four warps
+ *                                   per tile parity, 2 = all eight warps on every tile (default:
+ *                                   chosen by shape)
  *   "ring_wait_ms"                  limit of the waits of the fused ring rounds (default 2000)
  *   "ring_tile"                     positions per tile of the fused ring rounds (a multiple of 4;
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters

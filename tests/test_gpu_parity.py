@@ -130,15 +130,17 @@ def test_tensor_core_tile_variants(cerar_mod, N, c, p):
     """The tensor-core contraction has two tilings for c <= 64: tiles of 256 positions,
     one contiguous range of the (worker, tile) list per CTA (ranges cross worker
     boundaries in these shapes) with one or two MMA issuers per half, and tiles of 128
-    positions per worker.  All must match the oracle, and each other bit for bit (same
-    products in the same order)."""
+    positions per worker; and two forms of the epilogue (all eight warps on every tile, or a
+    group of four warps per tile parity).  All must match the oracle, and each other bit for
+    bit (same products in the same order)."""
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(100 * N + c))
     g = _inputs().gradients_numpy(N, c * p, "normal", seed=8)
     ora = run_oracle(des.U, des.R, g, 0.25)
     outs = []
     try:
-        for variant in (0, 1, 2, 3):
+        for variant, epi in ((0, 0), (1, 1), (1, 2), (2, 1), (2, 2), (3, 1), (3, 2)):
             assert cerar_mod.cerar_set_tuning("tc_variant", variant) == 0
+            assert cerar_mod.cerar_set_tuning("tc_epi", epi) == 0
             plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
             plan.set_kernel_mode(cerar_mod.KERNEL_TC)
             res = run_library(plan, g, 0.25)
@@ -146,6 +148,7 @@ def test_tensor_core_tile_variants(cerar_mod, N, c, p):
             outs.append(res)
     finally:
         cerar_mod.cerar_set_tuning("tc_variant", 0)
+        cerar_mod.cerar_set_tuning("tc_epi", 0)
     for other in outs[1:]:
         assert np.array_equal(outs[0]["Delta"], other["Delta"])
         assert np.array_equal(outs[0]["out"], other["out"])
@@ -466,12 +469,14 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
             c = max(N, int(rng.choice([32, 36, 40, 48, 56, 64, 72, 96, 128])))
             p = int(rng.choice([4, 128, 132, 256, 260, 1028, 4104, 20000, 65540]))
             variant = int(rng.choice([0, 0, 1, 2, 3]))
+            epi = int(rng.choice([0, 1, 2]))
             d = c * p
             des = Dz.custom_orthogonal(N, c, np.random.default_rng(trial))
             g = torch.randn(N * d, device="cuda")
             outs = {}
             for mode, v in ((cerar_mod.KERNEL_TC, variant), (cerar_mod.KERNEL_STAGED, 0)):
                 cerar_mod.cerar_set_tuning("tc_variant", v)
+                cerar_mod.cerar_set_tuning("tc_epi", epi)
                 plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
                 plan.set_kernel_mode(mode)
                 ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
@@ -483,10 +488,11 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
                 outs[mode] = out
                 plan.destroy()
             a, b = outs[cerar_mod.KERNEL_TC], outs[cerar_mod.KERNEL_STAGED]
-            assert bool(torch.isfinite(a).all()), (N, c, p, variant)
-            assert float((a - b).norm() / b.norm()) < 3e-6, (N, c, p, variant)
+            assert bool(torch.isfinite(a).all()), (N, c, p, variant, epi)
+            assert float((a - b).norm() / b.norm()) < 3e-6, (N, c, p, variant, epi)
     finally:
         cerar_mod.cerar_set_tuning("tc_variant", 0)
+        cerar_mod.cerar_set_tuning("tc_epi", 0)
 
 
 @pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (3, 5, 1031), (16, 16, 1028), (2, 2, 4), (5, 7, 3),
