@@ -416,6 +416,8 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "tc_epi"                        epilogue of the tensor-core kernels: 1 = a group of four warps
  *                                   per tile parity, 2 = all eight warps on every tile (default:
  *                                   chosen by shape)
+ *   "round_split"                   ring round with few positions: 1 = never, 2 = always one thread per
+ *                                   group of 4 workers (default: where the plain grid has at most 148 blocks)
  *   "ring_wait_ms"                  limit of the waits of the fused ring rounds (default 2000)
  *   "ring_tile"                     positions per tile of the fused ring rounds (a multiple of 4;
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters

@@ -306,6 +306,51 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
     round_body<VT, WG>(reinterpret_cast<VT*>(a.ws) + v, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, a.k);
 }
 
+// The same round for few positions (the grid above would leave SMs idle and every thread with N / 4
+// dependent groups of loads): thread (v, q) takes workers 4q .. 4q+3 of position vector v, the
+// 256 / ceil(N/4) vectors of a block are contiguous.  The slot a message lands in is the cancel
+// operand of the worker it belongs to, which another thread of the same block reads: all loads,
+// one block barrier, then all stores.  Same operations in the same order per element as round_body.
+__global__ void __launch_bounds__(256) round_split_kernel(const RoundArgs a, int groups) {
+    const int64_t nv = a.p / 4;
+    const int pvb = blockDim.x / groups;                       // position vectors per block
+    const int64_t blk = a.reverse ? (int64_t)gridDim.x - 1 - blockIdx.x : (int64_t)blockIdx.x;
+    const int q = threadIdx.x / pvb;
+    const int64_t v = blk * pvb + (threadIdx.x - q * pvb);
+    const int N = a.N, c = a.c, k = a.k;
+    const bool has_prev = k >= 2, has_cancel = (k - 1) >= N, has_add = k <= c;
+    const int64_t wstride = (int64_t)(c + N) * nv;
+    const int64_t off_prev = (int64_t)(k - 2) * nv, off_land = (int64_t)(k - 1) * nv, off_add = (int64_t)(N - 1 + k) * nv;
+    float4* base = reinterpret_cast<float4*>(a.ws) + v;
+    const bool active = v < nv && q < groups;
+    float4 x[4];
+    grid_dependency_wait();
+    if (active) {
+        float4 y[4], dc[4], da[4];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int i = 4 * q + g;
+            y[g] = dc[g] = da[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < N) {
+                const float4* wb = base + (int64_t)i * wstride;
+                if (has_prev) y[g] = wb[off_prev];
+                if (has_cancel) dc[g] = wb[off_land];
+                if (has_add) da[g] = wb[off_add];
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < 4; ++g) x[g] = combine(y[g], dc[g], da[g]);
+    }
+    __syncthreads();
+    if (active) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int i = 4 * q + g;
+            if (i < N) base[(int64_t)((i + 1 == N) ? 0 : i + 1) * wstride + off_land] = x[g];
+        }
+    }
+}
+
 // Rounds k .. k_last in one launch, one THREAD per position vector: the thread owns its positions
 // for all N workers, and a round touches nothing else, so it simply runs the rounds one after the
 // other (its own stores are visible to its own later loads).  Latency-bound (L dependent rounds
@@ -461,6 +506,7 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 }  // namespace
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
+int g_tune_round_split = 0;
 int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
     g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0, g_tune_rounds_multi_form = 0, g_tune_rounds_coop_shape = 0, g_tune_rounds_hints = 0;
 
@@ -561,6 +607,17 @@ cudaError_t launch_round(const RoundArgs& a_in, cudaStream_t s, uint64_t* launch
     if (a.p % 4 == 0 && aligned16(a.ws)) {
         const int64_t nv = a.p / 4;
         const unsigned blocks = (unsigned)((nv + threads - 1) / threads);
+        const int groups = (a.N + 3) / 4;
+        // Fewer blocks than SMs and more than 4 workers: one thread per group of 4 workers.  Measured on B200
+        // over N = 8, 16, 32 and c = 8 .. 128: +10 .. +70 % up to p = 131072, -1 .. -8 % at p = 262144, 0 .. +7 %
+        // at p = 524288, nothing from 2^20 on (tuning: 1 = never, 2 = always)
+        const bool split = g_tune_round_split ? g_tune_round_split == 2 : (blocks <= 148);
+        if (split && groups >= 2 && groups <= 8) {
+            const int pvb = threads / groups;
+            e = launch_pdl(round_split_kernel, dim3((unsigned)((nv + pvb - 1) / pvb)), dim3(pvb * groups), 0, s, a, groups);
+            if (e == cudaSuccess && launches) ++*launches;
+            return e;
+        }
         // plain loads and stores, 4 workers in flight per thread: streaming cache hints (also with an L2
         // evict_last policy on the message stores: -1..-4 %), 512-thread blocks and 8 workers per group were
         // all measured and are not faster at d = 1.4e9

@@ -495,6 +495,45 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
         cerar_mod.cerar_set_tuning("tc_epi", 0)
 
 
+@pytest.mark.parametrize("N,c,p", [(5, 7, 4100), (8, 32, 4), (8, 8, 151556), (16, 20, 40004), (13, 16, 1028),
+                                   (32, 32, 260), (33, 34, 36), (6, 6, 37889)])
+def test_round_kernel_forms_leave_the_same_slots(cerar_mod, N, c, p):
+    """One ring round has two kernels for rows of whole 16-byte vectors: one thread per position vector
+    that walks all N workers, and (the default where there are few positions) one thread per group of
+    four workers with a block barrier between the loads and the stores.  Forced either way, every
+    round leaves the same slots bit for bit, and the observations match the oracle's rounds on the
+    device's own encoded vectors.  (N = 33 has too many groups for one block and p = 37889 has rows
+    that are not whole vectors: both settings then run the same kernel.)"""
+    import torch
+    d = c * p
+    L = c + N - 2
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(N * c))
+    g = torch.randn(N * d, device="cuda")
+    s = torch_stream()
+    res = []
+    try:
+        for setting in (1, 2, 0):
+            assert cerar_mod.cerar_set_tuning("round_split", setting) == 0
+            plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+            ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
+            plan.encode(g, d, ws, d, s)
+            Delta = ws.view(N, c + N, p)[:, N:, :].cpu().numpy().astype(np.float64)
+            for k in range(1, L + 1):
+                plan.ring_round(ws, d, k, s)
+            torch.cuda.synchronize()
+            plan.device_status(s)
+            res.append(ws.clone())
+    finally:
+        cerar_mod.cerar_set_tuning("round_split", 0)
+    for w in res[1:]:
+        assert torch.equal(torch.nan_to_num(w, nan=-1.0), torch.nan_to_num(res[0], nan=-1.0))
+    wsn = res[0].view(N, c + N, p).cpu().numpy()
+    Y_dev = np.concatenate([wsn[:, :L, :], wsn[:, L + 1:L + 2, :]], axis=1)
+    if p <= 4100:
+        Y_ref, _, _ = P.run_rounds([Delta[i].T for i in range(N)])
+        assert rel_l2(Y_dev, np.stack([Y_ref[i].T for i in range(N)])) < 2e-6
+
+
 @pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (3, 5, 1031), (16, 16, 1028), (2, 2, 4), (5, 7, 3),
                                    (8, 16, 40004), (32, 32, 36), (7, 9, 37889), (4, 8, 76036), (33, 33, 20), (32, 32, 76036), (20, 24, 76032)])
 def test_rounds_in_one_launch_equal_round_by_round(cerar_mod, N, c, p):
