@@ -414,8 +414,9 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *                                   positions for c <= 64); 2 / 3 = tiles of 256 with one /
  *                                   two MMA issuers per half
  *   "tc_epi"                        epilogue of the tensor-core kernels: 1 = a group of four warps
- *                                   per tile parity, 2 = all eight warps on every tile (default:
- *                                   chosen by shape)
+ *                                   per tile parity, 2 = all eight warps on every tile, 3 = one group
+ *                                   of four warps for all tiles (one output tile less in shared
+ *                                   memory), 4 = two groups (default: chosen by shape)
  *   "round_split"                   ring round with few positions: 1 = never, 2 = always one thread per
  *                                   group of 4 workers (default: where the plain grid has at most 148 blocks)
  *   "ring_wait_ms"                  limit of the waits of the fused ring rounds (default 2000)

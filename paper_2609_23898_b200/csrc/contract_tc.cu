@@ -65,7 +65,7 @@ struct PairParams {
     int Npad;          // J rounded up to 32
     int tmem_cols;     // power of two >= HALVES * (2*Npad + NAh*2*KC)
     int four_issuers;  // 1: every half has one issuer per accumulator (even / odd tiles)
-    int out_rows;        // output rows per TMA store (32; 16 with the group epilogue where that buys a stage)
+    int epi_groups;      // group epilogue: 2 = one group per tile parity, 1 = one group for all tiles (one output tile less)
     int group_epilogue;  // 1: each group of four epilogue warps works on tiles of its own (hardware barriers inside the group)
     int64_t tiles_per_worker;
     int64_t total_tiles;
@@ -90,11 +90,11 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     unsigned char* smem_al = smem_dyn + (smem_base - smem_u32(smem_dyn));
     const uint32_t b_bytes = (uint32_t)K_pad * Npad * 4u;            // one of B_hi / B_lo
     constexpr uint32_t chunk_bytes = (uint32_t)KC * TILE_W * 4u;
-    const uint32_t out_bytes = (uint32_t)tp.out_rows * TILE_W * 4u;
+    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * TILE_W * 4u;
     const uint32_t bhi_u32 = smem_base, blo_u32 = smem_base + b_bytes;
     const uint32_t raw_u32 = smem_base + 2u * b_bytes;
     const uint32_t out_u32 = raw_u32 + (uint32_t)stages * chunk_bytes;
-    const uint32_t bar_u32 = out_u32 + 2u * out_bytes;
+    const uint32_t bar_u32 = out_u32 + (uint32_t)tp.epi_groups * out_bytes;
     const uint32_t raw_full = bar_u32, raw_empty = raw_full + 8u * stages;
     // "A buffer filled": one barrier per (half, tile parity, buffer), so that each has ONE waiter
     // (the issuer of that half and parity) who sees all of its phases in order; a barrier that two
@@ -220,17 +220,18 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 // the group waits for its previous store.
                 const bool elected = ((warp - WARP_EPI0) & 3) == 0 && lane == 0;
                 auto run = [&](auto rows_c) {
-                    constexpr int R = decltype(rows_c)::value;          // output rows per block and store: 32 or 16
+                    constexpr int R = decltype(rows_c)::value;          // output rows per block and store
                     float* o = out_s + (size_t)g * (R * TILE_W) + pos;
                     const int nb_e = Npad / R;
                     bool pending = false, stop = false;
                     for (int64_t t = t_begin; t < t_end && !stop; ++t, ++tc) {
-                        if ((tc & 1u) != (uint32_t)g) continue;
+                        const uint32_t buf = tc & 1u;
+                        if (tp.epi_groups == 2 ? buf != (uint32_t)g : g != 0) continue;
                         const uint32_t aph = (tc >> 1) & 1u;
                         for (int nb = 0; nb < nb_e && !stop; ++nb) {
 #pragma unroll
                             for (int h = 0; h < HALVES; ++h) {
-                                const uint32_t acc = 2u * h + (uint32_t)g;
+                                const uint32_t acc = 2u * h + buf;
                                 if (nb == 0 && !failed && !warp_wait(acc_full + 8u * acc, aph)) failed = true;
                                 tc_fence_after();
                                 float v[R];
@@ -264,7 +265,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                         }
                     }
                 };
-                if (tp.out_rows == 16) run(std::integral_constant<int, 16>{}); else run(std::integral_constant<int, 32>{});
+                run(std::integral_constant<int, OUT_ROWS>{});
             } else
             for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
                 const uint32_t buf = tc & 1u, aph = (tc >> 1) & 1u;
@@ -409,7 +410,7 @@ cudaError_t launch_halves(int KC, const CUtensorMap& tin, const CUtensorMap& tou
 // possible, with at least 3 stages in the shared memory that the coefficient copies and the
 // output tiles leave and at least two A buffers per half in the tensor memory that the
 // accumulators leave.
-int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_rows = OUT_ROWS) {
+int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_tiles = 2) {
     const int tile_w = halves * HALF_M;
     tp->K_rows = a.K + a.skip_count;                        // decode: physical rows that are not part of Y
     tp->Npad = ((a.J + 31) / 32) * 32;
@@ -421,7 +422,7 @@ int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_rows
         if (g_tune_tc_kc && kc != g_tune_tc_kc) continue;
         if (halves * (2 * tp->Npad + 2 * 2 * kc) > 512) continue;
         const int kpad = ((tp->K_rows + kc - 1) / kc) * kc;
-        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp->Npad * 4 + 2 * (size_t)out_rows * tile_w * 4 + 512;
+        const size_t fixed_c = 1024 + 2 * (size_t)kpad * tp->Npad * 4 + out_tiles * (size_t)OUT_ROWS * tile_w * 4 + 512;
         const size_t stage_c = (size_t)kc * tile_w * 4;
         if (fixed_c + 3 * stage_c > budget) continue;
         int st = (int)((budget - fixed_c) / stage_c);
@@ -475,21 +476,24 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     // columns and more than 32 input rows (decode at c <= 32) all eight warps on every tile are 2-4 % ahead.
     tp.group_epilogue = (tp.Npad <= 32 && tp.K_rows > 32) ? 0 : 1;
     if (g_tune_tc_epi) tp.group_epilogue = g_tune_tc_epi == 2 ? 0 : 1;
-    tp.out_rows = OUT_ROWS;
-    if (tp.group_epilogue && g_tune_tc_epi == 3) {      // smaller output tiles, the stages chosen again with what they free
-        tp.out_rows = 16;
-        KC = choose_chunk(a, halves, &tp, 16);
+    // With 128 output columns the two coefficient copies leave 46-64 KB for the input stages: one group for
+    // all tiles needs one output tile less, which buys one or two stages (measured: encode +3 %, decode +7 % at
+    // c = 128, nothing at c = 112, -14 % for the encode at c = 80).  tc_epi 3 / 4 force one / two groups.
+    tp.epi_groups = (tp.group_epilogue && halves == 1 && tp.Npad > 96) ? 1 : 2;
+    if (tp.group_epilogue && g_tune_tc_epi >= 3) tp.epi_groups = g_tune_tc_epi == 3 ? 1 : 2;
+    if (tp.epi_groups == 1) {                           // the stages chosen again with what that frees
+        KC = choose_chunk(a, halves, &tp, 1);
         tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
         if (tp.NAh > 4) tp.NAh = 4;
     }
     tp.tmem_cols = 32;
     while (tp.tmem_cols < halves * (2 * tp.Npad + tp.NAh * 2 * KC)) tp.tmem_cols *= 2;
     const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * tile_w * 4 +
-                        2 * (size_t)tp.out_rows * tile_w * 4 + 512;
+                        (size_t)tp.epi_groups * OUT_ROWS * tile_w * 4 + 512;
 
     CUtensorMap tin, tout;
     if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, tile_w, KC)) return cudaErrorInvalidValue;
-    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, tile_w, tp.out_rows)) return cudaErrorInvalidValue;
+    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, tile_w, OUT_ROWS)) return cudaErrorInvalidValue;
 
     tp.tiles_per_worker = (a.p + tile_w - 1) / tile_w;
     tp.total_tiles = tp.tiles_per_worker * a.N;

@@ -130,15 +130,15 @@ def test_tensor_core_tile_variants(cerar_mod, N, c, p):
     """The tensor-core contraction has two tilings for c <= 64: tiles of 256 positions,
     one contiguous range of the (worker, tile) list per CTA (ranges cross worker
     boundaries in these shapes) with one or two MMA issuers per half, and tiles of 128
-    positions per worker; and two forms of the epilogue (all eight warps on every tile, or a
-    group of four warps per tile parity).  All must match the oracle, and each other bit for
+    positions per worker; and three forms of the epilogue (all eight warps on every tile, a
+    group of four warps per tile parity, one group for all tiles).  All must match the oracle, and each other bit for
     bit (same products in the same order)."""
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(100 * N + c))
     g = _inputs().gradients_numpy(N, c * p, "normal", seed=8)
     ora = run_oracle(des.U, des.R, g, 0.25)
     outs = []
     try:
-        for variant, epi in ((0, 0), (1, 1), (1, 2), (2, 1), (2, 2), (3, 1), (3, 2)):
+        for variant, epi in ((0, 0), (1, 1), (1, 2), (1, 3), (2, 1), (2, 2), (2, 3), (3, 4), (3, 2)):
             assert cerar_mod.cerar_set_tuning("tc_variant", variant) == 0
             assert cerar_mod.cerar_set_tuning("tc_epi", epi) == 0
             plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
@@ -469,7 +469,7 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
             c = max(N, int(rng.choice([32, 36, 40, 48, 56, 64, 72, 96, 128])))
             p = int(rng.choice([4, 128, 132, 256, 260, 1028, 4104, 20000, 65540]))
             variant = int(rng.choice([0, 0, 1, 2, 3]))
-            epi = int(rng.choice([0, 1, 2]))
+            epi = int(rng.choice([0, 1, 2, 3, 4]))
             d = c * p
             des = Dz.custom_orthogonal(N, c, np.random.default_rng(trial))
             g = torch.randn(N * d, device="cuda")
