@@ -60,7 +60,8 @@ typedef enum {
     CERAR_ERR_CUDA = 6,          /* a CUDA runtime call failed, or no device             */
     CERAR_ERR_NOMEM = 7,
     CERAR_ERR_TIMEOUT = 8,
-    CERAR_ERR_TOO_LARGE = 9      /* request exceeds the built-in workspace (see below)    */
+    CERAR_ERR_TOO_LARGE = 9,     /* request exceeds the built-in workspace (see below)    */
+    CERAR_ERR_BOUNDS = 10        /* checked build only: a kernel formed an address outside its buffer */
 } cerar_status_t;
 
 typedef enum {
@@ -388,6 +389,15 @@ cerar_status_t cerar_get_counters(const cerar_plan_t* plan, cerar_counters_t* ou
 /* Number of kernels this library has launched through this plan so far. */
 uint64_t       cerar_launch_count(const cerar_plan_t* plan);
 
+/* 1 if this library is the checked build (libcerar_checked.so, compiled with
+ * -DCERAR_BOUNDS_CHECK), 0 otherwise.  In the checked build the kernels of the in-HBM
+ * pipeline that use plain loads, stores and 1-D bulk copies (the FMA contractions, the ring
+ * rounds in all their forms) compare every address they form with the extent of its buffer;
+ * an address outside is not accessed, and the next cerar_device_status returns
+ * CERAR_ERR_BOUNDS.  It is the stand-in for a memory checker where none can be run; it
+ * costs bandwidth and is not what bench.py times.  The paper has no counterpart. */
+int            cerar_build_is_checked(void);
+
 /* Synchronises `stream` and reports CERAR_ERR_TIMEOUT if a kernel of this plan
  * gave up on one of its bounded device-side waits since the last check (the
  * results of that call are then invalid); CERAR_OK otherwise. */
@@ -419,6 +429,8 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *                                   memory), 4 = two groups (default: chosen by shape)
  *   "round_split"                   ring round with few positions: 1 = never, 2 = always one thread per
  *                                   group of 4 workers (default: where the plain grid has at most 148 blocks)
+ *   "checked_shrink"                checked build, tests only: the extents that stores are checked
+ *                                   against end this many floats early (the buffers do not change)
  *   "ring_wait_ms"                  limit of the waits of the fused ring rounds (default 2000)
  *   "ring_tile"                     positions per tile of the fused ring rounds (a multiple of 4;
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters

@@ -18,7 +18,7 @@ VANDERMONDE, EPSILON, KAPPA = 0, 1, 2
 KERNEL_AUTO, KERNEL_REF, KERNEL_STAGED, KERNEL_TC = 0, 1, 2, 3
 
 STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "SINGULAR", 4: "NOT_CONVERGED",
-                5: "STATE", 6: "CUDA", 7: "NOMEM", 8: "TIMEOUT", 9: "TOO_LARGE"}
+                5: "STATE", 6: "CUDA", 7: "NOMEM", 8: "TIMEOUT", 9: "TOO_LARGE", 10: "BOUNDS"}
 
 
 class CerarError(RuntimeError):
@@ -48,9 +48,11 @@ class Counters(C.Structure):
 
 
 def _load() -> C.CDLL:
-    path = _build.LIB_PATH
-    if _build.is_stale():
-        path = _build.build()
+    # CERAR_LIBRARY=checked selects the build whose kernels check every address they form (tests)
+    checked = os.environ.get("CERAR_LIBRARY", "") == "checked"
+    path = _build.CHECKED_LIB_PATH if checked else _build.LIB_PATH
+    if _build.is_stale(path):
+        path = _build.build(checked=checked)
     if not os.path.exists(path):
         raise ImportError(f"{path} is missing and could not be built")
     return C.CDLL(path)
@@ -112,6 +114,7 @@ lib.cerar_set_tuning.argtypes = [C.c_char_p, C.c_int]
 lib.cerar_status_string.argtypes = [C.c_int]
 lib.cerar_status_string.restype = C.c_char_p
 lib.cerar_last_error.restype = C.c_char_p
+lib.cerar_build_is_checked.restype = C.c_int
 
 
 def _check(status: int):

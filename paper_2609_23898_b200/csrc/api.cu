@@ -132,11 +132,20 @@ const char* cerar_status_string(cerar_status_t s) {
         case CERAR_ERR_NOMEM: return "out of memory";
         case CERAR_ERR_TIMEOUT: return "device-side wait timed out";
         case CERAR_ERR_TOO_LARGE: return "size beyond a fixed capacity";
+        case CERAR_ERR_BOUNDS: return "checked build: address outside its buffer";
     }
     return "unknown status";
 }
 
 const char* cerar_last_error(void) { return g_err.c_str(); }
+
+int cerar_build_is_checked(void) {
+#ifdef CERAR_BOUNDS_CHECK
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 // for the library's other translation units
 void cerar_internal_set_error(const char* msg) { g_err = msg ? msg : ""; }
@@ -321,6 +330,7 @@ cerar_status_t cerar_ring_round(cerar_plan_t* P, float* ws, int64_t d, int k, ce
     if (!P->encoded || d != P->cur_d) return fail(CERAR_ERR_STATE, "encode (with the same d) must come first");
     if (k != P->rounds_done + 1 || k > P->host.L) return fail(CERAR_ERR_STATE, "rounds must run in order 1..L");
     cerar::RoundArgs a{ws, p, P->host.N, P->host.c, k, 0};
+    a.status = P->d_status;
     cudaError_t e = cerar::launch_round(a, (cudaStream_t)stream, &P->launches);
     if (e != cudaSuccess) return cuda_fail(e, "round launch");
     P->rounds_done = k;
@@ -338,6 +348,7 @@ cerar_status_t cerar_ring_rounds(cerar_plan_t* P, float* ws, int64_t d, int k_fi
     if (k_first != P->rounds_done + 1 || k_last < k_first || k_last > P->host.L)
         return fail(CERAR_ERR_STATE, "rounds must run in order 1..L");
     cerar::RoundArgs a{ws, p, P->host.N, P->host.c, k_first, 0};
+    a.status = P->d_status;
     cudaError_t e = cerar::launch_rounds_multi(a, k_last, (cudaStream_t)stream, &P->launches);
     if (e != cudaSuccess) return cuda_fail(e, "rounds launch");
     P->rounds_done = k_last;
@@ -748,6 +759,8 @@ cerar_status_t cerar_device_status(cerar_plan_t* P, cerar_stream_t stream) {
     if (e != cudaSuccess) return cuda_fail(e, "status read");
     if (flag != 0) {
         cudaMemsetAsync(P->d_status, 0, sizeof(int), (cudaStream_t)stream);
+        if (flag == cerar::STATUS_BOUNDS)
+            return fail(CERAR_ERR_BOUNDS, "checked build: a kernel formed an address outside its buffer (the access was skipped)");
         return fail(CERAR_ERR_TIMEOUT, "a kernel gave up on a bounded wait");
     }
     return CERAR_OK;
@@ -780,6 +793,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "tc_min_c") cerar::g_tune_tc_min_c = value;
     else if (n == "tc_epi") cerar::g_tune_tc_epi = value;
     else if (n == "round_split") cerar::g_tune_round_split = value;
+    else if (n == "checked_shrink") cerar::g_tune_checked_shrink = value;
     else if (n == "rounds_one_launch_off") cerar::g_tune_rounds_one_launch_off = value;
     else if (n == "rounds_one_launch_mb") cerar::g_tune_rounds_one_launch_mb = value;
     else if (n == "rounds_multi_form") cerar::g_tune_rounds_multi_form = value;

@@ -29,11 +29,13 @@ __global__ void contract_ref_kernel(const ContractArgs a) {
     const float* cf = a.coef + (size_t)w * a.K * a.J;
     for (int k = 0; k < a.K; ++k) {
         const int row = (k < a.skip_row) ? k : k + a.skip_count;
-        const float x = in[(int64_t)row * a.in_rstride];
+        float x = 0.f;
+        if (CERAR_RANGE_OK(in + (int64_t)row * a.in_rstride, 4, a.in_range, a.status)) x = in[(int64_t)row * a.in_rstride];
         for (int j = 0; j < a.J; ++j) acc[j] = fmaf(cf[(size_t)k * a.J + j], x, acc[j]);
     }
     float* out = a.out + (int64_t)w * a.out_wstride + q;
-    for (int j = 0; j < a.J; ++j) out[(int64_t)j * a.out_rstride] = acc[j] * a.scale;
+    for (int j = 0; j < a.J; ++j)
+        if (CERAR_RANGE_OK(out + (int64_t)j * a.out_rstride, 4, a.out_range, a.status)) out[(int64_t)j * a.out_rstride] = acc[j] * a.scale;
 }
 
 // ------------------------------------------------------------------ tiled contraction, any alignment
@@ -63,7 +65,8 @@ __global__ void __launch_bounds__(256) contract_tile_kernel(const ContractArgs a
         const float* in = a.in + (int64_t)w * a.in_wstride + q;
         for (int k = 0; k < a.K; ++k) {
             const int row = (k < a.skip_row) ? k : k + a.skip_count;
-            in_s[(size_t)k * TP + threadIdx.x] = in[(int64_t)row * a.in_rstride];
+            in_s[(size_t)k * TP + threadIdx.x] =
+                CERAR_RANGE_OK(in + (int64_t)row * a.in_rstride, 4, a.in_range, a.status) ? in[(int64_t)row * a.in_rstride] : 0.f;
         }
     }
     __syncthreads();
@@ -84,7 +87,8 @@ __global__ void __launch_bounds__(256) contract_tile_kernel(const ContractArgs a
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j)
-            if (jc + j < a.J) out[(int64_t)(jc + j) * a.out_rstride] = acc[j] * a.scale;
+            if (jc + j < a.J && CERAR_RANGE_OK(out + (int64_t)(jc + j) * a.out_rstride, 4, a.out_range, a.status))
+                out[(int64_t)(jc + j) * a.out_rstride] = acc[j] * a.scale;
     }
 }
 
@@ -157,8 +161,11 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                 for (int r = lane; r < kcount; r += 32) {
                     const int k = k0 + r;
                     const int row = (k < a.skip_row) ? k : k + a.skip_count;
-                    bulk_load(stage0 + s * stage_bytes + (uint32_t)r * tile_p * 4u,
-                              in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, full0 + 8u * s);
+                    // (checked build: a copy that is skipped leaves its bytes outstanding, so the consumers' wait
+                    // runs out and the launch ends with both codes' worth of evidence in the status word)
+                    if (CERAR_RANGE_OK(in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, a.in_range, a.status))
+                        bulk_load(stage0 + s * stage_bytes + (uint32_t)r * tile_p * 4u,
+                                  in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, full0 + 8u * s);
                 }
             }
         }
@@ -225,7 +232,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                     float* orow = out_w + (int64_t)jj * a.out_rstride + q0;
 #pragma unroll
                     for (int v = 0; v < PV; ++v)
-                        if (pos[v] < valid) {
+                        if (pos[v] < valid && CERAR_RANGE_OK(orow + pos[v], 16, a.out_range, a.status)) {
                             float4 o;
                             o.x = acc[j][v * 4 + 0] * a.scale;
                             o.y = acc[j][v * 4 + 1] * a.scale;
@@ -259,12 +266,12 @@ __device__ __forceinline__ float4 combine(float4 y, float4 dc, float4 da) {
 
 // One round k for the position vector at `base` (all N workers), as described above.
 template <typename VT, int WG>
-__device__ __forceinline__ void round_body(VT* base, int64_t pv, int64_t wstride, int N, int c, int k) {
+__device__ __forceinline__ void round_body(VT* base, int64_t pv, int64_t wstride, int N, int c, int k, Range range, int* status) {
     const bool has_prev = k >= 2, has_cancel = (k - 1) >= N, has_add = k <= c;
     const int64_t off_prev = (int64_t)(k - 2) * pv, off_land = (int64_t)(k - 1) * pv,
                   off_add = (int64_t)(N - 1 + k) * pv;
     VT carry = vzero<VT>();
-    if (has_cancel) carry = base[off_land];                   // worker 0's delta_{0,k-N}
+    if (has_cancel && CERAR_RANGE_OK(base + off_land, sizeof(VT), range, status)) carry = base[off_land];   // worker 0's delta_{0,k-N}
     for (int i0 = N - 1; i0 >= 0; i0 -= WG) {
         VT y[WG], dc[WG], da[WG];
 #pragma unroll
@@ -273,9 +280,9 @@ __device__ __forceinline__ void round_body(VT* base, int64_t pv, int64_t wstride
             y[g] = dc[g] = da[g] = vzero<VT>();
             if (i >= 0) {
                 const VT* wb = base + (int64_t)i * wstride;
-                if (has_prev) y[g] = wb[off_prev];
-                if (has_cancel) dc[g] = (i == 0) ? carry : wb[off_land];
-                if (has_add) da[g] = wb[off_add];
+                if (has_prev && CERAR_RANGE_OK(wb + off_prev, sizeof(VT), range, status)) y[g] = wb[off_prev];
+                if (has_cancel) dc[g] = (i == 0) ? carry : CERAR_RANGE_OK(wb + off_land, sizeof(VT), range, status) ? wb[off_land] : vzero<VT>();
+                if (has_add && CERAR_RANGE_OK(wb + off_add, sizeof(VT), range, status)) da[g] = wb[off_add];
             }
         }
 #pragma unroll
@@ -283,7 +290,8 @@ __device__ __forceinline__ void round_body(VT* base, int64_t pv, int64_t wstride
             const int i = i0 - g;
             if (i >= 0) {
                 const int dst = (i + 1 == N) ? 0 : i + 1;
-                base[(int64_t)dst * wstride + off_land] = combine(y[g], dc[g], da[g]);
+                if (CERAR_RANGE_OK(base + (int64_t)dst * wstride + off_land, sizeof(VT), range, status))
+                    base[(int64_t)dst * wstride + off_land] = combine(y[g], dc[g], da[g]);
             }
         }
     }
@@ -303,7 +311,7 @@ __global__ void __launch_bounds__(256) round_kernel(const RoundArgs a) {
     grid_dependency_wait();
     if (v >= nv) return;
     const int64_t pv = a.p / VW;                               // row pitch in vectors
-    round_body<VT, WG>(reinterpret_cast<VT*>(a.ws) + v, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, a.k);
+    round_body<VT, WG>(reinterpret_cast<VT*>(a.ws) + v, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, a.k, a.range, a.status);
 }
 
 // The same round for few positions (the grid above would leave SMs idle and every thread with N / 4
@@ -333,9 +341,9 @@ __global__ void __launch_bounds__(256) round_split_kernel(const RoundArgs a, int
             y[g] = dc[g] = da[g] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (i < N) {
                 const float4* wb = base + (int64_t)i * wstride;
-                if (has_prev) y[g] = wb[off_prev];
-                if (has_cancel) dc[g] = wb[off_land];
-                if (has_add) da[g] = wb[off_add];
+                if (has_prev && CERAR_RANGE_OK(wb + off_prev, 16, a.range, a.status)) y[g] = wb[off_prev];
+                if (has_cancel && CERAR_RANGE_OK(wb + off_land, 16, a.range, a.status)) dc[g] = wb[off_land];
+                if (has_add && CERAR_RANGE_OK(wb + off_add, 16, a.range, a.status)) da[g] = wb[off_add];
             }
         }
 #pragma unroll
@@ -346,7 +354,8 @@ __global__ void __launch_bounds__(256) round_split_kernel(const RoundArgs a, int
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
             const int i = 4 * q + g;
-            if (i < N) base[(int64_t)((i + 1 == N) ? 0 : i + 1) * wstride + off_land] = x[g];
+            float4* dstp = base + (int64_t)((i + 1 == N) ? 0 : i + 1) * wstride + off_land;
+            if (i < N && CERAR_RANGE_OK(dstp, 16, a.range, a.status)) *dstp = x[g];
         }
     }
 }
@@ -366,7 +375,7 @@ __global__ void __launch_bounds__(256) rounds_multi_kernel(const RoundArgs a, in
     if (v >= nv) return;
     const int64_t pv = a.p / VW;
     VT* base = reinterpret_cast<VT*>(a.ws) + v;
-    for (int k = a.k; k <= k_last; ++k) round_body<VT, WG>(base, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, k);
+    for (int k = a.k; k <= k_last; ++k) round_body<VT, WG>(base, pv, (int64_t)(a.c + a.N) * pv, a.N, a.c, k, a.range, a.status);
 }
 
 // The same rounds k .. k_last in one launch with one WARP per worker: a block of N warps owns 32 PV
@@ -429,14 +438,14 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
 #pragma unroll
     for (int j = 0; j < PV; ++j) {
         y[j] = vzero<VT>();
-        if (live[j] && k >= 2) y[j] = own[(int64_t)(k - 2) * pv + 32 * j];
+        if (live[j] && k >= 2 && CERAR_RANGE_OK(own + (int64_t)(k - 2) * pv + 32 * j, sizeof(VT), a.range, a.status)) y[j] = own[(int64_t)(k - 2) * pv + 32 * j];
 #pragma unroll
         for (int t = 0; t < DIST; ++t) {
             const int kt = k + t;
             da[t][j] = dc[t][j] = vzero<VT>();
             if (live[j] && kt <= k_last) {
-                if (kt <= c) da[t][j] = hints ? ld_keep(own + (int64_t)(N - 1 + kt) * pv + 32 * j, pol) : own[(int64_t)(N - 1 + kt) * pv + 32 * j];
-                if (kt - 1 >= N) dc[t][j] = hints ? ld_last_use(own + (int64_t)(kt - 1) * pv + 32 * j) : own[(int64_t)(kt - 1) * pv + 32 * j];
+                if (kt <= c && CERAR_RANGE_OK(own + (int64_t)(N - 1 + kt) * pv + 32 * j, sizeof(VT), a.range, a.status)) da[t][j] = hints ? ld_keep(own + (int64_t)(N - 1 + kt) * pv + 32 * j, pol) : own[(int64_t)(N - 1 + kt) * pv + 32 * j];
+                if (kt - 1 >= N && CERAR_RANGE_OK(own + (int64_t)(kt - 1) * pv + 32 * j, sizeof(VT), a.range, a.status)) dc[t][j] = hints ? ld_last_use(own + (int64_t)(kt - 1) * pv + 32 * j) : own[(int64_t)(kt - 1) * pv + 32 * j];
             }
         }
     }
@@ -446,7 +455,9 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
 #pragma unroll
         for (int j = 0; j < PV; ++j) {
             const VT x = combine(y[j], dc[0][j], da[0][j]);
-            if (live[j]) { if (hints) st_stream(nxt + (int64_t)(k - 1) * pv + 32 * j, x); else nxt[(int64_t)(k - 1) * pv + 32 * j] = x; }
+            if (live[j] && CERAR_RANGE_OK(nxt + (int64_t)(k - 1) * pv + 32 * j, sizeof(VT), a.range, a.status)) {
+                if (hints) st_stream(nxt + (int64_t)(k - 1) * pv + 32 * j, x); else nxt[(int64_t)(k - 1) * pv + 32 * j] = x;
+            }
             hb[(dst * PV + j) * 32 + lane] = x;
         }
         // shift the operand queue and fetch round k + DIST (its slots are not written before that round)
@@ -457,8 +468,8 @@ __global__ void __launch_bounds__(MAXT) rounds_coop_kernel(const RoundArgs a, in
             for (int t = 0; t + 1 < DIST; ++t) { da[t][j] = da[t + 1][j]; dc[t][j] = dc[t + 1][j]; }
             da[DIST - 1][j] = dc[DIST - 1][j] = vzero<VT>();
             if (live[j] && kn <= k_last) {
-                if (kn <= c) da[DIST - 1][j] = hints ? ld_keep(own + (int64_t)(N - 1 + kn) * pv + 32 * j, pol) : own[(int64_t)(N - 1 + kn) * pv + 32 * j];
-                if (kn - 1 >= N) dc[DIST - 1][j] = hints ? ld_last_use(own + (int64_t)(kn - 1) * pv + 32 * j) : own[(int64_t)(kn - 1) * pv + 32 * j];
+                if (kn <= c && CERAR_RANGE_OK(own + (int64_t)(N - 1 + kn) * pv + 32 * j, sizeof(VT), a.range, a.status)) da[DIST - 1][j] = hints ? ld_keep(own + (int64_t)(N - 1 + kn) * pv + 32 * j, pol) : own[(int64_t)(N - 1 + kn) * pv + 32 * j];
+                if (kn - 1 >= N && CERAR_RANGE_OK(own + (int64_t)(kn - 1) * pv + 32 * j, sizeof(VT), a.range, a.status)) dc[DIST - 1][j] = hints ? ld_last_use(own + (int64_t)(kn - 1) * pv + 32 * j) : own[(int64_t)(kn - 1) * pv + 32 * j];
             }
         }
         __syncthreads();
@@ -507,11 +518,15 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
 int g_tune_round_split = 0;
+int g_tune_checked_shrink = 0;   // checked build, tests only: the extents that stores are checked against end this many floats early
 int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
     g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0, g_tune_rounds_multi_form = 0, g_tune_rounds_coop_shape = 0, g_tune_rounds_hints = 0;
 
 cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t s, uint64_t* launches) {
     if (a.p <= 0 || a.N <= 0) return cudaSuccess;
+    a.in_range = Range{a.in, a.in + (int64_t)(a.N - 1) * a.in_wstride + (int64_t)(a.K + a.skip_count - 1) * a.in_rstride + a.p};
+    a.out_range = Range{a.out, a.out + (int64_t)(a.N - 1) * a.out_wstride + (int64_t)(a.J - 1) * a.out_rstride + a.p -
+                                   g_tune_checked_shrink};
     bool can_stage = (a.p % 4 == 0) && aligned16(a.in) && aligned16(a.out) && (a.in_wstride % 4 == 0) &&
                      (a.out_wstride % 4 == 0) && (a.in_rstride % 4 == 0) && (a.out_rstride % 4 == 0);
     if (mode == KERNEL_TC && !tc_eligible(a)) return cudaErrorInvalidValue;
@@ -601,6 +616,7 @@ cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_n
 cudaError_t launch_round(const RoundArgs& a_in, cudaStream_t s, uint64_t* launches) {
     if (a_in.p <= 0) return cudaSuccess;
     RoundArgs a = a_in;
+    a.range = Range{a.ws, a.ws + (int64_t)a.N * (a.c + a.N) * a.p - g_tune_checked_shrink};
     a.reverse = (a.k % 2 == 0 && !g_tune_serpentine_off) ? 1 : 0;
     const int threads = 256;
     cudaError_t e;
@@ -631,6 +647,7 @@ cudaError_t launch_round(const RoundArgs& a_in, cudaStream_t s, uint64_t* launch
 
 cudaError_t launch_rounds_multi(const RoundArgs& a_in, int k_last, cudaStream_t s, uint64_t* launches) {
     RoundArgs a = a_in;
+    a.range = Range{a.ws, a.ws + (int64_t)a.N * (a.c + a.N) * a.p - g_tune_checked_shrink};
     // L2 residency hints (measured: +6..+13 % at N = 8, +1..+4 % at N = 16, -1..-4 % at N = 4, where the
     // delta to cancel is still in L2 anyway); tuning: 1 = off, 2 = on
     a.hints = g_tune_rounds_hints ? (g_tune_rounds_hints == 2) : (a.N >= 8);

@@ -5,6 +5,29 @@
 
 namespace cerar {
 
+// Checked build (-DCERAR_BOUNDS_CHECK, libcerar_checked.so): every address that the kernels of the in-HBM
+// pipeline form for a plain load, a plain store or a 1-D bulk copy is compared with the extent of
+// the buffer it belongs to.  An address outside is recorded in the plan's status word (STATUS_BOUNDS;
+// the first offender wins) and the access is skipped, so nothing faults; cerar_device_status then
+// reports CERAR_ERR_BOUNDS.  The release build compiles the checks away.  Tensor-map (TMA) copies need no
+// check of this kind: the hardware clips them at the extents in the map, which are the buffer's own.
+constexpr int STATUS_BOUNDS = 16;
+struct Range {            // [lo, hi) in floats
+    const float* lo;
+    const float* hi;
+};
+#ifdef CERAR_BOUNDS_CHECK
+__device__ __forceinline__ bool range_ok(const void* p, size_t bytes, Range r, int* status) {
+    const char* b = static_cast<const char*>(p);
+    if (b >= reinterpret_cast<const char*>(r.lo) && b + bytes <= reinterpret_cast<const char*>(r.hi)) return true;
+    atomicCAS(status, 0, STATUS_BOUNDS);
+    return false;
+}
+#define CERAR_RANGE_OK(p, bytes, r, status) ::cerar::range_ok((p), (bytes), (r), (status))
+#else
+#define CERAR_RANGE_OK(p, bytes, r, status) true
+#endif
+
 // A skinny contraction out[j][q] = scale * sum_k coef[k][j] * in[row(k)][q] over
 // positions q in [0, p), for N workers.  Encoding (Delta_i = G_i U_i) and
 // decoding (G_hat_i = Y_i R_i) are both of this form.
@@ -27,6 +50,7 @@ struct ContractArgs {
     int KC, stages, slabs, jgroups, tile_p;
     int tiles_per_worker;
     int64_t total_tiles;
+    Range in_range, out_range;   // extents of the two buffers (filled in by the launcher; read by the checked build)
 };
 
 struct RoundArgs {
@@ -35,6 +59,8 @@ struct RoundArgs {
     int N, c, k;            // round k in 1..L
     int reverse;            // round_kernel: 1 = blocks walk the positions downwards (set by the launcher)
     int hints;              // rounds_coop_kernel: 1 = L2 residency hints on the delta rows (set by the launcher)
+    int* status;            // device word of the plan
+    Range range;            // extent of the workspace (filled in by the launcher; read by the checked build)
 };
 
 // One worker's ring round in the one-worker-per-GPU layout ((c+N+1) x p per worker).
@@ -76,7 +102,7 @@ bool tc_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
 extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant,
-           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off, g_tune_serpentine_off, g_tune_tc_min_c, g_tune_tc_epi, g_tune_round_split,
+           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off, g_tune_serpentine_off, g_tune_tc_min_c, g_tune_tc_epi, g_tune_round_split, g_tune_checked_shrink,
            g_tune_rounds_one_launch_off, g_tune_rounds_one_launch_mb, g_tune_rounds_multi_form, g_tune_rounds_coop_shape, g_tune_rounds_hints;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
 // Rounds a.k .. k_last in one launch (for states that are cache-resident anyway).
