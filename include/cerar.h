@@ -392,7 +392,8 @@ uint64_t       cerar_launch_count(const cerar_plan_t* plan);
 /* 1 if this library is the checked build (libcerar_checked.so, compiled with
  * -DCERAR_BOUNDS_CHECK), 0 otherwise.  In the checked build the kernels of the in-HBM
  * pipeline that use plain loads, stores and 1-D bulk copies (the FMA contractions, the ring
- * rounds in all their forms) compare every address they form with the extent of its buffer;
+ * rounds in all their forms, the tensor-core contraction on rows that are not 16-byte
+ * aligned) compare every address they form with the extent of its buffer;
  * an address outside is not accessed, and the next cerar_device_status returns
  * CERAR_ERR_BOUNDS.  It is the stand-in for a memory checker where none can be run; it
  * costs bandwidth and is not what bench.py times.  The paper has no counterpart. */
@@ -436,7 +437,10 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters
  *   "pdl_off"                       1 = launch without programmatic stream serialization
  *   "serpentine_off"                1 = every ring round walks the positions upwards
- *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24)
+ *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24; 16 for
+ *                                   rows that do not start on 16-byte boundaries)
+ *   "tc_unaligned_off"              1 = rows that do not start on 16-byte boundaries never run on the
+ *                                   tensor-core kernel (they take the tiled plain-load kernel)
  *   "rounds_one_launch_off"         1 = cerar_allreduce_sim always launches round by round
  *   "rounds_one_launch_mb"          if set, cerar_allreduce_sim runs the rounds in one launch exactly
  *                                   for workspaces up to this many MB (default rule: see

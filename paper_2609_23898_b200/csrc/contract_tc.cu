@@ -41,6 +41,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <cstring>
 #include <type_traits>
 
 #include "kernels.cuh"
@@ -72,11 +73,18 @@ struct PairParams {
 };
 
 // shared memory (1024-aligned): B_hi | B_lo | raw stages | 2 output tiles | barriers | tmem slot
-template <int KC, int HALVES>
+template <int KC, int HALVES, bool UNAL>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_constant__ CUtensorMap tmap_out,
                    const __grid_constant__ ContractArgs a, const __grid_constant__ PairParams tp) {
     constexpr int TILE_W = HALVES * HALF_M;      // positions per tile
+    // UNAL: rows that do not start on 16-byte boundaries (p not a multiple of 4, or an unaligned buffer).
+    // Tensor-map copies cannot address them, so every row of a chunk comes in with a 1-D bulk copy of its
+    // own that starts at the 16-byte boundary below the row's first element; the row sits in shared memory
+    // with the same offset (0..3 floats) it has in global memory, which the splitter adds when it reads.
+    // Output rows are laid out with THEIR offsets, so that the 16-byte aligned middle of a row leaves with
+    // one bulk store and the up to three elements on either side with plain stores.
+    constexpr int PITCH = TILE_W + (UNAL ? 4 : 0);   // floats between rows of a stage and of an output tile
     extern __shared__ unsigned char smem_dyn[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int stages = tp.stages, Npad = tp.Npad, K_pad = tp.K_pad;
@@ -89,8 +97,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     unsigned char* smem_al = smem_dyn + (smem_base - smem_u32(smem_dyn));
     const uint32_t b_bytes = (uint32_t)K_pad * Npad * 4u;            // one of B_hi / B_lo
-    constexpr uint32_t chunk_bytes = (uint32_t)KC * TILE_W * 4u;
-    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * TILE_W * 4u;
+    constexpr uint32_t chunk_bytes = (uint32_t)KC * PITCH * 4u;
+    constexpr uint32_t out_bytes = (uint32_t)OUT_ROWS * PITCH * 4u;
     const uint32_t bhi_u32 = smem_base, blo_u32 = smem_base + b_bytes;
     const uint32_t raw_u32 = smem_base + 2u * b_bytes;
     const uint32_t out_u32 = raw_u32 + (uint32_t)stages * chunk_bytes;
@@ -153,7 +161,41 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             // a wait of this warp ran out in an earlier segment: only keep the CTA barriers company
         } else if (warp == 0) {
             // ================= producer
-            if (lane == 0) {
+            if constexpr (UNAL) {
+                // one bulk copy per row, issued by the lanes in parallel; lane 0 announces their total first
+                const uintptr_t in_w = reinterpret_cast<uintptr_t>(a.in + (int64_t)w * a.in_wstride);
+                for (int64_t t = t_begin; t < t_end && !failed; ++t) {
+                    const int64_t q0 = t * TILE_W;
+                    const uint32_t valid = (uint32_t)(a.p - q0 < TILE_W ? a.p - q0 : TILE_W);
+                    for (int kc = 0; kc < nkc; ++kc, ++it) {
+                        const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                        if (!warp_wait(raw_empty + 8u * s, ph ^ 1u)) { failed = true; break; }
+                        uint32_t bytes[(KC + 31) / 32];
+                        uintptr_t src[(KC + 31) / 32];
+                        uint32_t total = 0;
+#pragma unroll
+                        for (int rr = 0; rr < (KC + 31) / 32; ++rr) {
+                            const int r = rr * 32 + lane, row = kc * KC + r;
+                            bytes[rr] = 0;
+                            if (r < KC && row < tp.K_rows) {
+                                const uintptr_t first = in_w + ((uintptr_t)row * (uintptr_t)a.in_rstride + (uintptr_t)q0) * 4u;
+                                src[rr] = first & ~(uintptr_t)15;
+                                bytes[rr] = (uint32_t)((first - src[rr]) + valid * 4u + 15u) & ~15u;
+                                if (!CERAR_RANGE_OK(reinterpret_cast<const void*>(first), valid * 4u, a.in_range, a.status)) bytes[rr] = 0;
+                            }
+                            total += bytes[rr];
+                        }
+                        total = __reduce_add_sync(0xffffffffu, total);
+                        if (lane == 0) mbar_arrive_expect_tx(raw_full + 8u * s, total);
+                        __syncwarp();
+#pragma unroll
+                        for (int rr = 0; rr < (KC + 31) / 32; ++rr)
+                            if (bytes[rr])
+                                bulk_load(raw_u32 + s * chunk_bytes + (uint32_t)(rr * 32 + lane) * (PITCH * 4u),
+                                          reinterpret_cast<const void*>(src[rr]), bytes[rr], raw_full + 8u * s);
+                    }
+                }
+            } else if (lane == 0) {
                 for (int64_t t = t_begin; t < t_end && !failed; ++t) {
                     const int q0 = (int)(t * TILE_W);
                     for (int kc = 0; kc < nkc; ++kc, ++it) {
@@ -221,7 +263,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                 const bool elected = ((warp - WARP_EPI0) & 3) == 0 && lane == 0;
                 auto run = [&](auto rows_c) {
                     constexpr int R = decltype(rows_c)::value;          // output rows per block and store
-                    float* o = out_s + (size_t)g * (R * TILE_W) + pos;
+                    float* o = out_s + (size_t)g * (R * PITCH) + pos;
                     const int nb_e = Npad / R;
                     bool pending = false, stop = false;
                     for (int64_t t = t_begin; t < t_end && !stop; ++t, ++tc) {
@@ -248,17 +290,48 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                                     if (lane == 0) mbar_arrive(acc_empty + 8u * acc);
                                 }
                                 if (h == 0) {
-                                    if (elected && pending) bulk_wait_read_0();      // the group's tile is free again
+                                    if ((UNAL ? ((warp - WARP_EPI0) & 3) == 0 : elected) && pending) bulk_wait_read_0();   // the group's tile is free again
                                     if (bar_red_or(1u + (uint32_t)g, 128u, failed)) { failed = true; stop = true; break; }
                                 }
+                                if constexpr (UNAL) {
+                                    const uint32_t o0 = (uint32_t)((reinterpret_cast<uintptr_t>(a.out + (int64_t)w * a.out_wstride) >> 2) +
+                                                                   (uint64_t)(t * TILE_W) + (uint64_t)(nb * R) * (uint64_t)a.out_rstride);
+                                    const uint32_t os = (uint32_t)(a.out_rstride & 3);
 #pragma unroll
-                                for (int j = 0; j < R; ++j) o[j * TILE_W + h * HALF_M] = v[j] * a.scale;
+                                    for (int j = 0; j < R; ++j) o[j * PITCH + h * HALF_M + (int)((o0 + (uint32_t)j * os) & 3u)] = v[j] * a.scale;
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < R; ++j) o[j * PITCH + h * HALF_M] = v[j] * a.scale;
+                                }
                             }
                             if (stop) break;
                             fence_proxy_async_smem();
                             bar_sync(1u + (uint32_t)g, 128u);
-                            if (elected) {
-                                tma_store_3d(&tmap_out, (int)(t * TILE_W), nb * R, w, out_u32 + (uint32_t)g * (uint32_t)(R * TILE_W * 4));
+                            if constexpr (UNAL) {
+                                // lane j of the group's first warp stores row j: the aligned middle with a bulk copy, the rest plainly
+                                if (((warp - WARP_EPI0) & 3) == 0) {
+                                    const int j = nb * R + lane;
+                                    const int64_t q0 = t * TILE_W;
+                                    const int valid = (int)(a.p - q0 < TILE_W ? a.p - q0 : TILE_W);
+                                    if (lane < R && j < a.J) {
+                                        float* dst = a.out + (int64_t)w * a.out_wstride + (int64_t)j * a.out_rstride + q0;
+                                        const int sh = (int)((reinterpret_cast<uintptr_t>(dst) >> 2) & 3u);
+                                        const float* srow = out_s + (size_t)g * (R * PITCH) + (size_t)lane * PITCH + sh;   // element 0 of the row
+                                        int head = (4 - sh) & 3;
+                                        if (head > valid) head = valid;
+                                        const int body = (valid - head) & ~3;
+                                        if (CERAR_RANGE_OK(dst, (size_t)valid * 4u, a.out_range, a.status)) {
+                                            if (body > 0)
+                                                bulk_store(dst + head, smem_u32(srow + head), (uint32_t)body * 4u);
+                                            for (int e = 0; e < head; ++e) dst[e] = srow[e];
+                                            for (int e = head + body; e < valid; ++e) dst[e] = srow[e];
+                                        }
+                                    }
+                                    bulk_commit();
+                                    pending = true;
+                                }
+                            } else if (elected) {
+                                tma_store_3d(&tmap_out, (int)(t * TILE_W), nb * R, w, out_u32 + (uint32_t)g * (uint32_t)(R * PITCH * 4));
                                 bulk_commit();
                                 pending = true;
                             }
@@ -322,7 +395,14 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
                     const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
                     const uint32_t abi = seq % NAh, pa = (seq / NAh) & 1u;
                     if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
-                    const float* col = raw_s + (size_t)s * (KC * TILE_W) + (size_t)r0 * TILE_W + pos;
+                    const float* col = raw_s + (size_t)s * (KC * PITCH) + (size_t)r0 * PITCH + pos;
+                    // UNAL: offset (in floats, mod 4) of the first element of row r0 of this chunk, and its step per row
+                    uint32_t sh0 = 0, shs = 0;
+                    if constexpr (UNAL) {
+                        shs = (uint32_t)(a.in_rstride & 3);
+                        sh0 = (uint32_t)((reinterpret_cast<uintptr_t>(a.in + (int64_t)w * a.in_wstride) >> 2) + (uint64_t)(t * TILE_W) +
+                                         (uint64_t)(kc * KC + r0) * (uint64_t)a.in_rstride);
+                    }
                     // rows of this chunk that some product reads (the last chunk may be short): rounded up
                     // to the k-step, rows beyond the data are zero (TMA fill)
                     const int rows_left = tp.K_rows - kc * KC;
@@ -333,8 +413,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
 #pragma unroll
                         for (int k = 0; k < KG; ++k) {
                             hi[k] = lo[k] = 0u;
-                            if ((k & ~3) < kuse) {
-                                const float x = col[k * TILE_W + h * HALF_M];
+                            if ((k & ~3) < kuse && (!UNAL || r0 + k < rows_left)) {     // (a tensor-map load fills rows beyond the data with zeros)
+                                const float x = col[k * PITCH + h * HALF_M + (UNAL ? (int)((sh0 + (uint32_t)k * shs) & 3u) : 0)];
                                 hi[k] = tf32_bits(x);
                                 lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
                             }
@@ -366,7 +446,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
         tc_fence_after();
     }
 
-    if ((warp == WARP_EPI0 || warp == WARP_EPI0 + 4) && lane == 0) bulk_wait_all();   // all output has left shared memory and is written
+    if ((warp == WARP_EPI0 || warp == WARP_EPI0 + 4) && (UNAL || lane == 0)) bulk_wait_all();   // all output has left shared memory and is written
     if (failed) {
         if (lane == 0) atomicExch(a.status, 2);
         const unsigned long long t0 = global_ns();
@@ -384,10 +464,10 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     }
 }
 
-template <int KC, int HALVES>
+template <int KC, int HALVES, bool UNAL>
 cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a, const PairParams& tp,
                       size_t smem, int grid, cudaStream_t s) {
-    auto kern = contract_tc_kernel<KC, HALVES>;
+    auto kern = contract_tc_kernel<KC, HALVES, UNAL>;
     {   // per device and cheap: set on every launch rather than cached
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -395,14 +475,14 @@ cudaError_t launch_kc(const CUtensorMap& tin, const CUtensorMap& tout, const Con
     return launch_pdl(kern, dim3((unsigned)grid), dim3(NUM_THREADS), smem, s, tin, tout, a, tp);
 }
 
-template <int HALVES>
+template <int HALVES, bool UNAL>
 cudaError_t launch_halves(int KC, const CUtensorMap& tin, const CUtensorMap& tout, const ContractArgs& a,
                           const PairParams& tp, size_t smem, int grid, cudaStream_t s) {
     switch (KC) {
-        case 40: return launch_kc<40, HALVES>(tin, tout, a, tp, smem, grid, s);
-        case 32: return launch_kc<32, HALVES>(tin, tout, a, tp, smem, grid, s);
-        case 24: return launch_kc<24, HALVES>(tin, tout, a, tp, smem, grid, s);
-        default: return launch_kc<16, HALVES>(tin, tout, a, tp, smem, grid, s);
+        case 40: return launch_kc<40, HALVES, UNAL>(tin, tout, a, tp, smem, grid, s);
+        case 32: return launch_kc<32, HALVES, UNAL>(tin, tout, a, tp, smem, grid, s);
+        case 24: return launch_kc<24, HALVES, UNAL>(tin, tout, a, tp, smem, grid, s);
+        default: return launch_kc<16, HALVES, UNAL>(tin, tout, a, tp, smem, grid, s);
     }
 }
 
@@ -410,8 +490,8 @@ cudaError_t launch_halves(int KC, const CUtensorMap& tin, const CUtensorMap& tou
 // possible, with at least 3 stages in the shared memory that the coefficient copies and the
 // output tiles leave and at least two A buffers per half in the tensor memory that the
 // accumulators leave.
-int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_tiles = 2) {
-    const int tile_w = halves * HALF_M;
+int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_tiles = 2, bool unal = false) {
+    const int tile_w = halves * HALF_M + (unal ? 4 : 0);      // row pitch in shared memory
     tp->K_rows = a.K + a.skip_count;                        // decode: physical rows that are not part of Y
     tp->Npad = ((a.J + 31) / 32) * 32;
     const size_t budget = 227 * 1024 - 1024;
@@ -440,15 +520,28 @@ int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_tile
 
 }  // namespace
 
-int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_variant = 0, g_tune_tc_min_c = 0, g_tune_tc_epi = 0;
+int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_variant = 0, g_tune_tc_min_c = 0, g_tune_tc_epi = 0, g_tune_tc_unaligned_off = 0;
+
+// Rows that start on 16-byte boundaries everywhere: what tensor-map copies need.
+static bool rows_aligned(const ContractArgs& a) {
+    if (a.p % 4 != 0) return false;
+    if ((reinterpret_cast<uintptr_t>(a.in) & 15u) || (a.in_rstride % 4) || (a.in_wstride % 4)) return false;
+    if ((reinterpret_cast<uintptr_t>(a.out) & 15u) || (a.out_rstride % 4) || (a.out_wstride % 4)) return false;
+    return true;
+}
 
 bool tc_eligible(const ContractArgs& a) {
     // N = J padded to 32 (rows beyond J are clipped by the output map); measured against the FMA kernel
     // on B200: +40 % at c = 28, +5 % at c = 24, -15 % at c = 20.  Two coefficient copies must fit in smem.
-    if (a.J < (g_tune_tc_min_c > 0 ? g_tune_tc_min_c : 24) || a.J > 128) return false;
-    if (a.p % 4 != 0 || a.p >= (int64_t)1 << 31) return false;
-    if ((reinterpret_cast<uintptr_t>(a.in) & 15u) || (a.in_rstride % 4) || (a.in_wstride % 4)) return false;
-    if ((reinterpret_cast<uintptr_t>(a.out) & 15u) || (a.out_rstride % 4) || (a.out_wstride % 4)) return false;
+    // Rows that are not 16-byte aligned run the same kernel with per-row bulk copies (no tensor maps); the
+    // alternative there is the tiled plain-load kernel, so the tensor cores take over from a smaller c.
+    const bool aligned = rows_aligned(a);
+    // (measured at unaligned p: c = 32 2.4-2.7 -> 4.9-5.4 TB/s, c = 64 1.1 -> 4.7-5.5, c = 16 3.1-3.5 -> 3.7-3.9; at c = 8
+    // the tiled kernel is twice as fast)
+    const int min_c = g_tune_tc_min_c > 0 ? g_tune_tc_min_c : (aligned ? 24 : 16);
+    if (a.J < min_c || a.J > 128) return false;
+    if (a.p >= (int64_t)1 << 31) return false;
+    if (!aligned && g_tune_tc_unaligned_off) return false;
     return get_encode_fn() != nullptr;
 }
 
@@ -456,11 +549,13 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     // tiles of 256 positions where four accumulators fit next to the A operand (c <= 64) and the
     // coefficient copies leave room for 256-position stages; tc_variant 1 forces tiles of 128
     PairParams tp;
+    const bool unal = !rows_aligned(a);
     int halves = (a.J <= 64 && g_tune_tc_variant != 1) ? 2 : 1;
-    int KC = choose_chunk(a, halves, &tp);
-    if (!KC && halves == 2) { halves = 1; KC = choose_chunk(a, halves, &tp); }
+    int KC = choose_chunk(a, halves, &tp, 2, unal);
+    if (!KC && halves == 2) { halves = 1; KC = choose_chunk(a, halves, &tp, 2, unal); }
     if (!KC) return cudaErrorInvalidConfiguration;
     const int tile_w = halves * HALF_M;
+    const int pitch = tile_w + (unal ? 4 : 0);
     tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
     if (tp.NAh > 4) tp.NAh = 4;
     // Issuers per half, measured on B200 with the k-steps issued in bursts of three products: a second one
@@ -474,33 +569,42 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     // Epilogue form, measured on B200 (medians of interleaved runs): a group of four warps per tile parity
     // with hardware barriers is 2-4 % ahead for encode and for 48 or more output columns; with 32 output
     // columns and more than 32 input rows (decode at c <= 32) all eight warps on every tile are 2-4 % ahead.
+    // Unaligned rows are stored row by row, which only the group form does.
     tp.group_epilogue = (tp.Npad <= 32 && tp.K_rows > 32) ? 0 : 1;
     if (g_tune_tc_epi) tp.group_epilogue = g_tune_tc_epi == 2 ? 0 : 1;
+    if (unal) tp.group_epilogue = 1;
     // With 128 output columns the two coefficient copies leave 46-64 KB for the input stages: one group for
     // all tiles needs one output tile less, which buys one or two stages (measured: encode +3 %, decode +7 % at
     // c = 128, nothing at c = 112, -14 % for the encode at c = 80).  tc_epi 3 / 4 force one / two groups.
     tp.epi_groups = (tp.group_epilogue && halves == 1 && tp.Npad > 96) ? 1 : 2;
     if (tp.group_epilogue && g_tune_tc_epi >= 3) tp.epi_groups = g_tune_tc_epi == 3 ? 1 : 2;
     if (tp.epi_groups == 1) {                           // the stages chosen again with what that frees
-        KC = choose_chunk(a, halves, &tp, 1);
+        KC = choose_chunk(a, halves, &tp, 1, unal);
         tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
         if (tp.NAh > 4) tp.NAh = 4;
     }
     tp.tmem_cols = 32;
     while (tp.tmem_cols < halves * (2 * tp.Npad + tp.NAh * 2 * KC)) tp.tmem_cols *= 2;
-    const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * tile_w * 4 +
-                        (size_t)tp.epi_groups * OUT_ROWS * tile_w * 4 + 512;
+    const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * pitch * 4 +
+                        (size_t)tp.epi_groups * OUT_ROWS * pitch * 4 + 512;
 
     CUtensorMap tin, tout;
-    if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, tile_w, KC)) return cudaErrorInvalidValue;
-    if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, tile_w, OUT_ROWS)) return cudaErrorInvalidValue;
+    if (unal) {
+        memset(&tin, 0, sizeof tin);      // no tensor maps: every row travels with a 1-D bulk copy of its own
+        memset(&tout, 0, sizeof tout);
+    } else {
+        if (!make_map(&tin, a.in, a.p, tp.K_rows, a.N, a.in_rstride, a.in_wstride, tile_w, KC)) return cudaErrorInvalidValue;
+        if (!make_map(&tout, a.out, a.p, a.J, a.N, a.out_rstride, a.out_wstride, tile_w, OUT_ROWS)) return cudaErrorInvalidValue;
+    }
 
     tp.tiles_per_worker = (a.p + tile_w - 1) / tile_w;
     tp.total_tiles = tp.tiles_per_worker * a.N;
     int grid = num_sms;
     if ((int64_t)grid > tp.total_tiles) grid = (int)tp.total_tiles;
-    cudaError_t e = halves == 2 ? launch_halves<2>(KC, tin, tout, a, tp, smem, grid, s)
-                                : launch_halves<1>(KC, tin, tout, a, tp, smem, grid, s);
+    cudaError_t e = unal ? (halves == 2 ? launch_halves<2, true>(KC, tin, tout, a, tp, smem, grid, s)
+                                        : launch_halves<1, true>(KC, tin, tout, a, tp, smem, grid, s))
+                         : (halves == 2 ? launch_halves<2, false>(KC, tin, tout, a, tp, smem, grid, s)
+                                        : launch_halves<1, false>(KC, tin, tout, a, tp, smem, grid, s));
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }

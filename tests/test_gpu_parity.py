@@ -495,6 +495,70 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
         cerar_mod.cerar_set_tuning("tc_epi", 0)
 
 
+@pytest.mark.parametrize("N,c,p,offset", [(8, 32, 2049, 0), (3, 16, 1031, 0), (5, 24, 77, 1), (2, 64, 51301, 0), (8, 48, 262, 3),
+                                          (16, 40, 1027, 2), (4, 100, 515, 0), (7, 128, 130, 1), (4, 16, 3, 0), (8, 32, 4100, 2)])
+def test_tensor_core_kernel_on_rows_that_are_not_16_byte_aligned(cerar_mod, N, c, p, offset):
+    """p not a multiple of 4 (or buffers that start `offset` floats off a 16-byte boundary): tensor-map
+    copies cannot address such rows, so the tensor-core kernel brings every row in with a bulk copy of
+    its own and stores the aligned middle of every output row with one, the few elements around it
+    plainly.  Out of place and in place, with guard regions around every buffer: the oracle's stages,
+    and the tiled plain-load kernel (the alternative for such shapes) within 3 x TF32 accuracy."""
+    import torch
+    d = c * p
+    L = c + N - 2
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(7 * N + c))
+    g = _inputs().gradients_numpy(N, d, "normal", seed=4)
+    ora = run_oracle(des.U, des.R, g, 0.5)
+    s = torch_stream()
+    G = 1024                                                   # guard floats around every buffer
+    pat = 0x7FC0DEAD
+    outs = {}
+    try:
+        for off_knob in (0, 1):                                # tensor-core kernel, then the tiled kernel
+            assert cerar_mod.cerar_set_tuning("tc_unaligned_off", off_knob) == 0
+            for inplace in (False, True):
+                plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+                nws = N * (c + N) * p
+                bufs = {}
+                for name, n in (("ws", nws), ("g", N * d), ("out", N * d)):
+                    whole = torch.empty(n + 2 * G + 4, dtype=torch.float32, device="cuda")
+                    whole.view(torch.int32).fill_(pat)
+                    bufs[name] = (whole, whole[G + offset:G + offset + n])
+                ws, gt, out = bufs["ws"][1], bufs["g"][1], bufs["out"][1]
+                ws.fill_(float("nan")); out.fill_(float("nan"))
+                gt.copy_(torch.from_numpy(g).reshape(-1))
+                if inplace:
+                    ws.view(N, c + N, p)[:, N:, :] = gt.view(N, c, p)
+                    gp, gs = ws.data_ptr() + 4 * N * p, (c + N) * p
+                    plan.encode(gp, gs, ws, d, s)
+                else:
+                    plan.encode(gt, d, ws, d, s)
+                Delta = ws.view(N, c + N, p)[:, N:, :].cpu().numpy()
+                for k in range(1, L + 1):
+                    plan.ring_round(ws, d, k, s)
+                if inplace:
+                    plan.decode(ws, gp, gs, d, 0.5, s)
+                    res = ws.view(N, c + N, p)[:, N:, :].reshape(N, d).cpu().numpy()
+                else:
+                    plan.decode(ws, out, d, d, 0.5, s)
+                    res = out.view(N, d).cpu().numpy()
+                torch.cuda.synchronize()
+                plan.device_status(s)
+                for name, (whole, view) in bufs.items():
+                    ints = whole.view(torch.int32)
+                    n = view.numel()
+                    assert bool((ints[:G + offset] == pat).all()), f"store in front of {name}"
+                    assert bool((ints[G + offset + n:] == pat).all()), f"store past the end of {name}"
+                assert rel_l2(Delta, ora["Delta_rows"]) < 2e-6
+                assert max(rel_l2(res[i], ora["out"][i]) for i in range(N)) < OUT_TOL
+                outs[(off_knob, inplace)] = res
+    finally:
+        cerar_mod.cerar_set_tuning("tc_unaligned_off", 0)
+    for inplace in (False, True):
+        assert rel_l2(outs[(0, inplace)], outs[(1, inplace)]) < 3e-6
+    assert np.array_equal(outs[(0, False)], outs[(0, True)])
+
+
 @pytest.mark.parametrize("N,c,p", [(5, 7, 4100), (8, 32, 4), (8, 8, 151556), (16, 20, 40004), (13, 16, 1028),
                                    (32, 32, 260), (33, 34, 36), (6, 6, 37889)])
 def test_round_kernel_forms_leave_the_same_slots(cerar_mod, N, c, p):
