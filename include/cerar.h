@@ -437,8 +437,10 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *                                   default 8192, 32768 from p = 2^23); set before sizing counters
  *   "pdl_off"                       1 = launch without programmatic stream serialization
  *   "serpentine_off"                1 = every ring round walks the positions upwards
- *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24; 16 for
+ *   "tc_min_c"                      smallest c that runs on the tensor-core kernel (default 24; 17 for
  *                                   rows that do not start on 16-byte boundaries)
+ *   "staged_unaligned_off"          1 = rows that do not start on 16-byte boundaries never run on the
+ *                                   staged FMA kernel (they take the tiled plain-load kernel)
  *   "tc_unaligned_off"              1 = rows that do not start on 16-byte boundaries never run on the
  *                                   tensor-core kernel (they take the tiled plain-load kernel)
  *   "rounds_one_launch_off"         1 = cerar_allreduce_sim always launches round by round

@@ -536,9 +536,10 @@ bool tc_eligible(const ContractArgs& a) {
     // Rows that are not 16-byte aligned run the same kernel with per-row bulk copies (no tensor maps); the
     // alternative there is the tiled plain-load kernel, so the tensor cores take over from a smaller c.
     const bool aligned = rows_aligned(a);
-    // (measured at unaligned p: c = 32 2.4-2.7 -> 4.9-5.4 TB/s, c = 64 1.1 -> 4.7-5.5, c = 16 3.1-3.5 -> 3.7-3.9; at c = 8
-    // the tiled kernel is twice as fast)
-    const int min_c = g_tune_tc_min_c > 0 ? g_tune_tc_min_c : (aligned ? 24 : 16);
+    // (measured at unaligned p against the tiled kernel: c = 32 2.4-2.7 -> 4.9-5.4 TB/s, c = 64 1.1 -> 4.7-5.5; up to
+    // c = 16 the staged FMA kernel's realigning form is ahead: 5.6-5.9 against 3.7-3.9 TB/s at c = 16; at c = 20 the
+    // tensor cores are: 4.2 against 3.6-3.9)
+    const int min_c = g_tune_tc_min_c > 0 ? g_tune_tc_min_c : (aligned ? 24 : 17);
     if (a.J < min_c || a.J > 128) return false;
     if (a.p >= (int64_t)1 << 31) return false;
     if (!aligned && g_tune_tc_unaligned_off) return false;

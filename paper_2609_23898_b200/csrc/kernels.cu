@@ -102,7 +102,13 @@ __global__ void __launch_bounds__(256) contract_tile_kernel(const ContractArgs a
 // input rows) safe: tiles are disjoint in positions.
 //
 // shared memory: [full[stages], empty[stages] mbarriers | coef K x Jpad | stages x KC x tile_p]
-template <int PV, int JT, int MAXW>
+//
+// UNAL: rows that do not start on 16-byte boundaries (p not a multiple of 4, offset buffers).  A row's bulk
+// copy then starts at the 16-byte boundary below its first element and the row sits in shared memory with
+// the same offset of 0..3 floats (row pitch tile_p + 4); a thread takes the positions lane, lane + 32, ... of
+// its 128 (instead of four consecutive ones), so that shared-memory reads and global stores of single
+// floats are conflict-free and coalesced.
+template <int PV, int JT, int MAXW, bool UNAL>
 __global__ void __launch_bounds__(32 * (MAXW + 1), 1)
 contract_staged_kernel(const __grid_constant__ ContractArgs a) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -110,6 +116,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
     const int CW = a.slabs * a.jgroups;                 // consumer warps; warp CW is the producer
     const int Jpad = a.jgroups * JT;
     const int stages = a.stages, KC = a.KC, tile_p = a.tile_p;
+    const int pitch = tile_p + (UNAL ? 4 : 0);          // floats between rows of a stage
     const int nkc = (a.K + KC - 1) / KC;
     const int w = blockIdx.y;
 
@@ -119,7 +126,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
     float* stage_s = coef_s + (((size_t)a.K * Jpad + 31) / 32) * 32;
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8u * stages;
     const uint32_t stage0 = smem_u32(stage_s);
-    const uint32_t stage_bytes = (uint32_t)KC * tile_p * 4u;
+    const uint32_t stage_bytes = (uint32_t)KC * pitch * 4u;
 
     // set-up (the only CTA-wide barrier, before any bounded wait)
     if (threadIdx.x == 0) {
@@ -156,16 +163,40 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                 if (!mbar_wait_bounded(empty0 + 8u * s, ph ^ 1u)) { failed = true; break; }
                 const int k0 = kc * KC;
                 const int kcount = (a.K - k0 < KC) ? (a.K - k0) : KC;
-                if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * s, (uint32_t)kcount * valid * 4u);
-                __syncwarp();
-                for (int r = lane; r < kcount; r += 32) {
-                    const int k = k0 + r;
-                    const int row = (k < a.skip_row) ? k : k + a.skip_count;
-                    // (checked build: a copy that is skipped leaves its bytes outstanding, so the consumers' wait
-                    // runs out and the launch ends with both codes' worth of evidence in the status word)
-                    if (CERAR_RANGE_OK(in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, a.in_range, a.status))
-                        bulk_load(stage0 + s * stage_bytes + (uint32_t)r * tile_p * 4u,
-                                  in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, full0 + 8u * s);
+                if constexpr (UNAL) {
+                    uint32_t total = 0;
+                    for (int r = lane; r < kcount; r += 32) {
+                        const int k = k0 + r;
+                        const int row = (k < a.skip_row) ? k : k + a.skip_count;
+                        const uintptr_t first = reinterpret_cast<uintptr_t>(in_w + (int64_t)row * a.in_rstride + q0);
+                        total += (uint32_t)((first & 15u) + valid * 4u + 15u) & ~15u;
+                    }
+                    total = __reduce_add_sync(0xffffffffu, total);
+                    if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * s, total);
+                    __syncwarp();
+                    for (int r = lane; r < kcount; r += 32) {
+                        const int k = k0 + r;
+                        const int row = (k < a.skip_row) ? k : k + a.skip_count;
+                        const uintptr_t first = reinterpret_cast<uintptr_t>(in_w + (int64_t)row * a.in_rstride + q0);
+                        const uint32_t bytes = (uint32_t)((first & 15u) + valid * 4u + 15u) & ~15u;
+                        // (checked build: the row proper is checked, not the up to 12 bytes around it that share its
+                        // 16-byte groups; a skipped copy leaves its bytes outstanding and the consumers' wait runs out)
+                        if (CERAR_RANGE_OK(reinterpret_cast<const void*>(first), valid * 4u, a.in_range, a.status))
+                            bulk_load(stage0 + s * stage_bytes + (uint32_t)r * pitch * 4u,
+                                      reinterpret_cast<const void*>(first & ~(uintptr_t)15), bytes, full0 + 8u * s);
+                    }
+                } else {
+                    if (lane == 0) mbar_arrive_expect_tx(full0 + 8u * s, (uint32_t)kcount * valid * 4u);
+                    __syncwarp();
+                    for (int r = lane; r < kcount; r += 32) {
+                        const int k = k0 + r;
+                        const int row = (k < a.skip_row) ? k : k + a.skip_count;
+                        // (checked build: a copy that is skipped leaves its bytes outstanding, so the consumers' wait
+                        // runs out and the launch ends with both codes' worth of evidence in the status word)
+                        if (CERAR_RANGE_OK(in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, a.in_range, a.status))
+                            bulk_load(stage0 + s * stage_bytes + (uint32_t)r * tile_p * 4u,
+                                      in_w + (int64_t)row * a.in_rstride + q0, valid * 4u, full0 + 8u * s);
+                    }
                 }
             }
         }
@@ -181,8 +212,10 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
         const float* coef_w = coef_s + jg * JT;
         uint32_t pos[PV];
 #pragma unroll
-        for (int v = 0; v < PV; ++v) pos[v] = (uint32_t)(((slab * PV + v) * 32 + lane) * 4);
+        for (int v = 0; v < PV; ++v)     // first position of this thread in vector group v (UNAL: its four are 32 apart)
+            pos[v] = UNAL ? (uint32_t)((slab * PV + v) * 128 + lane) : (uint32_t)(((slab * PV + v) * 32 + lane) * 4);
         float* out_w = a.out + (int64_t)w * a.out_wstride;
+        const float* in_w = a.in + (int64_t)w * a.in_wstride;
         for (int64_t t = blockIdx.x; t < a.tiles_per_worker && !failed; t += gridDim.x) {
             const int64_t q0 = t * tile_p;
             const int64_t rem = a.p - q0;
@@ -197,14 +230,25 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                 if (!mbar_wait_bounded(full0 + 8u * s, ph)) { failed = true; break; }
                 const int k0 = kc * KC;
                 const int kcount = (a.K - k0 < KC) ? (a.K - k0) : KC;
-                const float* st = stage_s + (size_t)s * KC * tile_p;
+                const float* st = stage_s + (size_t)s * KC * pitch;
                 const float* cfa = coef_w + (size_t)k0 * Jpad;
 #pragma unroll 2
                 for (int kk = 0; kk < kcount; ++kk, cfa += Jpad) {
                     float4 x[PV];
+                    if constexpr (UNAL) {
+                        const int k = k0 + kk;
+                        const int row = (k < a.skip_row) ? k : k + a.skip_count;
+                        const uint32_t sh = (uint32_t)((reinterpret_cast<uintptr_t>(in_w + (int64_t)row * a.in_rstride + q0) >> 2) & 3u);
 #pragma unroll
-                    for (int v = 0; v < PV; ++v)
-                        x[v] = *reinterpret_cast<const float4*>(st + (size_t)kk * tile_p + pos[v]);
+                        for (int v = 0; v < PV; ++v) {
+                            const float* xr = st + (size_t)kk * pitch + sh + pos[v];
+                            x[v] = make_float4(xr[0], xr[32], xr[64], xr[96]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < PV; ++v)
+                            x[v] = *reinterpret_cast<const float4*>(st + (size_t)kk * tile_p + pos[v]);
+                    }
 #pragma unroll
                     for (int j4 = 0; j4 < JT / 4; ++j4) {
                         const float4 cc = *reinterpret_cast<const float4*>(cfa + 4 * j4);
@@ -231,8 +275,13 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                 if (jj < a.J) {
                     float* orow = out_w + (int64_t)jj * a.out_rstride + q0;
 #pragma unroll
-                    for (int v = 0; v < PV; ++v)
-                        if (pos[v] < valid && CERAR_RANGE_OK(orow + pos[v], 16, a.out_range, a.status)) {
+                    for (int v = 0; v < PV; ++v) {
+                        if constexpr (UNAL) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                if (pos[v] + 32u * e < valid && CERAR_RANGE_OK(orow + pos[v] + 32 * e, 4, a.out_range, a.status))
+                                    orow[pos[v] + 32 * e] = acc[j][v * 4 + e] * a.scale;
+                        } else if (pos[v] < valid && CERAR_RANGE_OK(orow + pos[v], 16, a.out_range, a.status)) {
                             float4 o;
                             o.x = acc[j][v * 4 + 0] * a.scale;
                             o.y = acc[j][v * 4 + 1] * a.scale;
@@ -240,6 +289,7 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
                             o.w = acc[j][v * 4 + 3] * a.scale;
                             *reinterpret_cast<float4*>(orow + pos[v]) = o;
                         }
+                    }
                 }
             }
         }
@@ -491,13 +541,13 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-template <int PV, int JT, int MAXW>
+template <int PV, int JT, int MAXW, bool UNAL>
 cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
-    auto kern = contract_staged_kernel<PV, JT, MAXW>;
+    auto kern = contract_staged_kernel<PV, JT, MAXW, UNAL>;
     const int Jpad = a.jgroups * JT;
     const size_t bar_bytes = ((2 * (size_t)a.stages * 8 + 127) / 128) * 128;
     const size_t coef_bytes = (((size_t)a.K * Jpad + 31) / 32) * 32 * 4;
-    const size_t smem = bar_bytes + coef_bytes + (size_t)a.stages * a.KC * a.tile_p * 4;
+    const size_t smem = bar_bytes + coef_bytes + (size_t)a.stages * a.KC * (a.tile_p + (UNAL ? 4 : 0)) * 4;
     {   // per device and cheap: set on every launch rather than cached
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -518,6 +568,7 @@ cudaError_t launch_staged(ContractArgs& a, int num_sms, cudaStream_t s) {
 
 // Tuning knobs (0 = default), settable through the C ABI for experiments.
 int g_tune_round_split = 0;
+int g_tune_staged_unaligned_off = 0;
 int g_tune_checked_shrink = 0;   // checked build, tests only: the extents that stores are checked against end this many floats early
 int g_tune_kc = 0, g_tune_stages = 0, g_tune_jt = 0, g_tune_slabs = 0, g_tune_pdl_off = 0, g_tune_serpentine_off = 0,
     g_tune_rounds_one_launch_off = 0, g_tune_rounds_one_launch_mb = 0, g_tune_rounds_multi_form = 0, g_tune_rounds_coop_shape = 0, g_tune_rounds_hints = 0;
@@ -534,17 +585,21 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
     if (mode == KERNEL_TC || (mode == KERNEL_AUTO && tc_eligible(a))) {
         return launch_contract_tc(a, num_sms, s, launches);
     }
-    if (mode == KERNEL_STAGED && !can_stage) return cudaErrorInvalidValue;
-    bool use_staged = can_stage && mode != KERNEL_REF;
+    // rows that are not 16-byte aligned: the same kernel with realigned bulk copies, for the small c that the
+    // tensor-core kernel leaves (tuning: staged_unaligned_off = 1 sends them to the tiled plain-load kernel)
+    const bool unal_staged = !can_stage && !g_tune_staged_unaligned_off && a.J <= 64;
+    if (mode == KERNEL_STAGED && !can_stage && !unal_staged) return cudaErrorInvalidValue;
+    bool use_staged = (can_stage || unal_staged) && mode != KERNEL_REF;
     if (use_staged) {
         // register tile: 8 outputs x 8 positions per thread where J allows it (more resident
         // warps than 16 x 8), 4 x 8 otherwise; as many position slabs as the warp budget
         // allows; stages of about 64 KB (values measured best on B200 for c = 8..24)
         int JT = g_tune_jt ? g_tune_jt : ((a.J % 8 == 0 && a.J >= 16) ? 8 : 4);
+        if (unal_staged && JT != 8) JT = 4;
         // c = 20 (the paper's 8-GPU configuration), decode: all 20 outputs of 4 positions in one
         // thread, so that the data is read from shared memory once instead of by five warps
         // (+7 % measured; neutral for encode, worse for c = 12 and for c padded up to 20)
-        if (!g_tune_jt && a.J == 20 && a.K > a.J) JT = 20;
+        if (!g_tune_jt && a.J == 20 && a.K > a.J && !unal_staged) JT = 20;
         const int PV = (JT == 20) ? 1 : 2;
         a.jgroups = (a.J + JT - 1) / JT;
         const int maxw = (JT == 16 || JT == 20) ? 8 : 16;
@@ -575,10 +630,13 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
             if (smem_of(a.stages) > 220 * 1024) use_staged = false;
             if (use_staged) {
                 cudaError_t e;
-                if (JT == 20) e = launch_staged<1, 20, 8>(a, num_sms, s);
-                else if (JT == 16) e = launch_staged<2, 16, 8>(a, num_sms, s);
-                else if (JT == 8) e = launch_staged<2, 8, 16>(a, num_sms, s);
-                else e = launch_staged<2, 4, 16>(a, num_sms, s);
+                if (!can_stage) {       // rows that are not 16-byte aligned
+                    if (JT == 8) e = launch_staged<2, 8, 16, true>(a, num_sms, s);
+                    else e = launch_staged<2, 4, 16, true>(a, num_sms, s);
+                } else if (JT == 20) e = launch_staged<1, 20, 8, false>(a, num_sms, s);
+                else if (JT == 16) e = launch_staged<2, 16, 8, false>(a, num_sms, s);
+                else if (JT == 8) e = launch_staged<2, 8, 16, false>(a, num_sms, s);
+                else e = launch_staged<2, 4, 16, false>(a, num_sms, s);
                 if (e == cudaSuccess && launches) ++*launches;
                 return e;
             }

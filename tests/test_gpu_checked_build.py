@@ -23,7 +23,7 @@ worst = 0.0
 # FMA contractions (staged, tiled for unaligned rows, plain), the tensor-core kernel's row-by-row copies for
 # unaligned rows, every form of the rounds, ragged tails
 cases = [(4, 8, 4096 + 64, 0), (8, 16, 2052, 0), (5, 7, 1031, 0), (3, 5, 37, 1), (16, 20, 1028, 0), (8, 32, 516, 0),
-         (32, 32, 260, 0), (33, 34, 36, 0), (8, 8, 151556, 0), (8, 32, 517, 0), (4, 64, 1030, 0)]
+         (32, 32, 260, 0), (33, 34, 36, 0), (8, 8, 151556, 0), (8, 32, 517, 0), (4, 64, 1030, 0), (4, 8, 4099, 0)]
 for N, c, p, mode in cases:
     d = c * p
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(N + c))

@@ -84,8 +84,9 @@ def test_surrogate_coefficients_every_stage(cerar_mod, N, c, p, mode):
 
 
 def test_staged_kernel_is_what_runs(cerar_mod):
-    """Forcing the staged kernel must succeed on aligned shapes (so 'auto' is not
-    silently the plain kernel) and fail loudly on shapes it cannot take."""
+    """Forcing the staged kernel must succeed on aligned shapes (so 'auto' is not silently the plain
+    kernel) and on rows that are not 16-byte aligned (its realigning form), and fail loudly where that
+    form is switched off."""
     N, c, p = 4, 8, 4096
     des = Dz.custom_orthogonal(N, c, np.random.default_rng(0))
     g = _inputs().gradients_numpy(N, c * p, "normal", seed=2)
@@ -97,8 +98,13 @@ def test_staged_kernel_is_what_runs(cerar_mod):
     plan2 = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
     plan2.set_kernel_mode(cerar_mod.KERNEL_STAGED)
     g2 = _inputs().gradients_numpy(N, c * 1031, "normal", seed=2)
-    with pytest.raises(cerar_mod.CerarError):
-        run_library(plan2, g2, 1.0)
+    _check_stages(run_library(plan2, g2, 1.0), run_oracle(des.U, des.R, g2, 1.0), OUT_TOL, N)
+    try:
+        assert cerar_mod.cerar_set_tuning("staged_unaligned_off", 1) == 0
+        with pytest.raises(cerar_mod.CerarError):
+            run_library(plan2, g2, 1.0)
+    finally:
+        cerar_mod.cerar_set_tuning("staged_unaligned_off", 0)
 
 
 def test_tensor_core_kernel_is_what_runs(cerar_mod):
@@ -496,13 +502,17 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
 
 
 @pytest.mark.parametrize("N,c,p,offset", [(8, 32, 2049, 0), (3, 16, 1031, 0), (5, 24, 77, 1), (2, 64, 51301, 0), (8, 48, 262, 3),
-                                          (16, 40, 1027, 2), (4, 100, 515, 0), (7, 128, 130, 1), (4, 16, 3, 0), (8, 32, 4100, 2)])
-def test_tensor_core_kernel_on_rows_that_are_not_16_byte_aligned(cerar_mod, N, c, p, offset):
-    """p not a multiple of 4 (or buffers that start `offset` floats off a 16-byte boundary): tensor-map
-    copies cannot address such rows, so the tensor-core kernel brings every row in with a bulk copy of
-    its own and stores the aligned middle of every output row with one, the few elements around it
-    plainly.  Out of place and in place, with guard regions around every buffer: the oracle's stages,
-    and the tiled plain-load kernel (the alternative for such shapes) within 3 x TF32 accuracy."""
+                                          (16, 40, 1027, 2), (4, 100, 515, 0), (7, 128, 130, 1), (4, 16, 3, 0), (8, 32, 4100, 2),
+                                          (4, 8, 1031, 0), (5, 7, 77, 1), (8, 12, 4099, 0), (3, 5, 3, 2), (4, 8, 70000, 3),
+                                          (6, 15, 2050, 0), (4, 17, 1031, 0), (3, 20, 515, 1)])
+def test_contractions_on_rows_that_are_not_16_byte_aligned(cerar_mod, N, c, p, offset):
+    """p not a multiple of 4 (or buffers that start `offset` floats off a 16-byte boundary): neither
+    tensor-map copies nor 16-byte vector accesses can address such rows.  The tensor-core kernel (c > 16)
+    brings every row in with a bulk copy of its own and stores the aligned middle of every output row
+    with one, the few elements around it plainly; the staged FMA kernel (smaller c) realigns its bulk
+    copies the same way and stores single floats.  Out of place and in place, with guard regions around
+    every buffer: the oracle's stages, and the tiled plain-load kernel (what such shapes ran on before,
+    and still do when both forms are switched off) within 3 x TF32 accuracy."""
     import torch
     d = c * p
     L = c + N - 2
@@ -516,6 +526,7 @@ def test_tensor_core_kernel_on_rows_that_are_not_16_byte_aligned(cerar_mod, N, c
     try:
         for off_knob in (0, 1):                                # tensor-core kernel, then the tiled kernel
             assert cerar_mod.cerar_set_tuning("tc_unaligned_off", off_knob) == 0
+            assert cerar_mod.cerar_set_tuning("staged_unaligned_off", off_knob) == 0
             for inplace in (False, True):
                 plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
                 nws = N * (c + N) * p
@@ -554,6 +565,7 @@ def test_tensor_core_kernel_on_rows_that_are_not_16_byte_aligned(cerar_mod, N, c
                 outs[(off_knob, inplace)] = res
     finally:
         cerar_mod.cerar_set_tuning("tc_unaligned_off", 0)
+        cerar_mod.cerar_set_tuning("staged_unaligned_off", 0)
     for inplace in (False, True):
         assert rel_l2(outs[(0, inplace)], outs[(1, inplace)]) < 3e-6
     assert np.array_equal(outs[(0, False)], outs[(0, True)])
