@@ -92,6 +92,14 @@ __global__ void __launch_bounds__(256) contract_tile_kernel(const ContractArgs a
     }
 }
 
+// Two fused multiply-adds with one coefficient in one instruction (fma.rn.f32x2: the same two IEEE results
+// as two fmaf, half the issue slots).  Measured on B200 in the staged contraction: +4 % at c = 16, +10 % for
+// the encode at c = 20.
+__device__ __forceinline__ void fma2(float& a0, float& a1, float c, float x0, float x1) {
+    asm("{\n .reg .b64 ra, rc, rx;\n mov.b64 ra, {%0, %1};\n mov.b64 rc, {%2, %2};\n mov.b64 rx, {%3, %4};\n"
+        " fma.rn.f32x2 ra, rc, rx, ra;\n mov.b64 {%0, %1}, ra;\n}\n"
+        : "+f"(a0), "+f"(a1) : "f"(c), "f"(x0), "f"(x1));
+}
 // ------------------------------------------------------------------ staged contraction
 //
 // grid = (CTAs per worker, N).  CTA (b, w) walks tiles b, b+gridDim.x, ... of
@@ -258,10 +266,8 @@ contract_staged_kernel(const __grid_constant__ ContractArgs a) {
 #pragma unroll
                             for (int v = 0; v < PV; ++v) {
                                 const int j = j4 * 4 + jj;
-                                acc[j][v * 4 + 0] = fmaf(cj[jj], x[v].x, acc[j][v * 4 + 0]);
-                                acc[j][v * 4 + 1] = fmaf(cj[jj], x[v].y, acc[j][v * 4 + 1]);
-                                acc[j][v * 4 + 2] = fmaf(cj[jj], x[v].z, acc[j][v * 4 + 2]);
-                                acc[j][v * 4 + 3] = fmaf(cj[jj], x[v].w, acc[j][v * 4 + 3]);
+                                fma2(acc[j][v * 4 + 0], acc[j][v * 4 + 1], cj[jj], x[v].x, x[v].y);
+                                fma2(acc[j][v * 4 + 2], acc[j][v * 4 + 3], cj[jj], x[v].z, x[v].w);
                             }
                     }
                 }
