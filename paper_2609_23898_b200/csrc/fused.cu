@@ -11,6 +11,7 @@
 #include <cstdint>
 
 #include "kernels.cuh"
+#include "ptx.cuh"
 
 namespace cerar {
 namespace {
@@ -24,17 +25,16 @@ __device__ __forceinline__ void fma_row(float2 (&acc)[C], const float* coef_row,
 #pragma unroll
         for (int j4 = 0; j4 < C / 4; ++j4) {
             const float4 u = *reinterpret_cast<const float4*>(coef_row + 4 * j4);
-            acc[4 * j4 + 0].x = fmaf(u.x, x.x, acc[4 * j4 + 0].x); acc[4 * j4 + 0].y = fmaf(u.x, x.y, acc[4 * j4 + 0].y);
-            acc[4 * j4 + 1].x = fmaf(u.y, x.x, acc[4 * j4 + 1].x); acc[4 * j4 + 1].y = fmaf(u.y, x.y, acc[4 * j4 + 1].y);
-            acc[4 * j4 + 2].x = fmaf(u.z, x.x, acc[4 * j4 + 2].x); acc[4 * j4 + 2].y = fmaf(u.z, x.y, acc[4 * j4 + 2].y);
-            acc[4 * j4 + 3].x = fmaf(u.w, x.x, acc[4 * j4 + 3].x); acc[4 * j4 + 3].y = fmaf(u.w, x.y, acc[4 * j4 + 3].y);
+            ptx::fma2(acc[4 * j4 + 0].x, acc[4 * j4 + 0].y, u.x, x.x, x.y);
+            ptx::fma2(acc[4 * j4 + 1].x, acc[4 * j4 + 1].y, u.y, x.x, x.y);
+            ptx::fma2(acc[4 * j4 + 2].x, acc[4 * j4 + 2].y, u.z, x.x, x.y);
+            ptx::fma2(acc[4 * j4 + 3].x, acc[4 * j4 + 3].y, u.w, x.x, x.y);
         }
     } else {
 #pragma unroll
         for (int j = 0; j < C; ++j) {
             const float u = coef_row[j];
-            acc[j].x = fmaf(u, x.x, acc[j].x);
-            acc[j].y = fmaf(u, x.y, acc[j].y);
+            ptx::fma2(acc[j].x, acc[j].y, u, x.x, x.y);
         }
     }
 }

@@ -92,14 +92,6 @@ __global__ void __launch_bounds__(256) contract_tile_kernel(const ContractArgs a
     }
 }
 
-// Two fused multiply-adds with one coefficient in one instruction (fma.rn.f32x2: the same two IEEE results
-// as two fmaf, half the issue slots).  Measured on B200 in the staged contraction: +4 % at c = 16, +10 % for
-// the encode at c = 20.
-__device__ __forceinline__ void fma2(float& a0, float& a1, float c, float x0, float x1) {
-    asm("{\n .reg .b64 ra, rc, rx;\n mov.b64 ra, {%0, %1};\n mov.b64 rc, {%2, %2};\n mov.b64 rx, {%3, %4};\n"
-        " fma.rn.f32x2 ra, rc, rx, ra;\n mov.b64 {%0, %1}, ra;\n}\n"
-        : "+f"(a0), "+f"(a1) : "f"(c), "f"(x0), "f"(x1));
-}
 // ------------------------------------------------------------------ staged contraction
 //
 // grid = (CTAs per worker, N).  CTA (b, w) walks tiles b, b+gridDim.x, ... of

@@ -54,6 +54,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 __device__ __forceinline__ void bulk_store(void* dst, uint32_t src, uint32_t bytes) {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
 }
+// Two fused multiply-adds with one coefficient in one instruction (fma.rn.f32x2: the same two IEEE results
+// as two fmaf, half the issue slots).  Measured on B200 in the staged contraction: +4 % at c = 16, +10 % for
+// the encode at c = 20.
+__device__ __forceinline__ void fma2(float& a0, float& a1, float c, float x0, float x1) {
+    asm("{\n .reg .b64 ra, rc, rx;\n mov.b64 ra, {%0, %1};\n mov.b64 rc, {%2, %2};\n mov.b64 rx, {%3, %4};\n"
+        " fma.rn.f32x2 ra, rc, rx, ra;\n mov.b64 {%0, %1}, ra;\n}\n"
+        : "+f"(a0), "+f"(a1) : "f"(c), "f"(x0), "f"(x1));
+}
 // Programmatic dependent launch (griddepcontrol): no-ops when the launch has no such dependency.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
