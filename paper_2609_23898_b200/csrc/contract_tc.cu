@@ -559,12 +559,12 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     const int pitch = tile_w + (unal ? 4 : 0);
     tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
     if (tp.NAh > 4) tp.NAh = 4;
-    // Issuers per half, measured on B200 with the k-steps issued in bursts of three products: a second one
-    // (even / odd tiles) pays for 32 output columns once a chunk has more than 4 k-steps (c = 32 decode
-    // 5.3 -> 6.0 TB/s; it costs 2 % below that), and costs 10-15 % for 64 columns (c = 48, 56, 64: the
-    // products are twice as long, two issuers already keep the pipe fed).  With one half per tile two
-    // issuers (even / odd tiles) are the minimum that keeps one issuing while the other drains.
-    tp.four_issuers = (halves == 1 || (tp.Npad <= 32 && (tp.K_rows + 7) / 8 > 4)) ? 1 : 0;
+    // Issuers per half: one per accumulator (even / odd tiles).  An issuing thread needs 150-160 clk per product
+    // inside this kernel (a lone thread in an empty SM: 54), so one thread per half holds a tile for 12 x 160 clk
+    // of the ~2400 a tile of 256 positions may take.  Measured on B200 (medians of interleaved runs, group
+    // epilogue): encode +7 % at c = 32, +16 % at c = 24, +34 % at c = 28; c = 48, 56: +4..+15 %; c = 40, 64: 0..+4 %.
+    // (With the eight-warp epilogue of earlier versions a second issuer cost 10-15 % at 64 columns.)
+    tp.four_issuers = 1;
     if (g_tune_tc_variant == 2) tp.four_issuers = 0;
     if (g_tune_tc_variant == 3) tp.four_issuers = 1;
     // Epilogue form, measured on B200 (medians of interleaved runs): a group of four warps per tile parity
