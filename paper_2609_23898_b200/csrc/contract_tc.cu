@@ -567,11 +567,11 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     tp.four_issuers = 1;
     if (g_tune_tc_variant == 2) tp.four_issuers = 0;
     if (g_tune_tc_variant == 3) tp.four_issuers = 1;
-    // Epilogue form, measured on B200 (medians of interleaved runs): a group of four warps per tile parity
-    // with hardware barriers is 2-4 % ahead for encode and for 48 or more output columns; with 32 output
-    // columns and more than 32 input rows (decode at c <= 32) all eight warps on every tile are 2-4 % ahead.
+    // Epilogue form, measured on B200 (medians of interleaved runs, c = 24 .. 128, one issuer per accumulator): a
+    // group of four warps per tile parity with hardware barriers is ahead of all eight warps on every tile by
+    // 3-10 % for most shapes (c = 32: within 3 % either way), so it is the default; tc_epi = 2 selects the other.
     // Unaligned rows are stored row by row, which only the group form does.
-    tp.group_epilogue = (tp.Npad <= 32 && tp.K_rows > 32) ? 0 : 1;
+    tp.group_epilogue = 1;
     if (g_tune_tc_epi) tp.group_epilogue = g_tune_tc_epi == 2 ? 0 : 1;
     if (unal) tp.group_epilogue = 1;
     // With 128 output columns the two coefficient copies leave 46-64 KB for the input stages: one group for
