@@ -569,9 +569,11 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     if (g_tune_tc_variant == 3) tp.four_issuers = 1;
     // Epilogue form, measured on B200 (medians of interleaved runs, c = 24 .. 128, one issuer per accumulator): a
     // group of four warps per tile parity with hardware barriers is ahead of all eight warps on every tile by
-    // 3-10 % for most shapes (c = 32: within 3 % either way), so it is the default; tc_epi = 2 selects the other.
-    // Unaligned rows are stored row by row, which only the group form does.
-    tp.group_epilogue = 1;
+    // 3-10 % for most shapes, so it is the default; the exception is c = 32 exactly (a full block of 32 output rows),
+    // where the eight-warp form is ahead by 3-4 % for the encode and 0-2 % for the decode, at d = 2^27 and at config 3's
+    // full size alike.  tc_epi = 1 / 2 force one or the other.  Unaligned rows are stored row by row, which only the
+    // group form does.
+    tp.group_epilogue = a.J == 32 ? 0 : 1;
     if (g_tune_tc_epi) tp.group_epilogue = g_tune_tc_epi == 2 ? 0 : 1;
     if (unal) tp.group_epilogue = 1;
     // With 128 output columns the two coefficient copies leave 46-64 KB for the input stages: one group for
