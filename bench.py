@@ -489,9 +489,28 @@ def ring_block(world, rank, dev, *, plan=None, d=None, reps=3, timer=None):
              ("peer_round_by_round", lambda: ring.DistributedRing(plan, d, device=dev), {"fused": False}),
              ("peer_fused_rounds", None, {"fused": True})]
     drv = None
+
+    def all_ranks_ok(ok: bool) -> bool:
+        """A form runs only if its set-up worked on EVERY rank: a rank that skipped the timed calls while the
+        others entered their barriers would leave them waiting."""
+        flag = torch.tensor([1 if ok else 0], dtype=torch.int32, device=dev)
+        dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+        return bool(flag.item())
+
     for name, make, kw in forms:
+        err = None
         try:
             drv = make() if make is not None else drv
+            if drv is None:
+                err = "the driver of the form before this one could not be created"
+        except Exception as exc:
+            err = f"{type(exc).__name__}: {exc}"
+            if make is not None:
+                drv = None
+        if not all_ranks_ok(err is None):
+            block[name] = {"error": err or "set-up failed on another rank"}
+            continue
+        try:
             out = torch.empty(d, dtype=torch.float32, device=dev)
             ms = timer(lambda: drv.allreduce(grad, out, 1.0 / N, stream, **kw))
             if on_gpu:
