@@ -571,6 +571,47 @@ def test_contractions_on_rows_that_are_not_16_byte_aligned(cerar_mod, N, c, p, o
     assert np.array_equal(outs[(0, False)], outs[(0, True)])
 
 
+@pytest.mark.parametrize("N,c,p", [(4, 8, 8192), (8, 32, 4100), (16, 128, 516)])
+def test_step_replays_from_a_cuda_graph(cerar_mod, N, c, p):
+    """cerar_encode, cerar_ring_round and cerar_decode are plain stream-ordered launches (with programmatic
+    stream serialization): a caller can capture the whole round-by-round step in a CUDA graph and replay it,
+    which takes the host out of a launch-bound loop (measured: 42 -> 25 us for N=4, c=8, p=8192).  The replay
+    must leave the same bits as the direct calls, also after the inputs have changed."""
+    import torch
+    d = c * p
+    L = c + N - 2
+    des = Dz.custom_orthogonal(N, c, np.random.default_rng(5))
+    plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
+    g = torch.randn(N * d, device="cuda")
+    ws = torch.empty(N * (c + N) * p, device="cuda")
+    out = torch.empty(N * d, device="cuda")
+
+    def step(stream):
+        plan.encode(g, d, ws, d, stream)
+        for k in range(1, L + 1):
+            plan.ring_round(ws, d, k, stream)
+        plan.decode(ws, out, d, d, 0.5, stream)
+
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        step(st.cuda_stream)                                  # warm-up outside the capture
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=st):
+            step(st.cuda_stream)
+        for seed in (1, 2):
+            g.copy_(torch.randn(N * d, device="cuda", generator=torch.Generator(device="cuda").manual_seed(seed)))
+            step(st.cuda_stream)
+            torch.cuda.synchronize()
+            want = out.clone()
+            out.fill_(float("nan"))
+            ws.fill_(float("nan"))
+            graph.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(out, want)
+        plan.device_status(st.cuda_stream)
+
+
 @pytest.mark.parametrize("N,c,p", [(5, 7, 4100), (8, 32, 4), (8, 8, 151556), (16, 20, 40004), (13, 16, 1028),
                                    (32, 32, 260), (33, 34, 36), (6, 6, 37889)])
 def test_round_kernel_forms_leave_the_same_slots(cerar_mod, N, c, p):
