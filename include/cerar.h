@@ -153,10 +153,14 @@ cerar_status_t cerar_design_optimize_h(int N, int c, const double* B, uint64_t s
 
 /* Smallest d' >= d that is a multiple of 4c.  The protocol needs c | d (the caller pads the
  * gradient with zeros, Sec. II); the fast kernels additionally need rows of p = d/c values to
- * start on 16-byte boundaries, i.e. 4 | p.  With c | d but p not a multiple of 4 every call
- * still works, through kernels with plain 4-byte accesses at about half the speed for
- * c <= 32 and less beyond (no tensor cores there): pad to this length instead (zeros in, the
- * padded tail of the result is zero as well). */
+ * start on 16-byte boundaries, i.e. 4 | p.  With c | d but p not a multiple of 4 (or buffers
+ * that start off a 16-byte boundary) every call still works: the contractions then bring
+ * every row in with a copy of its own that starts at the 16-byte boundary below the row and
+ * ends at the one above it, i.e. they may READ up to 12 bytes before and after a row, inside
+ * 16-byte groups that hold at least one element of the buffer (nothing outside a buffer is
+ * ever written), and run at 0.8-0.9 of the aligned speed for c <= 64, far less beyond.
+ * Padding to this length avoids all that (zeros in, the padded tail of the result is zero
+ * as well). */
 int64_t        cerar_padded_length(const cerar_plan_t* plan, int64_t d);
 
 /* Bytes of the device workspace for gradient length d: 4 * N * (c+N) * (d/c);
