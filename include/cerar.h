@@ -428,6 +428,9 @@ int            cerar_set_kernel_mode(cerar_plan_t* plan, int mode);
  *   "tc_variant"                    1 = always tiles of 128 positions (default: tiles of 256
  *                                   positions for c <= 64); 2 / 3 = tiles of 256 with one /
  *                                   two MMA issuers per half
+ *   "tc_split"                      tensor-core kernels with tiles of 256 positions: 1 = each splitter warp
+ *                                   takes all rows of one half of the tile, 2 = half of the rows of both
+ *                                   halves (default: 1 where a tile has two or more chunks)
  *   "tc_epi"                        epilogue of the tensor-core kernels: 1 = a group of four warps
  *                                   per tile parity, 2 = all eight warps on every tile, 3 = one group
  *                                   of four warps for all tiles (one output tile less in shared

@@ -793,6 +793,7 @@ int cerar_set_tuning(const char* name, int value) {
     else if (n == "tc_min_c") cerar::g_tune_tc_min_c = value;
     else if (n == "tc_epi") cerar::g_tune_tc_epi = value;
     else if (n == "tc_unaligned_off") cerar::g_tune_tc_unaligned_off = value;
+    else if (n == "tc_split") cerar::g_tune_tc_split = value;
     else if (n == "staged_unaligned_off") cerar::g_tune_staged_unaligned_off = value;
     else if (n == "round_split") cerar::g_tune_round_split = value;
     else if (n == "checked_shrink") cerar::g_tune_checked_shrink = value;

@@ -67,6 +67,7 @@ struct PairParams {
     int tmem_cols;     // power of two >= HALVES * (2*Npad + NAh*2*KC)
     int four_issuers;  // 1: every half has one issuer per accumulator (even / odd tiles)
     int epi_groups;      // group epilogue: 2 = one group per tile parity, 1 = one group for all tiles (one output tile less)
+    int split_by_half; // two halves per tile: 1 = each splitter warp takes all rows of ONE half (one hand-off per chunk), 0 = half of the rows of both
     int group_epilogue;  // 1: each group of four epilogue warps works on tiles of its own (hardware barriers inside the group)
     int64_t tiles_per_worker;
     int64_t total_tiles;
@@ -119,7 +120,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
     // ---------------- set-up
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) { mbar_init(raw_full + 8u * s, 1); mbar_init(raw_empty + 8u * s, 8); }
-        for (uint32_t b = 0; b < 2u * HALVES * NAh; ++b) mbar_init(a_full + 8u * b, 8);
+        for (uint32_t b = 0; b < 2u * HALVES * NAh; ++b) mbar_init(a_full + 8u * b, (HALVES == 2 && tp.split_by_half) ? 4 : 8);
         for (uint32_t b = 0; b < HALVES * NAh; ++b) mbar_init(a_empty + 8u * b, 1);
         for (int b = 0; b < 2 * HALVES; ++b) { mbar_init(acc_full + 8u * b, 1); mbar_init(acc_empty + 8u * b, tp.group_epilogue ? 4 : 8); }
         for (int b = 0; b < 2; ++b) { mbar_init(out_full + 8u * b, 8); mbar_init(out_free + 8u * b, 1); }
@@ -389,6 +390,62 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap tmap_in, const __grid_con
             const int qd = warp & 3, g = (warp - WARP_SPLIT0) >> 2;
             const int pos = qd * 32 + lane;
             const int r0 = g * KG;
+            if (HALVES == 2 && tp.split_by_half) {
+                // warp group g writes half g: all rows of the chunk in two batches of KG, one wait for the A buffer
+                // and one hand-off to the issuer per chunk (every warp still meets every chunk, so no barrier is
+                // ever a phase ahead of a waiter)
+                const int h = g;
+                for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
+                    for (int kc = 0; kc < nkc && !failed; ++kc, ++it) {
+                        const uint32_t s = it % stages, ph = (it / stages) & 1u;
+                        const uint32_t seq = tc * (uint32_t)nkc + (uint32_t)kc;
+                        const uint32_t abi = seq % NAh, pa = (seq / NAh) & 1u;
+                        if (!warp_wait(raw_full + 8u * s, ph)) { failed = true; break; }
+                        const float* colh = raw_s + (size_t)s * (KC * PITCH) + pos + h * HALF_M;
+                        const int rows_left = tp.K_rows - kc * KC;
+                        const int kround = ((rows_left < KC ? rows_left : KC) + 7) / 8 * 8;
+                        const uint32_t ab = (uint32_t)h * NAh + abi;
+#pragma unroll
+                        for (int b = 0; b < 2; ++b) {
+                            const int rb = b * KG;
+                            const int kuse = kround - rb;
+                            uint32_t sh0 = 0, shs = 0;
+                            if constexpr (UNAL) {
+                                shs = (uint32_t)(a.in_rstride & 3);
+                                sh0 = (uint32_t)((reinterpret_cast<uintptr_t>(a.in + (int64_t)w * a.in_wstride) >> 2) + (uint64_t)(t * TILE_W) +
+                                                 (uint64_t)(kc * KC + rb) * (uint64_t)a.in_rstride);
+                            }
+                            uint32_t hi[KG], lo[KG];
+#pragma unroll
+                            for (int k = 0; k < KG; ++k) {
+                                hi[k] = lo[k] = 0u;
+                                if ((k & ~3) < kuse && (!UNAL || rb + k < rows_left)) {
+                                    const float x = colh[(rb + k) * PITCH + (UNAL ? (int)((sh0 + (uint32_t)k * shs) & 3u) : 0)];
+                                    hi[k] = tf32_bits(x);
+                                    lo[k] = tf32_bits(x - __uint_as_float(hi[k]));
+                                }
+                            }
+                            if (b == 1) {
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive(raw_empty + 8u * s);        // this warp has all it needs of the chunk
+                            } else {
+                                if (!warp_wait(a_empty + 8u * ab, pa ^ 1u)) { failed = true; break; }
+                                tc_fence_after();
+                            }
+                            const uint32_t ta = tmem_base + ((uint32_t)(qd * 32) << 16) + a_col0 + ab * (2u * KC) + (uint32_t)rb;
+                            if (kuse > 0) {
+                                tc_st_cols<KG>(ta, hi);
+                                tc_st_cols<KG>(ta + KC, lo);
+                            }
+                        }
+                        if (failed) break;
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(a_full + 8u * ((2u * (uint32_t)h + (tc & 1u)) * NAh + abi));
+                    }
+                }
+            } else
             for (int64_t t = t_begin; t < t_end && !failed; ++t, ++tc) {
                 for (int kc = 0; kc < nkc && !failed; ++kc, ++it) {
                     const uint32_t s = it % stages, ph = (it / stages) & 1u;
@@ -520,7 +577,7 @@ int choose_chunk(const ContractArgs& a, int halves, PairParams* tp, int out_tile
 
 }  // namespace
 
-int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_variant = 0, g_tune_tc_min_c = 0, g_tune_tc_epi = 0, g_tune_tc_unaligned_off = 0;
+int g_tune_tc_kc = 0, g_tune_tc_stages = 0, g_tune_tc_variant = 0, g_tune_tc_min_c = 0, g_tune_tc_epi = 0, g_tune_tc_unaligned_off = 0, g_tune_tc_split = 0;
 
 // Rows that start on 16-byte boundaries everywhere: what tensor-map copies need.
 static bool rows_aligned(const ContractArgs& a) {
@@ -586,6 +643,13 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
         tp.NAh = (512 - 2 * halves * tp.Npad) / (halves * 2 * KC);
         if (tp.NAh > 4) tp.NAh = 4;
     }
+    // Two halves per tile: the two splitter warps of a lane quadrant either take half of a chunk's rows each, for
+    // both halves, or all rows of one half each: then a warp waits for one A buffer and hands over once per chunk
+    // instead of twice.  Measured on B200 where a tile has two or more chunks: c = 40, 48: +9 % (encode), +12 %
+    // (decode); c = 56: +7 % / -1 %; c = 64: -1 % / +22 %; with one chunk per tile (c <= 32) it is neutral, +-2 %.
+    // tc_split forces it off (2) or on (1).
+    tp.split_by_half = (halves == 2 && tp.K_pad / KC >= 2) ? 1 : 0;
+    if (g_tune_tc_split) tp.split_by_half = (halves == 2 && g_tune_tc_split == 1) ? 1 : 0;
     tp.tmem_cols = 32;
     while (tp.tmem_cols < halves * (2 * tp.Npad + tp.NAh * 2 * KC)) tp.tmem_cols *= 2;
     const size_t smem = 1024 + 2 * (size_t)tp.K_pad * tp.Npad * 4 + (size_t)tp.stages * KC * pitch * 4 +

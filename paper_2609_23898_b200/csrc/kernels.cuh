@@ -102,7 +102,7 @@ bool tc_eligible(const ContractArgs& a);
 cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint64_t* launches);
 // Tuning knobs (0 = default), settable through cerar_set_tuning.
 extern int g_tune_kc, g_tune_stages, g_tune_jt, g_tune_slabs, g_tune_tc_kc, g_tune_tc_stages, g_tune_tc_variant,
-           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off, g_tune_serpentine_off, g_tune_tc_min_c, g_tune_tc_epi, g_tune_tc_unaligned_off, g_tune_staged_unaligned_off, g_tune_round_split, g_tune_checked_shrink,
+           g_tune_ring_wait_ms, g_tune_ring_tile, g_tune_pdl_off, g_tune_serpentine_off, g_tune_tc_min_c, g_tune_tc_epi, g_tune_tc_unaligned_off, g_tune_tc_split, g_tune_staged_unaligned_off, g_tune_round_split, g_tune_checked_shrink,
            g_tune_rounds_one_launch_off, g_tune_rounds_one_launch_mb, g_tune_rounds_multi_form, g_tune_rounds_coop_shape, g_tune_rounds_hints;
 cudaError_t launch_round(const RoundArgs& a, cudaStream_t s, uint64_t* launches);
 // Rounds a.k .. k_last in one launch (for states that are cache-resident anyway).

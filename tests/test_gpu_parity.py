@@ -147,6 +147,7 @@ def test_tensor_core_tile_variants(cerar_mod, N, c, p):
         for variant, epi in ((0, 0), (1, 1), (1, 2), (1, 3), (2, 1), (2, 2), (2, 3), (3, 4), (3, 2)):
             assert cerar_mod.cerar_set_tuning("tc_variant", variant) == 0
             assert cerar_mod.cerar_set_tuning("tc_epi", epi) == 0
+            assert cerar_mod.cerar_set_tuning("tc_split", 1 + (variant + epi) % 2) == 0    # both splitter forms
             plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
             plan.set_kernel_mode(cerar_mod.KERNEL_TC)
             res = run_library(plan, g, 0.25)
@@ -155,6 +156,7 @@ def test_tensor_core_tile_variants(cerar_mod, N, c, p):
     finally:
         cerar_mod.cerar_set_tuning("tc_variant", 0)
         cerar_mod.cerar_set_tuning("tc_epi", 0)
+        cerar_mod.cerar_set_tuning("tc_split", 0)
     for other in outs[1:]:
         assert np.array_equal(outs[0]["Delta"], other["Delta"])
         assert np.array_equal(outs[0]["out"], other["out"])
@@ -483,6 +485,7 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
             for mode, v in ((cerar_mod.KERNEL_TC, variant), (cerar_mod.KERNEL_STAGED, 0)):
                 cerar_mod.cerar_set_tuning("tc_variant", v)
                 cerar_mod.cerar_set_tuning("tc_epi", epi)
+                cerar_mod.cerar_set_tuning("tc_split", trial % 3)
                 plan = cerar_mod.Plan.create_custom(N, c, des.U, des.R)
                 plan.set_kernel_mode(mode)
                 ws = torch.full((N * (c + N) * p,), float("nan"), device="cuda")
@@ -499,6 +502,7 @@ def test_tensor_core_against_fma_kernel_on_random_shapes(cerar_mod):
     finally:
         cerar_mod.cerar_set_tuning("tc_variant", 0)
         cerar_mod.cerar_set_tuning("tc_epi", 0)
+        cerar_mod.cerar_set_tuning("tc_split", 0)
 
 
 @pytest.mark.parametrize("N,c,p,offset", [(8, 32, 2049, 0), (3, 16, 1031, 0), (5, 24, 77, 1), (2, 64, 51301, 0), (8, 48, 262, 3),
