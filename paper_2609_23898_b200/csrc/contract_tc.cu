@@ -621,16 +621,18 @@ cudaError_t launch_contract_tc(ContractArgs a, int num_sms, cudaStream_t s, uint
     // of the ~2400 a tile of 256 positions may take.  Measured on B200 (medians of interleaved runs, group
     // epilogue): encode +7 % at c = 32, +16 % at c = 24, +34 % at c = 28; c = 48, 56: +4..+15 %; c = 40, 64: 0..+4 %.
     // (With the eight-warp epilogue of earlier versions a second issuer cost 10-15 % at 64 columns.)
-    tp.four_issuers = 1;
+    // The exception, measured inside the pipeline (whole steps: encode, rounds, decode, as bench.py runs them, at config
+    // 3's full size) is c = 32: one issuer per half with the group epilogue, encode 6.15 against 5.85 TB/s, decode 5.95
+    // against 5.90.  (Back to back, in loops of one kernel under the power cap, the same shape prefers the second
+    // pair by 7 %: what counts is the kernel between the launches it runs between.)
+    tp.four_issuers = a.J == 32 ? 0 : 1;
     if (g_tune_tc_variant == 2) tp.four_issuers = 0;
     if (g_tune_tc_variant == 3) tp.four_issuers = 1;
     // Epilogue form, measured on B200 (medians of interleaved runs, c = 24 .. 128, one issuer per accumulator): a
     // group of four warps per tile parity with hardware barriers is ahead of all eight warps on every tile by
-    // 3-10 % for most shapes, so it is the default; the exception is c = 32 exactly (a full block of 32 output rows),
-    // where the eight-warp form is ahead by 3-4 % for the encode and 0-2 % for the decode, at d = 2^27 and at config 3's
-    // full size alike.  tc_epi = 1 / 2 force one or the other.  Unaligned rows are stored row by row, which only the
-    // group form does.
-    tp.group_epilogue = a.J == 32 ? 0 : 1;
+    // 3-10 % for most shapes and never behind inside the pipeline, so it is the default; tc_epi = 2 selects the
+    // eight-warp form.  Unaligned rows are stored row by row, which only the group form does.
+    tp.group_epilogue = 1;
     if (g_tune_tc_epi) tp.group_epilogue = g_tune_tc_epi == 2 ? 0 : 1;
     if (unal) tp.group_epilogue = 1;
     // With 128 output columns the two coefficient copies leave 46-64 KB for the input stages: one group for
