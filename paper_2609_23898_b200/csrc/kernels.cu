@@ -593,6 +593,9 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
         // warps than 16 x 8), 4 x 8 otherwise; as many position slabs as the warp budget
         // allows; stages of about 64 KB (values measured best on B200 for c = 8..24)
         int JT = g_tune_jt ? g_tune_jt : ((a.J % 8 == 0 && a.J >= 16) ? 8 : 4);
+        // decode at c = 16 (19-31 input rows): 4 outputs per thread and twice the warps per output group, measured inside
+        // the pipeline: +4 % at p = 2^20, +10 % at p = 2^22 (the encode loses 5 % with it and keeps 8)
+        if (!g_tune_jt && a.J == 16 && a.K > a.J) JT = 4;
         if (unal_staged && JT != 8) JT = 4;
         // c = 20 (the paper's 8-GPU configuration), decode: all 20 outputs of 4 positions in one
         // thread, so that the data is read from shared memory once instead of by five warps
