@@ -19,22 +19,26 @@
 // contiguous range per CTA, so every SM is busy whatever N is; a range that crosses a worker
 // boundary is processed in two segments (the coefficients are per worker).
 //   warp 0        producer: one TMA load per chunk ([KC rows] x [tile positions])
-//   warps 11-18   splitter: thread = position (of every half); the two warps of a lane
-//                 quadrant take one half of the chunk's rows each; values are split into
+//   warps 11-18   splitter: thread = position; the two warps of a lane quadrant take one half of
+//                 the chunk's rows each, for every half of the tile (or, with two halves and two
+//                 or more chunks per tile, all rows of one half each); values are split into
 //                 tf32 hi | lo and written to tensor memory (tcgen05.st), where they are
 //                 the A operand of their half: shared memory is read once per element
 //   warps 1, 2    MMA issuers (one lane each) for half 0 / 1, even tiles; warps 19, 20 the
-//                 same for the odd tiles when a tile has more than four k-steps (an issuing
-//                 thread is limited by its own instruction stream, not by the tensor pipe):
+//                 same for the odd tiles (an issuing thread is limited by its own instruction
+//                 stream, not by the tensor pipe; at c = 32 warps 1, 2 take all tiles):
 //                 tcgen05.mma kind::tf32, A from TMEM, B = the coefficients (hi and lo
 //                 copies) in shared memory, M=128, N=Npad, K=8; two accumulators per half,
 //                 so that the epilogue of one tile overlaps the products of the next;
 //                 warp 1 owns the TMEM allocation
 //   warps 3-10    epilogue: tcgen05.ld, scale, transpose through a shared-memory tile, one TMA
-//                 store per 32 output rows.  Two forms: all eight warps on every tile (16 of
-//                 every 32 rows per warp, two tiles handed round with mbarriers), or one group
-//                 of four warps per tile parity, each with a tile of its own and a hardware
-//                 barrier inside the group (no polling between the warps)
+//                 store per 32 output rows.  One group of four warps per tile parity, each with
+//                 a tile of its own and a hardware barrier inside the group (no polling between
+//                 the warps); one group for all tiles at 128 output columns; or, on request,
+//                 all eight warps on every tile (16 of every 32 rows per warp, two tiles handed
+//                 round with mbarriers)
+// Rows that do not start on 16-byte boundaries run the same kernel with UNAL = true: per-row bulk
+// copies instead of tensor-map copies (see the kernel).
 // Every wait is bounded; a wait that runs out sets the status word and the CTA leaves
 // through the common exit, where tensor memory is freed.
 #include <cuda.h>
