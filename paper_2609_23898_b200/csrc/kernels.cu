@@ -619,7 +619,9 @@ cudaError_t launch_contract(ContractArgs a, int mode, int num_sms, cudaStream_t 
                 if (a.KC > fit) a.KC = fit < 2 ? 2 : fit;
             }
             if (a.KC > a.K) a.KC = a.K;
-            a.stages = g_tune_stages ? g_tune_stages : 3;
+            // three stages; two for c <= 8 (a tile is one or two chunks): measured inside the pipeline at c = 8, +4..+7 %
+            // for both contractions (at c = 16, where the decode has three or four chunks per tile, two stages cost it 10-25 %)
+            a.stages = g_tune_stages ? g_tune_stages : (a.J <= 8 ? 2 : 3);
             a.tiles_per_worker = (int)((a.p + a.tile_p - 1) / a.tile_p);
             a.total_tiles = (int64_t)a.tiles_per_worker * a.N;
             // shared memory must fit: shrink the pipeline, then give up
